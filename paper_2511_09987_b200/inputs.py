@@ -1,0 +1,172 @@
+"""Seeded synthetic operands for the recurrence-matmul workloads.
+
+This module only makes input data (host numpy arrays) and describes the five
+workload configurations; it contains none of the recurrence's arithmetic.  The
+same bytes are handed to the CUDA library and to whatever checks it.
+
+Generator: counter based, so any element can be regenerated independently.
+``bits(seed, tensor, index) = splitmix64_finalise(seed * C1 + tensor * C2 + index * GOLDEN)``
+with the published splitmix64 finaliser.  From the 64 bits:
+
+* uniform in ``[0,1)``: the top 24 bits times ``2**-24``, mapped to ``[lo,hi)``;
+* normal: Box-Muller in float64 from two uniforms taken from the top and the
+  bottom 32 bits of the same word (``u1`` shifted into ``(0,1]``), scaled by the
+  standard deviation;
+* int8: the top byte reinterpreted as a signed byte, uniform on ``[-128,127]``.
+
+bf16 operands are the float32 values rounded to nearest-even and returned as
+``uint16`` bit patterns.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+_GOLDEN = np.uint64(0x9E3779B97F4A7C15)
+_C1 = np.uint64(0xD1342543DE82EF95)
+_C2 = np.uint64(0xA0761D6478BD642F)
+_M1 = np.uint64(0xBF58476D1CE4E5B9)
+_M2 = np.uint64(0x94D049BB133111EB)
+_CHUNK = 1 << 22
+
+TENSOR_A = 0
+TENSOR_B = 1
+
+
+def _bits(seed: int, tensor: int, start: int, count: int) -> np.ndarray:
+    with np.errstate(over="ignore"):
+        idx = np.arange(start, start + count, dtype=np.uint64)
+        z = np.uint64(seed) * _C1 + np.uint64(tensor) * _C2 + (idx + np.uint64(1)) * _GOLDEN
+        z = (z ^ (z >> np.uint64(30))) * _M1
+        z = (z ^ (z >> np.uint64(27))) * _M2
+        z = z ^ (z >> np.uint64(31))
+    return z
+
+
+def _fill(n: int, fn, dtype) -> np.ndarray:
+    out = np.empty(n, dtype=dtype)
+    for s in range(0, n, _CHUNK):
+        c = min(_CHUNK, n - s)
+        out[s:s + c] = fn(s, c)
+    return out
+
+
+def uniform_f32(seed: int, tensor: int, n: int, lo: float, hi: float) -> np.ndarray:
+    def fn(s, c):
+        u = (_bits(seed, tensor, s, c) >> np.uint64(40)).astype(np.float64) * 2.0 ** -24
+        return (lo + (hi - lo) * u).astype(np.float32)
+    return _fill(n, fn, np.float32)
+
+
+def normal_f32(seed: int, tensor: int, n: int, std: float) -> np.ndarray:
+    def fn(s, c):
+        z = _bits(seed, tensor, s, c)
+        u1 = ((z >> np.uint64(32)).astype(np.float64) + 1.0) * 2.0 ** -32      # (0,1]
+        u2 = (z & np.uint64(0xFFFFFFFF)).astype(np.float64) * 2.0 ** -32       # [0,1)
+        return (std * np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)).astype(np.float32)
+    return _fill(n, fn, np.float32)
+
+
+def uniform_i8(seed: int, tensor: int, n: int) -> np.ndarray:
+    def fn(s, c):
+        return (_bits(seed, tensor, s, c) >> np.uint64(56)).astype(np.uint8).view(np.int8)
+    return _fill(n, fn, np.int8)
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to bf16 (nearest, ties to even); returns uint16 bit patterns."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    bias = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    return ((u + bias) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(h: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(h, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+@dataclass(frozen=True)
+class Workload:
+    """One synthetic configuration.  ``dtype`` is ``"f32"``, ``"bf16"`` or ``"i8"``."""
+    name: str
+    dtype: str
+    M: int
+    N: int
+    K: int
+    seed: int
+    batch: int = 1
+    b_col_major: bool = False
+    fixed_k_order: bool = False
+    a_dist: tuple = ("uniform", -1.0, 1.0)
+    b_dist: tuple = ("uniform", -1.0, 1.0)
+
+    @property
+    def macs(self) -> int:
+        return self.batch * self.M * self.N * self.K
+
+    @property
+    def in_bytes(self) -> int:
+        return {"f32": 4, "bf16": 2, "i8": 1}[self.dtype]
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        """A and B read once, C written once."""
+        return self.batch * ((self.M * self.K + self.K * self.N) * self.in_bytes + self.M * self.N * 4)
+
+
+WORKLOADS = {
+    # fp32 64^3, uniform[-1,1), strict increasing-k accumulation
+    "c1": Workload("c1", "f32", 64, 64, 64, seed=0, fixed_k_order=True),
+    # int8 x int8 -> int32, 4096^3, A row-major, B column-major
+    "c2": Workload("c2", "i8", 4096, 4096, 4096, seed=1, b_col_major=True,
+                   a_dist=("int8",), b_dist=("int8",)),
+    # bf16 in, fp32 accumulate/out, 8192^3, normal(0,1)
+    "c3": Workload("c3", "bf16", 8192, 8192, 8192, seed=2, a_dist=("normal", 1.0), b_dist=("normal", 1.0)),
+    # fp32 tall-skinny, A uniform[-1,1), B normal(0, sigma=0.1)
+    "c4": Workload("c4", "f32", 65536, 256, 256, seed=3, b_dist=("normal", 0.1)),
+    # 1024 independent bf16 problems of 256^3, uniform[-2,2)
+    "c5": Workload("c5", "bf16", 256, 256, 256, seed=4, batch=1024,
+                   a_dist=("uniform", -2.0, 2.0), b_dist=("uniform", -2.0, 2.0)),
+}
+
+
+def _draw(dist: tuple, dtype: str, seed: int, tensor: int, n: int) -> np.ndarray:
+    if dist[0] == "int8":
+        if dtype != "i8":
+            raise ValueError("int8 distribution needs dtype i8")
+        return uniform_i8(seed, tensor, n)
+    if dist[0] == "uniform":
+        x = uniform_f32(seed, tensor, n, dist[1], dist[2])
+    elif dist[0] == "normal":
+        x = normal_f32(seed, tensor, n, dist[1])
+    else:
+        raise ValueError("unknown distribution %r" % (dist,))
+    if dtype == "f32":
+        return x
+    if dtype == "bf16":
+        return f32_to_bf16_bits(x)
+    # small integers for int8 tests drawn from a float distribution are not provided
+    raise ValueError("distribution %r not available for dtype %r" % (dist, dtype))
+
+
+def make_operands(w: Workload):
+    """Host arrays ``(A, B)`` for a workload.
+
+    ``A`` has shape ``[batch,] M, K``.  ``B`` has shape ``[batch,] K, N`` or, when
+    ``w.b_col_major``, ``[batch,] N, K`` (the element ``B_kj`` stored at ``[j, k]``).
+    The batch axis is present only when ``w.batch > 1``.
+    """
+    A = _draw(w.a_dist, w.dtype, w.seed, TENSOR_A, w.batch * w.M * w.K)
+    B = _draw(w.b_dist, w.dtype, w.seed, TENSOR_B, w.batch * w.K * w.N)
+    bshape = (w.N, w.K) if w.b_col_major else (w.K, w.N)
+    if w.batch > 1:
+        return A.reshape(w.batch, w.M, w.K), B.reshape((w.batch,) + bshape)
+    return A.reshape(w.M, w.K), B.reshape(bshape)
+
+
+def scaled(w: Workload, **kw) -> Workload:
+    """A copy of ``w`` with some fields replaced (smaller shapes of the same recipe)."""
+    d = dict(name=w.name, dtype=w.dtype, M=w.M, N=w.N, K=w.K, seed=w.seed, batch=w.batch, b_col_major=w.b_col_major,
+             fixed_k_order=w.fixed_k_order, a_dist=w.a_dist, b_dist=w.b_dist)
+    d.update(kw)
+    return Workload(**d)
