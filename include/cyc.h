@@ -1,0 +1,132 @@
+/*
+ * cyc.h -- C ABI of the B200 (sm_100a) evaluator of the weight-stationary
+ * systolic matrix-multiply recurrence
+ *
+ *        [i,k]_C <- [i,k-1]_C + [i,k]_W * [i,k]_B ,   [i,0-1]_C = 0 ,
+ *        C_ij    <- [i,k_end]_C
+ *
+ * (weight-stationary program of Section "Space-time Mappings of Dataflow
+ * Recurrences" and the nine per-cell programs of Figure "perPE": W = A_ik is
+ * held in cell (i,k), B_kj is injected at the north boundary and copied along
+ * i, the partial sum moves along k, and C_ij = sum_k A_ik B_kj leaves the
+ * array at k_end -- the export rule of Section "Explicit Communication and
+ * Loads into Iteration Space").
+ *
+ * All pointers are DEVICE pointers unless a function says otherwise.  The
+ * caller owns every buffer; the library reads A and B, overwrites C, and keeps
+ * no reference once the kernels it enqueued have completed.  C must not
+ * overlap A or B.  Calls are asynchronous: work is enqueued on `stream` and the
+ * function returns without synchronising.  The functions never throw, never
+ * abort and are safe to call from several host threads.
+ *
+ * Layouts.  A is [M][K] row-major (K contiguous).  B is [K][N] row-major, or,
+ * with CYC_FLAG_B_COL_MAJOR, stored as [N][K] (element B_kj at B[j*K + k]).
+ * C is [M][N] row-major and is written completely (the recurrence starts from
+ * zero; there is no accumulate-into-C).
+ *
+ * Arithmetic.
+ *   CYC_F32       A, B, C float.   With CYC_FLAG_FIXED_K_ORDER every C_ij is
+ *                 the chain acc = fma(A_ik, B_kj, acc), k = 0,1,..,K-1, acc
+ *                 starting at +0 (one rounding per cell, round to nearest
+ *                 even): bit-reproducible.  Without the flag the library may
+ *                 evaluate the sum on tensor cores with each operand split
+ *                 into two TF32 parts and fp32 accumulation (error well inside
+ *                 1e-5 * sum_k |A_ik||B_kj|).
+ *   CYC_BF16_F32  A, B bfloat16; products exact; fp32 accumulation; C float.
+ *                 k-blocks are accumulated in increasing order by one owner
+ *                 per C_ij (never split-K, never atomics), so results are
+ *                 run-to-run identical with or without the flag.
+ *   CYC_I8_I32    A, B signed 8-bit; C int32; exact for K <= 131071.
+ */
+#ifndef CYC_H_
+#define CYC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CYC_F32 = 0,
+    CYC_BF16_F32 = 1,
+    CYC_I8_I32 = 2
+} cyc_dtype_t;
+
+enum {
+    CYC_FLAG_FIXED_K_ORDER = 1u, /* deterministic; one owner per C_ij; k strictly increasing */
+    CYC_FLAG_B_COL_MAJOR = 2u    /* B is stored as [N][K] */
+};
+
+typedef enum {
+    CYC_OK = 0,
+    CYC_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, unknown dtype or flag bit, bad stride */
+    CYC_ERR_UNSUPPORTED = 2, /* valid request this build cannot serve (e.g. int8 with K > 131071, not an sm_100 device) */
+    CYC_ERR_CUDA = 3,        /* a CUDA runtime or driver call failed; see cyc_last_cuda_error */
+    CYC_ERR_TIMEOUT = 4      /* a bounded device-side wait ran out; C is undefined */
+} cyc_status_t;
+
+/*
+ * Evaluate the recurrence for one problem: C[M][N] = sum_k A[M][K] B[K][N]
+ * (the whole hot path: weight load, B injection, zero initial partial sum,
+ * the multiply-accumulate along k, and the export of C_ij at k_end).
+ *
+ *   M, N, K  >= 1; any values (no tile-multiple requirement).
+ *   dtype    a cyc_dtype_t.
+ *   A, B, C  device pointers, aligned to the element size; 16-byte alignment
+ *            and row pitches that are multiples of 16 bytes select the
+ *            tensor-core kernels, anything else runs on a slower general kernel.
+ *   stream   a cudaStream_t (0 = the default stream).
+ *   flags    OR of CYC_FLAG_*.
+ * Returns a cyc_status_t.  Argument errors are found on the host before any
+ * CUDA call is made.
+ */
+int cyc_recurrence_matmul(int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B, void* C, void* stream,
+                          unsigned flags);
+
+/*
+ * `batch` independent recurrences in one launch: problem b uses
+ * A + b*strideA, B + b*strideB, C + b*strideC (strides in ELEMENTS of the
+ * respective type; 0 selects the contiguous default M*K, K*N, M*N).  Strides
+ * smaller than one matrix are rejected.  Everything else as above.
+ */
+int cyc_recurrence_matmul_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, int64_t strideA,
+                                  const void* B, int64_t strideB, void* C, int64_t strideC, void* stream, unsigned flags);
+
+/*
+ * HOST-memory convenience: A, B and C are host pointers (same layouts).  The
+ * library allocates device buffers, copies A and B in, evaluates the
+ * recurrence, copies C out, frees the buffers and synchronises `stream`
+ * before returning.  For callers without their own device memory management
+ * and for end-to-end timing.
+ */
+int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A_host,
+                               const void* B_host, void* C_host, void* stream, unsigned flags);
+
+/*
+ * Synchronise `stream` and report whether a kernel enqueued by this library on
+ * the current device since the previous call of this function gave up on a
+ * bounded wait.  *out (HOST pointer, may be NULL) receives CYC_OK or
+ * CYC_ERR_TIMEOUT; the return value is CYC_OK unless the synchronisation
+ * itself failed (CYC_ERR_CUDA).
+ */
+int cyc_last_device_status(void* stream, int* out);
+
+/* Name of the kernel family the dispatcher would pick ("simt", "tcgen05",
+ * "tcgen05_3xtf32") for these arguments, or NULL if they are invalid.  Host only. */
+const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
+                           const void* C, unsigned flags);
+
+/* Number of kernels this library has launched in the calling process (monotonic). */
+int64_t cyc_launch_count(void);
+
+/* Text of the last CUDA error this library saw in the calling thread ("" if none). */
+const char* cyc_last_cuda_error(void);
+
+const char* cyc_status_string(int status);
+int cyc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CYC_H_ */

@@ -1,0 +1,149 @@
+"""ctypes binding of ``libcyc.so`` (see ``include/cyc.h``): argument marshalling only.
+
+The functions named ``cyc_*`` take the same arguments as the C entry points
+(integers and raw device/host addresses).  :func:`recurrence_matmul`,
+:func:`recurrence_matmul_batched` and :func:`recurrence_matmul_host` accept torch
+tensors, allocate the result with torch and pass the current torch stream; every
+step of the computation runs in the library's kernels.  There is no CPU fallback:
+if the library is missing or fails to load, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libcyc.so")
+
+CYC_F32, CYC_BF16_F32, CYC_I8_I32 = 0, 1, 2
+CYC_FLAG_FIXED_K_ORDER, CYC_FLAG_B_COL_MAJOR = 1, 2
+CYC_OK, CYC_ERR_INVALID_ARG, CYC_ERR_UNSUPPORTED, CYC_ERR_CUDA, CYC_ERR_TIMEOUT = 0, 1, 2, 3, 4
+DTYPE_CODES = {"f32": CYC_F32, "bf16": CYC_BF16_F32, "i8": CYC_I8_I32}
+
+# every symbol include/cyc.h declares: name -> (restype, argtypes)
+_i64, _int, _u32, _ptr = ctypes.c_int64, ctypes.c_int, ctypes.c_uint, ctypes.c_void_p
+SYMBOLS = {
+    "cyc_recurrence_matmul": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
+    "cyc_recurrence_matmul_batched": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _i64, _ptr, _i64, _ptr, _i64, _ptr, _u32]),
+    "cyc_recurrence_matmul_host": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
+    "cyc_last_device_status": (_int, [_ptr, ctypes.POINTER(ctypes.c_int)]),
+    "cyc_kernel_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
+    "cyc_launch_count": (_i64, []),
+    "cyc_last_cuda_error": (ctypes.c_char_p, []),
+    "cyc_status_string": (ctypes.c_char_p, [_int]),
+    "cyc_version": (_int, []),
+}
+
+
+class CycError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        name = _lib.cyc_status_string(status).decode()
+        super().__init__("cyc: %s (status %d)%s" % (name, status, (": " + detail) if detail else ""))
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("%s is missing: build it with `python -m paper_2511_09987_b200.build`" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    for name, (res, args) in SYMBOLS.items():
+        fn = getattr(lib, name)  # AttributeError if the library does not export it
+        fn.restype, fn.argtypes = res, args
+    return lib
+
+
+_lib = _load()
+
+cyc_recurrence_matmul = _lib.cyc_recurrence_matmul
+cyc_recurrence_matmul_batched = _lib.cyc_recurrence_matmul_batched
+cyc_recurrence_matmul_host = _lib.cyc_recurrence_matmul_host
+cyc_last_device_status = _lib.cyc_last_device_status
+cyc_kernel_for = _lib.cyc_kernel_for
+cyc_launch_count = _lib.cyc_launch_count
+cyc_last_cuda_error = _lib.cyc_last_cuda_error
+cyc_status_string = _lib.cyc_status_string
+cyc_version = _lib.cyc_version
+
+
+def check(status: int) -> None:
+    if status != CYC_OK:
+        raise CycError(status, cyc_last_cuda_error().decode() if status == CYC_ERR_CUDA else "")
+
+
+def _flags(b_col_major: bool, fixed_k_order: bool) -> int:
+    return (CYC_FLAG_B_COL_MAJOR if b_col_major else 0) | (CYC_FLAG_FIXED_K_ORDER if fixed_k_order else 0)
+
+
+def _torch_dtype_code(t) -> int:
+    import torch
+    return {torch.float32: CYC_F32, torch.bfloat16: CYC_BF16_F32, torch.int8: CYC_I8_I32}[t.dtype]
+
+
+def _stream() -> int:
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def recurrence_matmul(A, B, C=None, *, b_col_major: bool = False, fixed_k_order: bool = False):
+    """``C[M,N] = sum_k A[M,K] B[K,N]`` for CUDA tensors (B is ``[N,K]`` when ``b_col_major``)."""
+    import torch
+    if not (A.is_cuda and B.is_cuda and A.is_contiguous() and B.is_contiguous() and A.dim() == 2 and B.dim() == 2):
+        raise ValueError("A and B must be contiguous CUDA matrices")
+    code = _torch_dtype_code(A)
+    if B.dtype != A.dtype:
+        raise ValueError("A and B must have the same dtype")
+    M, K = A.shape
+    N = B.shape[0] if b_col_major else B.shape[1]
+    if (B.shape[1] if b_col_major else B.shape[0]) != K:
+        raise ValueError("inner dimensions differ")
+    if C is None:
+        C = torch.empty((M, N), dtype=torch.int32 if code == CYC_I8_I32 else torch.float32, device=A.device)
+    check(cyc_recurrence_matmul(M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(),
+                                _flags(b_col_major, fixed_k_order)))
+    return C
+
+
+def recurrence_matmul_batched(A, B, C=None, *, b_col_major: bool = False, fixed_k_order: bool = False):
+    """Batched form for contiguous ``A[batch,M,K]``, ``B[batch,K,N]`` (or ``[batch,N,K]``)."""
+    import torch
+    if not (A.is_cuda and B.is_cuda and A.is_contiguous() and B.is_contiguous() and A.dim() == 3 and B.dim() == 3):
+        raise ValueError("A and B must be contiguous CUDA tensors of rank 3")
+    code = _torch_dtype_code(A)
+    batch, M, K = A.shape
+    N = B.shape[1] if b_col_major else B.shape[2]
+    if B.shape[0] != batch or (B.shape[2] if b_col_major else B.shape[1]) != K or B.dtype != A.dtype:
+        raise ValueError("operand shapes or dtypes differ")
+    if C is None:
+        C = torch.empty((batch, M, N), dtype=torch.int32 if code == CYC_I8_I32 else torch.float32, device=A.device)
+    check(cyc_recurrence_matmul_batched(batch, M, N, K, code, A.data_ptr(), 0, B.data_ptr(), 0, C.data_ptr(), 0, _stream(),
+                                        _flags(b_col_major, fixed_k_order)))
+    return C
+
+
+def recurrence_matmul_host(A, B, C, *, b_col_major: bool = False, fixed_k_order: bool = False):
+    """Host tensors in, host tensor out (copies inside the call); ``A`` is ``[M,K]`` or ``[batch,M,K]``."""
+    if A.is_cuda or B.is_cuda or C.is_cuda:
+        raise ValueError("host tensors expected")
+    code = _torch_dtype_code(A)
+    if A.dim() == 2:
+        batch, (M, K) = 1, A.shape
+        N = B.shape[0] if b_col_major else B.shape[1]
+    else:
+        batch, M, K = A.shape
+        N = B.shape[1] if b_col_major else B.shape[2]
+    if C.numel() != batch * M * N or not (A.is_contiguous() and B.is_contiguous() and C.is_contiguous()):
+        raise ValueError("bad result shape or non-contiguous tensors")
+    check(cyc_recurrence_matmul_host(batch, M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(),
+                                     _flags(b_col_major, fixed_k_order)))
+    return C
+
+
+def last_device_status() -> int:
+    out = ctypes.c_int(0)
+    check(cyc_last_device_status(_stream(), ctypes.byref(out)))
+    return out.value
+
+
+def kernel_for(batch, M, N, K, dtype, a_ptr=256, b_ptr=1 << 40, c_ptr=1 << 41, *, b_col_major=False, fixed_k_order=False):
+    r = cyc_kernel_for(batch, M, N, K, DTYPE_CODES.get(dtype, dtype), a_ptr, b_ptr, c_ptr, _flags(b_col_major, fixed_k_order))
+    return r.decode() if r else None

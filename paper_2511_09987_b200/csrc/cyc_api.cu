@@ -1,0 +1,326 @@
+// C ABI of the library: argument validation, kernel selection, tensor-map
+// construction and launches.  See include/cyc.h for the contract.
+#include <atomic>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/cyc.h"
+#include "simt_kernel.cuh"
+#include "umma_kernel.cuh"
+
+namespace cyc {
+
+// raised by a kernel whose bounded wait ran out; one word per device (module scope)
+__device__ int g_device_status = 0;
+
+static std::atomic<long long> g_launches{0};
+static thread_local char g_err[512] = "";
+
+static int cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_err, sizeof g_err, "%s: %s", what, cudaGetErrorString(e));
+    return CYC_ERR_CUDA;
+}
+#define CYC_CUDA(call)                                    \
+    do {                                                  \
+        cudaError_t e_ = (call);                          \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+static int elem_bytes(int dtype) { return dtype == CYC_F32 ? 4 : (dtype == CYC_BF16_F32 ? 2 : 1); }
+
+struct Problem {
+    long long batch, M, N, K;
+    int dtype;
+    const void *A, *B;
+    void* C;
+    long long sA, sB, sC;
+    unsigned flags;
+};
+
+// host-side validation; no CUDA call
+static int validate(const Problem& q) {
+    if (q.dtype != CYC_F32 && q.dtype != CYC_BF16_F32 && q.dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
+    if (q.flags & ~(CYC_FLAG_FIXED_K_ORDER | CYC_FLAG_B_COL_MAJOR)) return CYC_ERR_INVALID_ARG;
+    if (q.batch <= 0 || q.M <= 0 || q.N <= 0 || q.K <= 0) return CYC_ERR_INVALID_ARG;
+    if (!q.A || !q.B || !q.C) return CYC_ERR_INVALID_ARG;
+    if (q.sA < q.M * q.K || q.sB < q.K * q.N || q.sC < q.M * q.N) return CYC_ERR_INVALID_ARG;
+    const int eb = elem_bytes(q.dtype);
+    if ((reinterpret_cast<uintptr_t>(q.A) % eb) || (reinterpret_cast<uintptr_t>(q.B) % eb) || (reinterpret_cast<uintptr_t>(q.C) % 4))
+        return CYC_ERR_INVALID_ARG;
+    // C must not overlap A or B
+    const uintptr_t c0 = reinterpret_cast<uintptr_t>(q.C), c1 = c0 + static_cast<uintptr_t>((q.batch - 1) * q.sC + q.M * q.N) * 4;
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(q.A), a1 = a0 + static_cast<uintptr_t>((q.batch - 1) * q.sA + q.M * q.K) * eb;
+    const uintptr_t b0 = reinterpret_cast<uintptr_t>(q.B), b1 = b0 + static_cast<uintptr_t>((q.batch - 1) * q.sB + q.K * q.N) * eb;
+    if ((c0 < a1 && a0 < c1) || (c0 < b1 && b0 < c1)) return CYC_ERR_INVALID_ARG;
+    if (q.M > 0x7fffffffll || q.N > 0x7fffffffll || q.K > 0x7fffffffll || q.batch > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
+    if (q.dtype == CYC_I8_I32 && q.K > 131071) return CYC_ERR_UNSUPPORTED;  // int32 partial sums stay exact: K * 2^14 < 2^31
+    return CYC_OK;
+}
+
+enum Family { FAM_SIMT = 0, FAM_UMMA = 1, FAM_UMMA_3XTF32 = 2 };
+
+// the tensor-core kernels move tiles with TMA: 16-byte aligned bases and pitches
+static bool tma_ok(const Problem& q) {
+    const int eb = elem_bytes(q.dtype);
+    const bool colmajor = (q.flags & CYC_FLAG_B_COL_MAJOR) != 0;
+    if (reinterpret_cast<uintptr_t>(q.A) % 16 || reinterpret_cast<uintptr_t>(q.B) % 16) return false;
+    if ((q.K * eb) % 16) return false;                  // A pitch (and B pitch when stored [N][K])
+    if (!colmajor && (q.N * eb) % 16) return false;     // B pitch when stored [K][N]
+    if (q.batch > 1 && ((q.sA * eb) % 16 || (q.sB * eb) % 16)) return false;
+    return true;
+}
+
+static Family choose(const Problem& q) {
+    if (q.dtype == CYC_F32) return FAM_SIMT;
+    return tma_ok(q) ? FAM_UMMA : FAM_SIMT;
+}
+
+// ------------------------------------------------------------------ SIMT launch
+template <typename TIn, typename TAcc>
+static int launch_simt(const Problem& q, cudaStream_t st) {
+    SimtParams p;
+    p.A = q.A; p.B = q.B; p.C = q.C;
+    p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
+    p.sA = q.sA; p.sB = q.sB; p.sC = q.sC;
+    const bool colmajor = (q.flags & CYC_FLAG_B_COL_MAJOR) != 0;
+    p.b_sk = colmajor ? 1 : q.N;
+    p.b_sj = colmajor ? q.K : 1;
+    p.tiles_m = static_cast<int>((q.M + SIMT_BM - 1) / SIMT_BM);
+    p.tiles_n = static_cast<int>((q.N + SIMT_BN - 1) / SIMT_BN);
+    const long long blocks = q.batch * p.tiles_m * p.tiles_n;
+    if (blocks > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
+    bool vec = false;
+    if constexpr (sizeof(TIn) == 4) {
+        vec = !colmajor && q.K % 4 == 0 && q.N % 4 == 0 && q.sA % 4 == 0 && q.sB % 4 == 0 && q.sC % 4 == 0 &&
+              reinterpret_cast<uintptr_t>(q.A) % 16 == 0 && reinterpret_cast<uintptr_t>(q.B) % 16 == 0 &&
+              reinterpret_cast<uintptr_t>(q.C) % 16 == 0;
+    }
+    if constexpr (sizeof(TIn) == 4) {
+        if (vec) simt_recurrence_kernel<TIn, TAcc, true><<<static_cast<unsigned>(blocks), SIMT_THREADS, 0, st>>>(p);
+        else simt_recurrence_kernel<TIn, TAcc, false><<<static_cast<unsigned>(blocks), SIMT_THREADS, 0, st>>>(p);
+    } else {
+        simt_recurrence_kernel<TIn, TAcc, false><<<static_cast<unsigned>(blocks), SIMT_THREADS, 0, st>>>(p);
+    }
+    CYC_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static int get_encoder(EncodeTiledFn* out) {
+    static std::mutex mu;
+    static EncodeTiledFn fn = nullptr;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        CYC_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr));
+        if (qr != cudaDriverEntryPointSuccess || !sym) {
+            snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled not available from the driver");
+            return CYC_ERR_CUDA;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    *out = fn;
+    return CYC_OK;
+}
+
+// rank-3 map over a [d2][d1][d0] array (d0 contiguous), box [1][box1][box0], 128-byte swizzle
+static int make_map(CUtensorMap* m, int dtype, const void* base, long long d0, long long d1, long long d2, long long pitch1_elems,
+                    long long pitch2_elems, int box0, int box1) {
+    EncodeTiledFn enc;
+    int rc = get_encoder(&enc);
+    if (rc) return rc;
+    const int eb = elem_bytes(dtype);
+    const CUtensorMapDataType dt = dtype == CYC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                    : (dtype == CYC_BF16_F32 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d0), static_cast<cuuint64_t>(d1), static_cast<cuuint64_t>(d2)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch1_elems) * eb, static_cast<cuuint64_t>(pitch2_elems) * eb};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(box0), static_cast<cuuint32_t>(box1), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+        return CYC_ERR_CUDA;
+    }
+    return CYC_OK;
+}
+
+struct DeviceInfo {
+    int sms = 0, cc_major = 0;
+    bool known = false;
+};
+static int device_info(DeviceInfo* out) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(mu);
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    if (!cache[dev].known) {
+        CYC_CUDA(cudaDeviceGetAttribute(&cache[dev].sms, cudaDevAttrMultiProcessorCount, dev));
+        CYC_CUDA(cudaDeviceGetAttribute(&cache[dev].cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+        cache[dev].known = true;
+    }
+    *out = cache[dev];
+    return CYC_OK;
+}
+
+// ------------------------------------------------------------------ tensor-core launch
+template <int KIND, bool B_MN, int BN, int STAGES>
+static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
+    using Sm = UmmaSmem<KIND, B_MN, BN, STAGES>;
+    constexpr int BK = Sm::BK;
+    constexpr int CH = 128 / UmmaTraits<KIND>::ELEM_BYTES;
+    CUtensorMap tmA, tmB;
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, q.K, q.sA, BK, UMMA_BM);
+    if (rc) return rc;
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, BN);
+    if (rc) return rc;
+
+    UmmaParams p;
+    p.C = q.C;
+    p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
+    p.sC = q.sC;
+    p.tiles_m = static_cast<int>((q.M + UMMA_BM - 1) / UMMA_BM);
+    p.tiles_n = static_cast<int>((q.N + BN - 1) / BN);
+    p.num_tiles = q.batch * p.tiles_m * p.tiles_n;
+    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+
+    auto kern = umma_recurrence_kernel<KIND, B_MN, BN, STAGES>;
+    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Sm::TOTAL));
+    const long long grid = p.num_tiles < sms ? p.num_tiles : sms;
+    kern<<<static_cast<unsigned>(grid), UMMA_THREADS, Sm::TOTAL, st>>>(tmA, tmB, p);
+    CYC_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
+template <int KIND>
+static int launch_umma(const Problem& q, cudaStream_t st) {
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    if (di.cc_major != 10) {
+        snprintf(g_err, sizeof g_err, "tensor-core kernels need an sm_100 device");
+        return CYC_ERR_UNSUPPORTED;
+    }
+    const bool b_mn = (q.flags & CYC_FLAG_B_COL_MAJOR) == 0;
+    const bool wide = q.N > 128;
+    if (b_mn) return wide ? launch_umma_cfg<KIND, true, 256, 4>(q, st, di.sms) : launch_umma_cfg<KIND, true, 128, 6>(q, st, di.sms);
+    return wide ? launch_umma_cfg<KIND, false, 256, 4>(q, st, di.sms) : launch_umma_cfg<KIND, false, 128, 6>(q, st, di.sms);
+}
+
+static int dispatch(const Problem& q, cudaStream_t st) {
+    int rc = validate(q);
+    if (rc) return rc;
+    switch (choose(q)) {
+        case FAM_UMMA:
+            return q.dtype == CYC_BF16_F32 ? launch_umma<KIND_BF16>(q, st) : launch_umma<KIND_I8>(q, st);
+        default:
+            if (q.dtype == CYC_F32) return launch_simt<float, float>(q, st);
+            if (q.dtype == CYC_BF16_F32) return launch_simt<__nv_bfloat16, float>(q, st);
+            return launch_simt<int8_t, int>(q, st);
+    }
+}
+
+}  // namespace cyc
+
+// ====================================================================== C ABI
+using namespace cyc;
+
+extern "C" int cyc_recurrence_matmul(int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B, void* C,
+                                     void* stream, unsigned flags) {
+    Problem q{1, M, N, K, dtype, A, B, C, M * K, K * N, M * N, flags};
+    if (M <= 0 || N <= 0 || K <= 0) return CYC_ERR_INVALID_ARG;
+    return dispatch(q, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int cyc_recurrence_matmul_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A,
+                                             int64_t strideA, const void* B, int64_t strideB, void* C, int64_t strideC,
+                                             void* stream, unsigned flags) {
+    if (batch <= 0 || M <= 0 || N <= 0 || K <= 0 || strideA < 0 || strideB < 0 || strideC < 0) return CYC_ERR_INVALID_ARG;
+    Problem q{batch, M, N, K, dtype, A, B, C, strideA ? strideA : M * K, strideB ? strideB : K * N, strideC ? strideC : M * N, flags};
+    return dispatch(q, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A_host,
+                                          const void* B_host, void* C_host, void* stream, unsigned flags) {
+    if (batch <= 0 || M <= 0 || N <= 0 || K <= 0 || !A_host || !B_host || !C_host) return CYC_ERR_INVALID_ARG;
+    if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
+    if (flags & ~(CYC_FLAG_FIXED_K_ORDER | CYC_FLAG_B_COL_MAJOR)) return CYC_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t eb = static_cast<size_t>(elem_bytes(dtype));
+    const size_t na = static_cast<size_t>(batch) * M * K * eb, nb = static_cast<size_t>(batch) * K * N * eb,
+                 nc = static_cast<size_t>(batch) * M * N * 4;
+    // one allocation, three 256-byte aligned regions
+    const size_t oa = 0, ob = (na + 255) & ~static_cast<size_t>(255), oc = ob + ((nb + 255) & ~static_cast<size_t>(255));
+    uint8_t* d = nullptr;
+    CYC_CUDA(cudaMallocAsync(reinterpret_cast<void**>(&d), oc + nc, st));
+    int rc = CYC_OK;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(d + oa, A_host, na, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(d + ob, B_host, nb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        rc = cuda_fail(e, "cudaMemcpyAsync(host to device)");
+    if (!rc) {
+        Problem q{batch, M, N, K, dtype, d + oa, d + ob, d + oc, M * K, K * N, M * N, flags};
+        rc = dispatch(q, st);
+    }
+    if (!rc && (e = cudaMemcpyAsync(C_host, d + oc, nc, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        rc = cuda_fail(e, "cudaMemcpyAsync(device to host)");
+    cudaFreeAsync(d, st);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess && !rc) rc = cuda_fail(e, "cudaStreamSynchronize");
+    return rc;
+}
+
+extern "C" int cyc_last_device_status(void* stream, int* out) {
+    CYC_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int word = 0;
+    CYC_CUDA(cudaMemcpyFromSymbol(&word, g_device_status, sizeof word));
+    if (word != 0) {
+        const int zero = 0;
+        CYC_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero));
+        snprintf(g_err, sizeof g_err, "device wait ran out (code 0x%x)", word);
+    }
+    if (out) *out = word != 0 ? CYC_ERR_TIMEOUT : CYC_OK;
+    return CYC_OK;
+}
+
+extern "C" const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
+                                      const void* C, unsigned flags) {
+    if (batch <= 0 || M <= 0 || N <= 0 || K <= 0) return nullptr;
+    Problem q{batch, M, N, K, dtype, A, B, const_cast<void*>(C), M * K, K * N, M * N, flags};
+    if (validate(q) != CYC_OK) return nullptr;
+    switch (choose(q)) {
+        case FAM_UMMA: return "tcgen05";
+        case FAM_UMMA_3XTF32: return "tcgen05_3xtf32";
+        default: return "simt";
+    }
+}
+
+extern "C" int64_t cyc_launch_count(void) { return g_launches.load(); }
+extern "C" const char* cyc_last_cuda_error(void) { return g_err; }
+
+extern "C" const char* cyc_status_string(int s) {
+    switch (s) {
+        case CYC_OK: return "ok";
+        case CYC_ERR_INVALID_ARG: return "invalid argument";
+        case CYC_ERR_UNSUPPORTED: return "unsupported";
+        case CYC_ERR_CUDA: return "CUDA error";
+        case CYC_ERR_TIMEOUT: return "device wait timed out";
+        default: return "unknown status";
+    }
+}
+extern "C" int cyc_version(void) { return 100; }

@@ -1,0 +1,75 @@
+"""The C ABI without a GPU: the library loads, exports every symbol the header
+declares, and rejects bad arguments on the host before any CUDA call."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2511_09987_b200 import build
+    build.build()
+    from paper_2511_09987_b200 import binding as b
+    return b
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "cyc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cyc_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(binding):
+    names = declared_symbols()
+    assert "cyc_recurrence_matmul" in names and "cyc_recurrence_matmul_batched" in names
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(binding.SYMBOLS) == names
+
+
+def test_status_strings_and_version(binding):
+    assert binding.cyc_version() >= 100
+    assert binding.cyc_status_string(0) == b"ok"
+    assert binding.cyc_status_string(4) == b"device wait timed out"
+    assert binding.cyc_launch_count() >= 0
+
+
+def test_invalid_arguments_rejected_on_host(binding):
+    b = binding
+    A, B, C = 1 << 20, 1 << 30, 1 << 40   # never dereferenced: validation comes first
+    f = b.cyc_recurrence_matmul
+    assert f(0, 4, 4, 0, A, B, C, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(4, -1, 4, 0, A, B, C, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(4, 4, 0, 0, A, B, C, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(4, 4, 4, 7, A, B, C, None, 0) == b.CYC_ERR_INVALID_ARG          # unknown dtype
+    assert f(4, 4, 4, 0, A, B, C, None, 8) == b.CYC_ERR_INVALID_ARG          # unknown flag
+    assert f(4, 4, 4, 0, None, B, C, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(4, 4, 4, 0, A, None, C, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(4, 4, 4, 0, A, B, None, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(4, 4, 4, 0, A + 2, B, C, None, 0) == b.CYC_ERR_INVALID_ARG      # fp32 operand not 4-byte aligned
+    assert f(4, 4, 4, 0, A, B, A + 16, None, 0) == b.CYC_ERR_INVALID_ARG     # C overlaps A
+    assert f(4, 4, 131072, 2, A, B, C, None, 0) == b.CYC_ERR_UNSUPPORTED     # int32 could overflow
+    g = b.cyc_recurrence_matmul_batched
+    assert g(0, 4, 4, 4, 0, A, 0, B, 0, C, 0, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert g(2, 4, 4, 4, 0, A, 15, B, 0, C, 0, None, 0) == b.CYC_ERR_INVALID_ARG   # stride smaller than a matrix
+    assert g(2, 4, 4, 4, 0, A, 0, B, 0, C, -1, None, 0) == b.CYC_ERR_INVALID_ARG
+    h = b.cyc_recurrence_matmul_host
+    assert h(1, 4, 4, 4, 0, None, B, C, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert h(1, 4, 4, 4, 9, A, B, C, None, 0) == b.CYC_ERR_INVALID_ARG
+
+
+def test_kernel_selection(binding):
+    k = binding.kernel_for
+    assert k(1, 64, 64, 64, "f32", fixed_k_order=True) == "simt"
+    assert k(1, 8192, 8192, 8192, "bf16") == "tcgen05"
+    assert k(1, 4096, 4096, 4096, "i8", b_col_major=True) == "tcgen05"
+    assert k(1024, 256, 256, 256, "bf16") == "tcgen05"
+    assert k(1, 65, 127, 33, "bf16") == "simt"               # pitches not multiples of 16 bytes
+    assert k(1, 64, 64, 64, "bf16", a_ptr=258) == "simt"     # base not 16-byte aligned
+    assert k(1, 64, 64, 64, "bf16", a_ptr=257) is None       # not even element aligned
+    assert k(1, 0, 64, 64, "bf16") is None

@@ -1,0 +1,179 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle
+on the same seeded operands.  int8 must be bit-exact; fp32 within 1e-5 * S and bf16
+within 4e-3 * S, S_ij = sum_k |A_ik||B_kj|; the strict fp32 path must reproduce the
+fused-multiply-add chain bit for bit."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2511_09987_b200 import inputs
+from parity_util import check_workload, gpu_run, to_device
+
+pytestmark = pytest.mark.gpu
+
+W = inputs.WORKLOADS
+
+
+def wl(dtype, M, N, K, seed, batch=1, col=False, fixed=False):
+    if dtype == "i8":
+        return inputs.Workload("t", "i8", M, N, K, seed, batch, col, fixed, ("int8",), ("int8",))
+    return inputs.Workload("t", dtype, M, N, K, seed, batch, col, fixed, ("uniform", -1.0, 1.0), ("normal", 1.0))
+
+
+def family(w):
+    from paper_2511_09987_b200 import binding
+    return binding.kernel_for(w.batch, w.M, w.N, w.K, w.dtype, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
+
+
+# ------------------------------------------------------------------ general (SIMT) kernel
+@pytest.mark.parametrize("shape", [(1, 1, 1), (64, 64, 64), (130, 70, 37), (257, 129, 513), (5, 300, 1), (128, 128, 16),
+                                   (256, 256, 64), (31, 1, 100)])
+@pytest.mark.parametrize("col", [False, True])
+def test_simt_fp32_strict_order_bit_exact(shape, col):
+    w = wl("f32", *shape, seed=11, col=col, fixed=True)
+    assert family(w) == "simt"
+    check_workload(w)   # includes the bit-for-bit comparison with the fused chain
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "i8"])
+@pytest.mark.parametrize("shape", [(1, 1, 1), (65, 127, 33), (200, 131, 77), (3, 5, 300)])
+@pytest.mark.parametrize("col", [False, True])
+def test_simt_unaligned_shapes(dtype, shape, col):
+    w = wl(dtype, *shape, seed=12, col=col)
+    assert family(w) == "simt"
+    A, B = inputs.make_operands(w)
+    C = gpu_run(w, A, B)
+    ref = oracle.collapsed(dtype, A, B, b_col_major=col)
+    assert C.tobytes() == ref.tobytes()   # a strict chain of exact products: identical in both types
+
+
+def test_simt_batched_fp32():
+    w = wl("f32", 70, 40, 50, seed=13, batch=4, fixed=True)
+    check_workload(w)
+
+
+def test_config_c1():
+    assert family(W["c1"]) == "simt"
+    worst = check_workload(W["c1"])
+    assert worst < 1e-5
+
+
+# ------------------------------------------------------------------ tensor-core kernel, small and ragged
+UMMA_SHAPES = [(128, 128, 64), (128, 256, 64), (128, 256, 128), (256, 512, 256), (256, 256, 1024), (300, 520, 200),
+               (129, 264, 72), (200, 96, 136), (1, 8, 8), (127, 392, 520)]
+
+
+@pytest.mark.parametrize("shape", UMMA_SHAPES)
+@pytest.mark.parametrize("col", [False, True])
+def test_umma_bf16(shape, col):
+    w = wl("bf16", *shape, seed=21, col=col)
+    assert family(w) == "tcgen05"
+    check_workload(w)
+
+
+@pytest.mark.parametrize("shape", [(128, 256, 128), (128, 128, 128), (384, 528, 400), (256, 256, 2048), (130, 272, 144),
+                                   (1, 16, 16), (250, 112, 1040)])
+@pytest.mark.parametrize("col", [True, False])
+def test_umma_int8_bit_exact(shape, col):
+    w = wl("i8", *shape, seed=22, col=col)
+    assert family(w) == "tcgen05"
+    check_workload(w)
+
+
+def test_umma_int8_extreme_values():
+    import torch
+    from paper_2511_09987_b200 import binding
+    K = 4096
+    A = torch.full((128, K), -128, dtype=torch.int8, device="cuda")
+    B = torch.full((256, K), -128, dtype=torch.int8, device="cuda")
+    C = binding.recurrence_matmul(A, B, b_col_major=True)
+    assert (C == K * 128 * 128).all().item()       # 2^26: every partial sum stays exact
+    B.fill_(127)
+    assert (binding.recurrence_matmul(A, B, b_col_major=True) == -K * 128 * 127).all().item()
+
+
+def test_umma_closed_forms_bf16():
+    import torch
+    from paper_2511_09987_b200 import binding
+    n = 384
+    X = torch.randint(-64, 64, (n, n), device="cuda").to(torch.bfloat16)
+    I = torch.eye(n, device="cuda", dtype=torch.bfloat16)
+    perm = torch.randperm(n, device="cuda")
+    P = I[perm]
+    assert torch.equal(binding.recurrence_matmul(I, X), X.float())            # A = I  =>  C = B
+    assert torch.equal(binding.recurrence_matmul(X, I), X.float())            # B = I  =>  C = A
+    assert torch.equal(binding.recurrence_matmul(P, X), X.float()[perm])      # row permutation
+    assert torch.equal(binding.recurrence_matmul(X, P, b_col_major=True), X.float()[:, perm])   # stored B^T = P
+    ones = torch.ones((n, n), device="cuda", dtype=torch.bfloat16)
+    assert (binding.recurrence_matmul(ones, ones) == n).all().item()
+
+
+def test_umma_many_tiles_per_cta():
+    # 512 tiles on 148 SMs: every CTA walks 3-4 tiles, both TMEM accumulators and both barrier phases
+    check_workload(wl("bf16", 4096, 4096, 64, seed=23), rows_per_problem=96)
+    check_workload(wl("i8", 4096, 4096, 128, seed=24, col=True), rows_per_problem=96)
+
+
+@pytest.mark.parametrize("dtype,col", [("bf16", False), ("bf16", True), ("i8", True)])
+def test_umma_batched(dtype, col):
+    check_workload(wl(dtype, 256, 256, 256, seed=25, batch=5, col=col))
+    check_workload(wl(dtype, 130, 136, 80, seed=26, batch=3, col=col))
+
+
+def test_batched_with_padding_strides():
+    import torch
+    from paper_2511_09987_b200 import binding
+    w = wl("bf16", 128, 136, 72, seed=27, batch=3)
+    A, B = inputs.make_operands(w)
+    pad = 64
+    dA = torch.zeros((3, 128 * 72 + pad), dtype=torch.bfloat16, device="cuda")
+    dB = torch.zeros((3, 72 * 136 + pad), dtype=torch.bfloat16, device="cuda")
+    dC = torch.full((3, 128 * 136 + pad), -7.0, dtype=torch.float32, device="cuda")
+    dA[:, :128 * 72] = to_device(A, "bf16").reshape(3, -1)
+    dB[:, :72 * 136] = to_device(B, "bf16").reshape(3, -1)
+    binding.check(binding.cyc_recurrence_matmul_batched(3, 128, 136, 72, binding.CYC_BF16_F32, dA.data_ptr(), dA.shape[1],
+                                                        dB.data_ptr(), dB.shape[1], dC.data_ptr(), dC.shape[1],
+                                                        torch.cuda.current_stream().cuda_stream, 0))
+    torch.cuda.synchronize()
+    out = dC.cpu().numpy()
+    assert (out[:, 128 * 136:] == -7.0).all()     # padding untouched
+    ref = oracle.batched_collapsed("bf16", A, B)
+    S = np.stack([oracle.abs_sum_rows("bf16", A[b], B[b])[0] for b in range(3)])
+    assert (np.abs(out[:, :128 * 136].reshape(3, 128, 136) - ref) <= 4e-3 * S).all()
+
+
+def test_results_are_reproducible():
+    for w in (wl("bf16", 512, 512, 512, seed=28), wl("f32", 300, 200, 100, seed=29, fixed=True)):
+        A, B = inputs.make_operands(w)
+        assert gpu_run(w, A, B).tobytes() == gpu_run(w, A, B).tobytes()
+
+
+def test_output_rows_outside_problem_untouched():
+    import torch
+    from paper_2511_09987_b200 import binding
+    # C is exactly M*N: a guard region after it must stay intact for ragged tiles
+    for dtype, M, N, K in (("bf16", 130, 264, 72), ("f32", 130, 70, 37)):
+        w = wl(dtype, M, N, K, seed=30, fixed=(dtype == "f32"))
+        A, B = inputs.make_operands(w)
+        buf = torch.full((M * N + 4096,), 123.0, dtype=torch.float32, device="cuda")
+        binding.recurrence_matmul(to_device(A, dtype), to_device(B, dtype), buf[:M * N].view(M, N), fixed_k_order=w.fixed_k_order)
+        torch.cuda.synchronize()
+        assert (buf[M * N:] == 123.0).all().item()
+
+
+def test_host_entry_point():
+    import torch
+    from paper_2511_09987_b200 import binding
+    w = wl("bf16", 256, 256, 128, seed=31, batch=2)
+    A, B = inputs.make_operands(w)
+    hA = torch.from_numpy(A).view(torch.bfloat16).pin_memory()
+    hB = torch.from_numpy(B).view(torch.bfloat16).pin_memory()
+    hC = torch.empty((2, 256, 256), dtype=torch.float32).pin_memory()
+    binding.recurrence_matmul_host(hA, hB, hC)
+    assert hC.numpy().tobytes() == gpu_run(w, A, B).tobytes()
+
+
+def test_device_status_is_clean():
+    from paper_2511_09987_b200 import binding
+    assert binding.last_device_status() == binding.CYC_OK
+    assert binding.cyc_launch_count() > 0
