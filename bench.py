@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the recurrence-matmul hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+One step = one evaluation of the whole recurrence (weight load, B injection, the
+multiply-accumulate chain along k, export of C) for one workload.  Prints ONE JSON
+line.  `value` is throughput with operands resident in HBM; `e2e` is the same metric
+through the host-buffer entry point, host<->device copies inside the timed region.
+With --gpus N > 1 (under torchrun) every rank runs an independent replica on its own
+GPU ("replicas only": the path has no exchange step) and the values add up.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2511_09987_b200 import inputs  # noqa: E402
+
+# nominal dense tensor ratios relative to bf16 (2.25 PFLOP/s): int8 4.5 POPS, tf32 1.1 PFLOP/s
+NOMINAL_RATIO = {"bf16": 1.0, "i8": 2.0, "tf32": 0.5}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126 * 1024 * 1024
+# FP32 FMA roof: 148 SMs x 128 lanes x 2 flop x max SM clock
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def unit_of(w):
+    return "TOPS" if w.dtype == "i8" else "TFLOPS"
+
+
+def bound_of(w, family):
+    """Which roof bounds the dominant kernel of this workload."""
+    if family == "simt":
+        return "alu"
+    ai = 2.0 * w.macs / w.algorithmic_bytes
+    ridge = {"bf16": 1663e12 / 6.55e12, "i8": 3326e12 / 6.55e12, "f32": 830e12 / 6.55e12}[w.dtype]
+    return "tensor" if ai > ridge else "hbm"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible:
+                try:
+                    phys = int(visible.split(",")[index])
+                except ValueError:
+                    phys = index
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                 "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def cpu_oracle_rate(w, target_seconds=12.0, threads=None):
+    """Time the oracle (collapsed walker, as it stands) on a bounded sample of workload `w`.
+
+    The sample is a prefix of rows of C (problems, for a batched workload; repeats of the whole workload when it
+    is tiny), grown until the walk takes about `target_seconds`."""
+    import oracle
+    threads = threads or os.cpu_count() or 1
+    one = inputs.scaled(w, batch=1)
+    if w.batch > 1:
+        A, B = inputs.make_operands(inputs.scaled(w, batch=min(w.batch, 64)))
+    else:
+        A, B = inputs.make_operands(one)
+
+    def walk(units):
+        t0 = time.perf_counter()
+        if w.batch > 1:
+            for b in range(units):
+                oracle.collapsed(one.dtype, A[b % len(A)], B[b % len(B)], b_col_major=one.b_col_major, threads=threads)
+        elif units <= one.M:
+            oracle.collapsed(one.dtype, A, B, b_col_major=one.b_col_major, rows=np.arange(units), threads=threads)
+        else:
+            for _ in range(units // one.M):
+                oracle.collapsed(one.dtype, A, B, b_col_major=one.b_col_major, threads=threads)
+        return time.perf_counter() - t0
+
+    units = 1 if w.batch > 1 else min(one.M, 2 * threads)
+    limit = w.batch if w.batch > 1 else (one.M if one.macs > 1e8 else one.M * 100000)
+    while True:
+        dt = walk(units)
+        if dt >= 0.5 * target_seconds or units >= limit:
+            break
+        grow = min(8.0, max(2.0, 0.9 * target_seconds / max(dt, 1e-3)))
+        units = int(min(limit, units * grow))
+        if w.batch == 1 and units > one.M:
+            units = (units // one.M) * one.M
+    if w.batch > 1:
+        ops, what = 2.0 * units * one.macs, "problems 0..%d" % (units - 1)
+    elif units <= one.M:
+        ops, what = 2.0 * units * one.N * one.K, "rows 0..%d" % (units - 1)
+    else:
+        ops, what = 2.0 * (units // one.M) * one.macs, "%d repeats of the whole workload" % (units // one.M)
+    sample = "%s of %s (M=%d N=%d K=%d), collapsed walker, %d threads, %.1f s" % (what, w.name, one.M, one.N, one.K, threads, dt)
+    return ops / dt / 1e12, threads, sample, dt
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    threads = os.cpu_count() or 1
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, sample = [], ""
+    for s in range(args.warmup + args.steps):
+        v, threads, sample, _ = cpu_oracle_rate(w, target_seconds=per_step, threads=threads)
+        if s >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    ops = 2.0 * w.macs
+    line = {
+        "impl": "reference", "metric": "recurrence_matmul_throughput", "value": value, "unit": unit_of(w), "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ops / (value * 1e12) * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": {"f32": "f32", "bf16": "bf16", "i8": "i8"}[w.dtype],
+        "data": "synthetic", "config": {"workload": describe(w), "note": "ms_per_step extrapolated from the sampled rate"},
+        "cpu_baseline": {"value": value, "unit": unit_of(w), "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": unit_of(w), "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def describe(w):
+    s = "%s: %s M=%d N=%d K=%d seed=%d" % (w.name, w.dtype, w.M, w.N, w.K, w.seed)
+    if w.batch > 1:
+        s += " batch=%d" % w.batch
+    if w.b_col_major:
+        s += " B column-major"
+    if w.fixed_k_order:
+        s += " fixed-k-order"
+    return s
+
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_09987_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks, peak_kind = load_peaks()
+
+    # ---- operands: generated once on the host, uploaded; several device copies rotate so that
+    # ---- a set has left L2 before it is used again
+    A, B = inputs.make_operands(w)
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i8": torch.int8}[w.dtype]
+    hA = torch.from_numpy(A)
+    hB = torch.from_numpy(B)
+    if w.dtype == "bf16":
+        hA, hB = hA.view(torch.bfloat16), hB.view(torch.bfloat16)
+    hA, hB = hA.pin_memory(), hB.pin_memory()
+    out_dt = torch.int32 if w.dtype == "i8" else torch.float32
+    cshape = (w.batch, w.M, w.N) if w.batch > 1 else (w.M, w.N)
+    set_bytes = w.algorithmic_bytes
+    nsets = int(min(8, max(2, -(-3 * L2_BYTES // set_bytes))))
+    sets = [(hA.cuda(), hB.cuda(), torch.empty(cshape, dtype=out_dt, device="cuda")) for _ in range(nsets)]
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        dA, dB, dC = sets[i % nsets]
+        if w.batch > 1:
+            binding.recurrence_matmul_batched(dA, dB, dC, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
+        else:
+            binding.recurrence_matmul(dA, dB, dC, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
+
+    family = binding.kernel_for(w.batch, w.M, w.N, w.K, w.dtype, sets[0][0].data_ptr(), sets[0][1].data_ptr(),
+                                sets[0][2].data_ptr(), b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = binding.cyc_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = binding.cyc_launch_count() - launches0
+    if binding.last_device_status() != binding.CYC_OK:
+        raise SystemExit("a device-side wait timed out during the benchmark")
+    # keep the GPU loaded a little longer if the timed region was too short to catch a clock sample
+    extra_note = None
+    if len(sampler.samples) < 3:
+        t_end = time.time() + 0.5
+        i = 0
+        while time.time() < t_end:
+            step(i)
+            i += 1
+            if i % 64 == 0:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        extra_note = "timed region shorter than the sampling period; clocks sampled under the same load right after it"
+    clocks = sampler.stop()
+    if extra_note:
+        clocks["note"] = extra_note
+
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    ms_per_step = ms / args.steps
+    ops_step = 2.0 * w.macs
+    value = world * ops_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end through the host entry point (pinned buffers, copies inside the timed region)
+    hC = torch.empty(cshape, dtype=out_dt).pin_memory()
+    e2e_steps = 0 if args.kernel_only else max(3, min(args.steps, 20))
+    for _ in range(0 if args.kernel_only else 2):
+        binding.recurrence_matmul_host(hA, hB, hC, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
+    barrier()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        binding.recurrence_matmul_host(hA, hB, hC, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(1, e2e_steps)
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * ops_step / (float(t.item()) * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant (only) kernel: one launch per step
+    kernel_s = ms_per_step * 1e-3
+    bound = bound_of(w, family)
+    traffic = load_traffic(w)
+    if bound == "hbm":
+        achieved, peak, runit = w.algorithmic_bytes / kernel_s / 1e9, float(peaks["hbm_gbs"]), "GB/s"
+        peak_note = "%s STREAM-style copy" % peak_kind
+    elif bound == "tensor":
+        base = float(peaks["bf16_tflops"]) if args.steps * kernel_s < 1.0 else float(peaks["bf16_tflops_sustained"])
+        which = "burst" if args.steps * kernel_s < 1.0 else "sustained"
+        kind = "tf32" if w.dtype == "f32" else w.dtype
+        achieved, peak, runit = ops_step / kernel_s / 1e12, base * NOMINAL_RATIO[kind], ("TOPS" if w.dtype == "i8" else "TFLOP/s")
+        peak_note = "%s bf16 cuBLAS %s x nominal %s/bf16 ratio %.1f" % (peak_kind, which, kind, NOMINAL_RATIO[kind])
+    else:
+        achieved, peak, runit = ops_step / kernel_s / 1e12, FP32_ALU_TFLOPS, "TFLOP/s"
+        peak_note = "FP32 FMA roof: 148 SMs x 128 lanes x 2 x 1.965 GHz (derived, not measured)"
+    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak, "traffic": traffic,
+                "peak_source": peak_note, "kernel": family, "kernel_us": kernel_s * 1e6}
+
+    if args.kernel_only:
+        cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
+        e2e_value = None
+    else:
+        cpu_v, cores, sample, _ = cpu_oracle_rate(w)
+    if nsets * set_bytes > 2 * L2_BYTES:
+        l2_note = "inputs rotate over %d device copies (%.0f MB in total, larger than the 126 MB L2)" % (nsets, nsets * set_bytes / 1e6)
+    else:
+        l2_note = ("working set of %d rotating copies is %.1f MB, far below L2: this workload is launch/latency-bound, "
+                   "no DRAM figure is claimed for it" % (nsets, nsets * set_bytes / 1e6))
+    line = {
+        "metric": "recurrence_matmul_throughput", "value": value, "unit": unit_of(w), "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": describe(w), "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": l2_note, "kernel": family},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": unit_of(w), "h2d_bytes_per_step": int(hA.numel() * hA.element_size() + hB.numel() * hB.element_size()),
+                "d2h_bytes_per_step": int(hC.numel() * hC.element_size()), "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_v, "unit": unit_of(w), "cores": cores, "kind": "oracle", "sample": sample},
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def kernel_source_digest():
+    """sha256 over the CUDA sources: ties a stored DRAM-traffic figure to the kernels it was taken from."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2511_09987_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(name.encode())
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def load_traffic(w):
+    """DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) for this workload's kernel.
+
+    Read from profiles/dram_traffic.txt, lines `workload bytes digest`; a figure whose digest does not match the
+    current kernel sources is stale and reported as null."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    digest = kernel_source_digest()
+    with open(path) as f:
+        for line in f:
+            parts = line.split()
+            if len(parts) >= 3 and not line.startswith("#") and parts[0] == w.name and parts[2] == digest:
+                return float(parts[1])
+    return None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--shape", default=None, help="M,N,K[,batch]: a smaller case of the workload's recipe (for profiling)")
+    ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs (for profiling)")
+    args = ap.parse_args()
+    w = inputs.WORKLOADS[args.workload]
+    if args.shape:
+        dims = [int(x) for x in args.shape.split(",")]
+        w = inputs.scaled(w, name=w.name + "@" + args.shape, M=dims[0], N=dims[1], K=dims[2], batch=dims[3] if len(dims) > 3 else w.batch)
+    if args.impl == "reference":
+        if args.steps is None:
+            args.steps = 3
+        run_reference(args, w)
+        return
+    if args.steps is None:
+        args.steps = {"c1": 2000, "c2": 2000, "c3": 200, "c4": 1000, "c5": 1000}[w.name.split("@")[0]]
+    run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
