@@ -13,6 +13,7 @@
 #include "../../include/cyc.h"
 #include "simt_kernel.cuh"
 #include "umma_kernel.cuh"
+#include "umma_pair_kernel.cuh"
 
 namespace cyc {
 
@@ -136,14 +137,11 @@ static int get_encoder(EncodeTiledFn* out) {
 }
 
 // rank-3 map over a [d2][d1][d0] array (d0 contiguous), box [1][box1][box0], 128-byte swizzle
-static int make_map(CUtensorMap* m, int dtype, const void* base, long long d0, long long d1, long long d2, long long pitch1_elems,
-                    long long pitch2_elems, int box0, int box1) {
+static int make_map_raw(CUtensorMap* m, CUtensorMapDataType dt, int eb, const void* base, long long d0, long long d1, long long d2,
+                        long long pitch1_elems, long long pitch2_elems, int box0, int box1) {
     EncodeTiledFn enc;
     int rc = get_encoder(&enc);
     if (rc) return rc;
-    const int eb = elem_bytes(dtype);
-    const CUtensorMapDataType dt = dtype == CYC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
-                                                    : (dtype == CYC_BF16_F32 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(d0), static_cast<cuuint64_t>(d1), static_cast<cuuint64_t>(d2)};
     cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch1_elems) * eb, static_cast<cuuint64_t>(pitch2_elems) * eb};
     cuuint32_t box[3] = {static_cast<cuuint32_t>(box0), static_cast<cuuint32_t>(box1), 1};
@@ -155,6 +153,20 @@ static int make_map(CUtensorMap* m, int dtype, const void* base, long long d0, l
         return CYC_ERR_CUDA;
     }
     return CYC_OK;
+}
+
+// operand map (A or B) in the problem's input type
+static int make_map(CUtensorMap* m, int dtype, const void* base, long long d0, long long d1, long long d2, long long pitch1_elems,
+                    long long pitch2_elems, int box0, int box1) {
+    const CUtensorMapDataType dt = dtype == CYC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                    : (dtype == CYC_BF16_F32 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
+    return make_map_raw(m, dt, elem_bytes(dtype), base, d0, d1, d2, pitch1_elems, pitch2_elems, box0, box1);
+}
+
+// result map: C[batch][M][N] of 32-bit words, boxes of 32 rows x 32 columns (128 bytes)
+static int make_c_map(CUtensorMap* m, int dtype, void* C, long long M, long long N, long long batch, long long sC) {
+    const CUtensorMapDataType dt = dtype == CYC_I8_I32 ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    return make_map_raw(m, dt, 4, C, N, M, batch, N, sC, 32, 32);
 }
 
 struct DeviceInfo {
@@ -208,6 +220,44 @@ static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
     return CYC_OK;
 }
 
+// ------------------------------------------------------------------ two-SM tensor-core launch
+template <int KIND, bool B_MN>
+static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms) {
+    constexpr int STAGES = 6;
+    constexpr int BK = 128 / UmmaTraits<KIND>::ELEM_BYTES;
+    constexpr int CH = 128 / UmmaTraits<KIND>::ELEM_BYTES;
+    constexpr int SMEM = pair_smem_bytes<STAGES>();
+    CUtensorMap tmA, tmB, tmC;
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, q.K, q.sA, BK, PAIR_HALF);
+    if (rc) return rc;
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, PAIR_HALF);
+    if (rc) return rc;
+    PairParams p;
+    p.tma_store = (reinterpret_cast<uintptr_t>(q.C) % 16 == 0 && q.N % 4 == 0 && (q.batch == 1 || q.sC % 4 == 0)) ? 1 : 0;
+    if (p.tma_store) {
+        rc = make_c_map(&tmC, q.dtype, q.C, q.M, q.N, q.batch, q.sC);
+        if (rc) return rc;
+    } else {
+        tmC = tmA;  // never used
+    }
+    p.C = q.C;
+    p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
+    p.sC = q.sC;
+    p.tiles_m = static_cast<int>((q.M + 255) / 256);
+    p.tiles_n = static_cast<int>((q.N + PAIR_BN - 1) / PAIR_BN);
+    p.num_tiles = q.batch * p.tiles_m * p.tiles_n;
+    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    auto kern = umma_pair_kernel<KIND, B_MN, STAGES>;
+    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
+    const long long max_pairs = sms / 2;
+    const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
+    kern<<<static_cast<unsigned>(2 * pairs), UMMA_THREADS, SMEM, st>>>(tmA, tmB, tmC, p);
+    CYC_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
 template <int KIND>
 static int launch_umma(const Problem& q, cudaStream_t st) {
     DeviceInfo di;
@@ -218,6 +268,8 @@ static int launch_umma(const Problem& q, cudaStream_t st) {
         return CYC_ERR_UNSUPPORTED;
     }
     const bool b_mn = (q.flags & CYC_FLAG_B_COL_MAJOR) == 0;
+    if (q.M > 128 && q.N > 128)  // enough rows and columns for a CTA pair
+        return b_mn ? launch_pair_cfg<KIND, true>(q, st, di.sms) : launch_pair_cfg<KIND, false>(q, st, di.sms);
     const bool wide = q.N > 128;
     if (b_mn) return wide ? launch_umma_cfg<KIND, true, 256, 4>(q, st, di.sms) : launch_umma_cfg<KIND, true, 128, 6>(q, st, di.sms);
     return wide ? launch_umma_cfg<KIND, false, 256, 4>(q, st, di.sms) : launch_umma_cfg<KIND, false, 128, 6>(q, st, di.sms);
