@@ -14,6 +14,7 @@
 #include "simt_kernel.cuh"
 #include "umma_kernel.cuh"
 #include "umma_pair_kernel.cuh"
+#include "umma_pair_tf32x3_kernel.cuh"
 
 namespace cyc {
 
@@ -78,7 +79,11 @@ static bool tma_ok(const Problem& q) {
 }
 
 static Family choose(const Problem& q) {
-    if (q.dtype == CYC_F32) return FAM_SIMT;
+    if (q.dtype == CYC_F32) {
+        // strict per-element k order, small or unaligned problems: the general kernel
+        if ((q.flags & CYC_FLAG_FIXED_K_ORDER) || !tma_ok(q) || q.M <= 128 || q.N <= 128) return FAM_SIMT;
+        return FAM_UMMA_3XTF32;
+    }
     return tma_ok(q) ? FAM_UMMA : FAM_SIMT;
 }
 
@@ -138,7 +143,8 @@ static int get_encoder(EncodeTiledFn* out) {
 
 // rank-3 map over a [d2][d1][d0] array (d0 contiguous), box [1][box1][box0], 128-byte swizzle
 static int make_map_raw(CUtensorMap* m, CUtensorMapDataType dt, int eb, const void* base, long long d0, long long d1, long long d2,
-                        long long pitch1_elems, long long pitch2_elems, int box0, int box1) {
+                        long long pitch1_elems, long long pitch2_elems, int box0, int box1,
+                        CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     EncodeTiledFn enc;
     int rc = get_encoder(&enc);
     if (rc) return rc;
@@ -147,7 +153,7 @@ static int make_map_raw(CUtensorMap* m, CUtensorMapDataType dt, int eb, const vo
     cuuint32_t box[3] = {static_cast<cuuint32_t>(box0), static_cast<cuuint32_t>(box1), 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = enc(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                     swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
         return CYC_ERR_CUDA;
@@ -157,10 +163,10 @@ static int make_map_raw(CUtensorMap* m, CUtensorMapDataType dt, int eb, const vo
 
 // operand map (A or B) in the problem's input type
 static int make_map(CUtensorMap* m, int dtype, const void* base, long long d0, long long d1, long long d2, long long pitch1_elems,
-                    long long pitch2_elems, int box0, int box1) {
+                    long long pitch2_elems, int box0, int box1, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     const CUtensorMapDataType dt = dtype == CYC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                                     : (dtype == CYC_BF16_F32 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
-    return make_map_raw(m, dt, elem_bytes(dtype), base, d0, d1, d2, pitch1_elems, pitch2_elems, box0, box1);
+    return make_map_raw(m, dt, elem_bytes(dtype), base, d0, d1, d2, pitch1_elems, pitch2_elems, box0, box1, swizzle);
 }
 
 // result map: C[batch][M][N] of 32-bit words, boxes of 32 rows x 32 columns (128 bytes)
@@ -258,6 +264,51 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms) {
     return CYC_OK;
 }
 
+template <bool B_MN>
+static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
+    CUtensorMap tmA, tmB, tmC;
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, q.K, q.sA, 32, PAIR_HALF);
+    if (rc) return rc;
+    // fp32 B stored [K][N] feeds the MMA column-contiguous: 32-byte-chunk swizzle (see umma_smem_desc)
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, 32, PAIR_HALF);
+    if (rc) return rc;
+    PairParams p;
+    p.tma_store = (reinterpret_cast<uintptr_t>(q.C) % 16 == 0 && q.N % 4 == 0 && (q.batch == 1 || q.sC % 4 == 0)) ? 1 : 0;
+    if (p.tma_store) {
+        rc = make_c_map(&tmC, q.dtype, q.C, q.M, q.N, q.batch, q.sC);
+        if (rc) return rc;
+    } else {
+        tmC = tmA;  // never used
+    }
+    p.C = q.C;
+    p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
+    p.sC = q.sC;
+    p.tiles_m = static_cast<int>((q.M + 255) / 256);
+    p.tiles_n = static_cast<int>((q.N + PAIR_BN - 1) / PAIR_BN);
+    p.num_tiles = q.batch * p.tiles_m * p.tiles_n;
+    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    auto kern = umma_pair_tf32x3_kernel<B_MN>;
+    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, X3_SMEM_BYTES));
+    const long long max_pairs = sms / 2;
+    const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
+    kern<<<static_cast<unsigned>(2 * pairs), X3_THREADS, X3_SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
+    CYC_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
+static int launch_tf32x3(const Problem& q, cudaStream_t st) {
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    if (di.cc_major != 10) {
+        snprintf(g_err, sizeof g_err, "tensor-core kernels need an sm_100 device");
+        return CYC_ERR_UNSUPPORTED;
+    }
+    return (q.flags & CYC_FLAG_B_COL_MAJOR) ? launch_tf32x3_cfg<false>(q, st, di.sms) : launch_tf32x3_cfg<true>(q, st, di.sms);
+}
+
 template <int KIND>
 static int launch_umma(const Problem& q, cudaStream_t st) {
     DeviceInfo di;
@@ -281,6 +332,8 @@ static int dispatch(const Problem& q, cudaStream_t st) {
     switch (choose(q)) {
         case FAM_UMMA:
             return q.dtype == CYC_BF16_F32 ? launch_umma<KIND_BF16>(q, st) : launch_umma<KIND_I8>(q, st);
+        case FAM_UMMA_3XTF32:
+            return launch_tf32x3(q, st);
         default:
             if (q.dtype == CYC_F32) return launch_simt<float, float>(q, st);
             if (q.dtype == CYC_BF16_F32) return launch_simt<__nv_bfloat16, float>(q, st);

@@ -61,14 +61,16 @@ struct UmmaTraits<KIND_TF32> {
 
 // 64-bit shared-memory matrix descriptor, 128-byte swizzle.
 //   bits [0,14) start address >> 4 ; [16,30) leading-dimension byte offset >> 4 ;
-//   [32,46) stride-dimension byte offset >> 4 ; [46,48) = 1 ; [61,64) = 2 (128B swizzle)
-__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+//   [32,46) stride-dimension byte offset >> 4 ; [46,48) = 1 ; [61,64) swizzle: 2 = 128 B rows
+//   with 16-byte chunks permuted over 8 rows, 1 = 128 B rows with 32-byte chunks permuted over 4
+//   rows (the only MN-major layout for 32-bit operands)
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle = 2) {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
     d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
     d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
     d |= 1ull << 46;
-    d |= 2ull << 61;
+    d |= static_cast<uint64_t>(swizzle) << 61;
     return d;
 }
 

@@ -1,0 +1,289 @@
+// fp32 recurrence on tensor cores (used when the caller does not ask for the strict
+// per-element k order): every operand x is split into two TF32 parts,
+//     hi = tf32(x)  (round to nearest),   lo = tf32(x - hi),
+// and each k-step accumulates  A_lo*B_hi + A_hi*B_lo + A_hi*B_hi  into the same fp32
+// TMEM accumulator (three tcgen05.mma kind::tf32 per k-step).  The dropped terms
+// (A_lo*B_lo and the rounding of lo) are below 2^-21 |A_ik||B_kj| per product, far
+// inside the 1e-5 * sum_k |A_ik||B_kj| acceptance bound.
+//
+// Same two-SM organisation as umma_pair_kernel.cuh (256 x 256 tile of C per CTA pair,
+// B half per CTA, double-buffered TMEM, TMA-store export) with one more role: four
+// "split" warps per CTA turn each landed fp32 stage into its hi part (in place) and
+// its lo part (second buffer) before the MMA thread may read it.  The split is
+// element-wise, so it is indifferent to the swizzled tile layout.
+//
+// Barriers: full[s] (per CTA: its own 32 KB of copies), ready[s] (leader: 8 arrivals =
+// 4 split warps of each CTA), empty[s] (both, by the leader's multicast commit),
+// acc_full[a] (both), acc_empty[a] (leader, 8 arrivals).
+#pragma once
+#include "umma_pair_kernel.cuh"
+
+namespace cyc {
+
+constexpr int X3_THREADS = 320;                // TMA, MMA, 4 epilogue, 4 split warps
+constexpr int X3_STAGE_HI = 2 * 128 * 128;     // A (128 rows) + B half (128 columns), 128 bytes of k each
+constexpr int X3_STAGE_BYTES = 2 * X3_STAGE_HI;  // hi parts followed by lo parts
+constexpr int X3_STAGES = 3;
+constexpr int X3_SMEM_BYTES = X3_STAGES * X3_STAGE_BYTES + PAIR_STAGING_BYTES + 1024 + 1024;
+
+struct X3Ctl {
+    uint64_t full[4];
+    uint64_t ready[4];
+    uint64_t empty[4];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    volatile int abort;
+};
+
+__device__ __forceinline__ bool x3_wait(uint64_t* bar, uint32_t parity, X3Ctl* ctl, int* status, int where) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if (ctl->abort) return false;
+        if (clock64() - t0 > UMMA_WAIT_CYCLES) {
+            ctl->abort = 1;
+            atomicExch(status, 0x200 | where);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ uint32_t tf32_rna(float x) {
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+    return u;
+}
+
+template <bool B_MN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(X3_THREADS, 1)
+umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                        const __grid_constant__ CUtensorMap tmC, const PairParams p) {
+    constexpr int BK = 32;   // fp32 elements per 128-byte swizzle row
+    constexpr int UK = 8;    // k extent of one kind::tf32 MMA
+    constexpr int CH = 32;   // B stored [K][N]: columns per 128-byte row
+    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t IDESC = umma_instr_desc(1, 2, B_MN, 256, PAIR_BN);
+    constexpr int STAGES = X3_STAGES;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* staging = smem + STAGES * X3_STAGE_BYTES;
+    X3Ctl* ctl = reinterpret_cast<X3Ctl*>(staging + PAIR_STAGING_BYTES);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();
+    const long long pair = blockIdx.x >> 1;
+    const long long num_pairs = gridDim.x >> 1;
+    const int num_kb = (p.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(&ctl->full[s], 1);
+            ptx::mbar_init(&ctl->ready[s], 8);
+            ptx::mbar_init(&ctl->empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(&ctl->acc_full[a], 1);
+            ptx::mbar_init(&ctl->acc_empty[a], 8);
+        }
+        ctl->abort = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmA);
+        ptx::prefetch_tensormap(&tmB);
+        ptx::prefetch_tensormap(&tmC);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc<2>(&ctl->tmem_base, TMEM_COLS);
+        ptx::tmem_relinquish<2>();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (both CTAs, own barrier)
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
+                int b, tm, tn;
+                umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);
+                const int m0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF;
+                const int n0 = tn * PAIR_BN + static_cast<int>(rank) * PAIR_HALF;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!x3_wait(&ctl->empty[stage], phase ^ 1, ctl, p.status, 1)) { ok = false; break; }
+                    uint8_t* sa = smem + stage * X3_STAGE_BYTES;
+                    uint8_t* sb = sa + 128 * 128;
+                    ptx::mbar_arrive_expect_tx(&ctl->full[stage], X3_STAGE_HI);
+                    ptx::tma_load_3d(sa, &tmA, &ctl->full[stage], kb * BK, m0, b);
+                    if constexpr (!B_MN) {
+                        ptx::tma_load_3d(sb, &tmB, &ctl->full[stage], kb * BK, n0, b);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < PAIR_HALF / CH; ++c)
+                            ptx::tma_load_3d(sb + c * (BK * 128), &tmB, &ctl->full[stage], n0 + c * CH, kb * BK, b);
+                    }
+                    ++issued;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (!ok) {
+                const int back = issued < STAGES ? static_cast<int>(issued) : STAGES;
+                int s = stage;
+                uint32_t ph = phase;
+                for (int n = 0; n < back; ++n) {
+                    if (--s < 0) { s = STAGES - 1; ph ^= 1; }
+                    const long long t0 = clock64();
+                    while (!ptx::mbar_try_wait(&ctl->full[s], ph) && clock64() - t0 < UMMA_WAIT_CYCLES) {}
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int local = 0;
+            bool ok = true;
+            for (long long t = pair; t < p.num_tiles && ok; t += num_pairs, ++local) {
+                const int ab = local & 1;
+                const uint32_t acc_phase = (local >> 1) & 1;
+                if (!x3_wait(&ctl->acc_empty[ab], acc_phase ^ 1, ctl, p.status, 2)) { ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * PAIR_BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!x3_wait(&ctl->ready[stage], phase, ctl, p.status, 3)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t sa = ptx::smem_u32(smem + stage * X3_STAGE_BYTES);
+                    const uint32_t sb = sa + 128 * 128;
+#pragma unroll
+                    for (int k = 0; k < BK / UK; ++k) {
+                        const uint64_t a_hi = umma_smem_desc(sa + k * 32, 16, 1024);
+                        const uint64_t a_lo = umma_smem_desc(sa + X3_STAGE_HI + k * 32, 16, 1024);
+                        uint64_t b_hi, b_lo;
+                        if constexpr (!B_MN) {
+                            b_hi = umma_smem_desc(sb + k * 32, 16, 1024);
+                            b_lo = umma_smem_desc(sb + X3_STAGE_HI + k * 32, 16, 1024);
+                        } else {
+                            // B stored [K][N]: 128-byte rows of 32 columns, 32-byte chunks permuted over groups of
+                            // 4 k-rows (512 B apart); the next 32 columns are BK*128 B further on
+                            b_hi = umma_smem_desc(sb + k * (UK * 128), BK * 128, 512, 1);
+                            b_lo = umma_smem_desc(sb + X3_STAGE_HI + k * (UK * 128), BK * 128, 512, 1);
+                        }
+                        ptx::umma<KIND_TF32, 2>(d_tmem, a_lo, b_hi, IDESC, (kb | k) != 0 ? 1u : 0u);
+                        ptx::umma<KIND_TF32, 2>(d_tmem, a_hi, b_lo, IDESC, 1u);
+                        ptx::umma<KIND_TF32, 2>(d_tmem, a_hi, b_hi, IDESC, 1u);
+                    }
+                    ptx::umma_commit_pair(&ctl->empty[stage], 3);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok) ptx::umma_commit_pair(&ctl->acc_full[ab], 3);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ split warps: x -> (hi, lo)
+        const int tid = threadIdx.x - 6 * 32;  // 0..127
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
+            for (int kb = 0; kb < num_kb; ++kb) {
+                if (!x3_wait(&ctl->full[stage], phase, ctl, p.status, 5)) { ok = false; break; }
+                uint8_t* base = smem + stage * X3_STAGE_BYTES;
+#pragma unroll 4
+                for (int it = 0; it < X3_STAGE_HI / (128 * 16); ++it) {
+                    const int off = (tid + 128 * it) * 16;
+                    const float4 v = *reinterpret_cast<const float4*>(base + off);
+                    const float x[4] = {v.x, v.y, v.z, v.w};
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        hi[e] = tf32_rna(x[e]);
+                        const float h = __uint_as_float(hi[e]);
+                        const float r = x[e] - h;                       // exact
+                        lo[e] = (fabsf(h) <= 3.0e38f) ? tf32_rna(r) : 0u;  // inf/NaN stay in the hi part only
+                    }
+                    *reinterpret_cast<uint4*>(base + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4*>(base + X3_STAGE_HI + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                }
+                ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(&ctl->ready[stage], 0);
+                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: C_ij <- [i,k_end]_C (both CTAs)
+        const int q = warp & 3;
+        uint8_t* my_stage = staging + q * 8192;
+        int local = 0, sbuf = 0;
+        bool ok = true;
+        for (long long t = pair; t < p.num_tiles && ok; t += num_pairs, ++local) {
+            const int ab = local & 1;
+            const uint32_t acc_phase = (local >> 1) & 1;
+            int b, tm, tn;
+            umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);
+            if (!x3_wait(&ctl->acc_full[ab], acc_phase, ctl, p.status, 4)) { ok = false; break; }
+            ptx::tc_fence_after();
+            const int row0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF + q * 32;
+            const int row = row0 + lane;
+            float* crow = static_cast<float*>(p.C) + static_cast<long long>(b) * p.sC + static_cast<long long>(row) * p.N;
+#pragma unroll 1
+            for (int c0 = 0; c0 < PAIR_BN; c0 += 32) {
+                const int col = tn * PAIR_BN + c0;
+                if (col >= p.N) break;
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(ab * PAIR_BN + c0), v);
+                if (p.tma_store) {
+                    uint8_t* buf = my_stage + sbuf * 4096;
+                    if (lane == 0) ptx::tma_store_wait_read<1>();
+                    __syncwarp();
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        *reinterpret_cast<uint4*>(buf + lane * 128 + ((g ^ (lane & 7)) << 4)) = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_3d(&tmC, buf, col, row0, b);
+                        ptx::tma_store_commit();
+                    }
+                    sbuf ^= 1;
+                } else {
+                    ptx::tmem_ld_wait();
+                    if (row < p.M) {
+#pragma unroll
+                        for (int g = 0; g < 32; ++g)
+                            if (col + g < p.N) reinterpret_cast<uint32_t*>(crow)[col + g] = v[g];
+                    }
+                }
+            }
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(&ctl->acc_empty[ab], 0);
+        }
+        if (lane == 0) ptx::tma_store_wait_all<0>();
+        __syncwarp();
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc<2>(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace cyc

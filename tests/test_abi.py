@@ -69,6 +69,9 @@ def test_kernel_selection(binding):
     assert k(1, 8192, 8192, 8192, "bf16") == "tcgen05"
     assert k(1, 4096, 4096, 4096, "i8", b_col_major=True) == "tcgen05"
     assert k(1024, 256, 256, 256, "bf16") == "tcgen05"
+    assert k(1, 65536, 256, 256, "f32") == "tcgen05_3xtf32"
+    assert k(1, 65536, 256, 256, "f32", fixed_k_order=True) == "simt"
+    assert k(1, 128, 256, 256, "f32") == "simt"
     assert k(1, 65, 127, 33, "bf16") == "simt"               # pitches not multiples of 16 bytes
     assert k(1, 64, 64, 64, "bf16", a_ptr=258) == "simt"     # base not 16-byte aligned
     assert k(1, 64, 64, 64, "bf16", a_ptr=257) is None       # not even element aligned

@@ -80,6 +80,31 @@ def test_umma_int8_bit_exact(shape, col):
     check_workload(w)
 
 
+@pytest.mark.parametrize("shape", [(256, 256, 256), (300, 520, 200), (129, 264, 72), (512, 384, 36), (1000, 260, 1028)])
+@pytest.mark.parametrize("col", [False, True])
+def test_fp32_split_tf32_on_tensor_cores(shape, col):
+    w = wl("f32", *shape, seed=41, col=col, fixed=False)
+    assert family(w) == "tcgen05_3xtf32"
+    worst = check_workload(w)          # 1e-5 * S
+    assert worst < 2e-6                # the split leaves about 2^-21 per product
+
+
+def test_fp32_split_closed_forms():
+    import torch
+    from paper_2511_09987_b200 import binding
+    n = 384
+    X = (torch.randn(n, n, device="cuda") * 3).float()
+    I = torch.eye(n, device="cuda")
+    assert binding.kernel_for(1, n, n, n, "f32") == "tcgen05_3xtf32"
+    # hi + lo carries 22 of the 24 significand bits, so A = I returns B to within 2^-21 relative
+    out = binding.recurrence_matmul(I, X)
+    assert (out - X).abs().max().item() <= 2.0 ** -21 * X.abs().max().item()
+    ones = torch.ones((n, n), device="cuda")
+    assert (binding.recurrence_matmul(ones, ones) == n).all().item()
+    Xi = torch.randint(-1000, 1000, (n, n), device="cuda").float()      # 11-bit integers: hi part exact, lo zero
+    assert torch.equal(binding.recurrence_matmul(I, Xi), Xi)
+
+
 def test_umma_int8_extreme_values():
     import torch
     from paper_2511_09987_b200 import binding
