@@ -1,16 +1,17 @@
 // fp32 recurrence on tensor cores (used when the caller does not ask for the strict
 // per-element k order): every operand x is split into two TF32 parts,
-//     hi = tf32(x)  (round to nearest),   lo = tf32(x - hi),
+//     hi = x with its 13 low significand bits dropped  (what a kind::tf32 MMA reads from an fp32 word),
+//     lo = tf32(x - hi)                                  (round to nearest),
 // and each k-step accumulates  A_lo*B_hi + A_hi*B_lo + A_hi*B_hi  into the same fp32
 // TMEM accumulator (three tcgen05.mma kind::tf32 per k-step).  The dropped terms
-// (A_lo*B_lo and the rounding of lo) are below 2^-21 |A_ik||B_kj| per product, far
+// (A_lo*B_lo < 2^-20 and the rounding of lo < 2^-22, relative to |A_ik||B_kj|) stay far
 // inside the 1e-5 * sum_k |A_ik||B_kj| acceptance bound.
 //
 // Same two-SM organisation as umma_pair_kernel.cuh (256 x 256 tile of C per CTA pair,
-// B half per CTA, double-buffered TMEM, TMA-store export) with one more role: four
-// "split" warps per CTA turn each landed fp32 stage into its hi part (in place) and
-// its lo part (second buffer) before the MMA thread may read it.  The split is
-// element-wise, so it is indifferent to the swizzled tile layout.
+// B half per CTA, double-buffered TMEM, TMA-store export) with one more role: two sets of four
+// "split" warps per CTA compute the lo part of each landed fp32 stage into a second
+// buffer before the MMA thread may read it (the landed tile itself serves as the hi
+// part).  The split is element-wise, so it is indifferent to the swizzled tile layout.
 //
 // Barriers: full[s] (per CTA: its own 32 KB of copies), ready[s] (leader: 8 arrivals =
 // 4 split warps of each CTA), empty[s] (both, by the leader's multicast commit),
@@ -20,10 +21,12 @@
 
 namespace cyc {
 
-constexpr int X3_THREADS = 320;                // TMA, MMA, 4 epilogue, 4 split warps
+constexpr int X3_SPLIT_SETS = 2;               // sets of four split warps, taking stages in turn
+constexpr int X3_THREADS = 192 + X3_SPLIT_SETS * 128;  // TMA, MMA, 4 epilogue warps, then the split warps
 constexpr int X3_STAGE_HI = 2 * 128 * 128;     // A (128 rows) + B half (128 columns), 128 bytes of k each
 constexpr int X3_STAGE_BYTES = 2 * X3_STAGE_HI;  // hi parts followed by lo parts
 constexpr int X3_STAGES = 3;
+constexpr int X3_PREFETCH = 8;  // k-blocks of A requested from L2 ahead of the ring
 constexpr int X3_SMEM_BYTES = X3_STAGES * X3_STAGE_BYTES + PAIR_STAGING_BYTES + 1024 + 1024;
 
 struct X3Ctl {
@@ -50,11 +53,9 @@ __device__ __forceinline__ bool x3_wait(uint64_t* bar, uint32_t parity, X3Ctl* c
     return true;
 }
 
-__device__ __forceinline__ uint32_t tf32_rna(float x) {
-    uint32_t u;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
-    return u;
-}
+// fp32 bit pattern -> nearest TF32 (10 explicit significand bits; ties away from zero), low 13 bits cleared.
+// Integer arithmetic on the encoding: adding half a TF32 ulp carries into the exponent exactly as rounding does.
+__device__ __forceinline__ uint32_t tf32_round(uint32_t bits) { return (bits + 0x1000u) & 0xFFFFE000u; }
 
 template <bool B_MN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(X3_THREADS, 1)
@@ -82,7 +83,7 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&ctl->full[s], 1);
-            ptx::mbar_init(&ctl->ready[s], 8);
+            ptx::mbar_init(&ctl->ready[s], 8);  // four split warps of each CTA
             ptx::mbar_init(&ctl->empty[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -113,12 +114,25 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
+            // A is streamed from HBM exactly once, and the ring is only three stages deep: a second cursor runs
+            // X3_PREFETCH k-blocks ahead and asks L2 for the A tiles, so the copies into the ring hit L2
+            long long pf_t = pair;
+            int pf_kb = 0;
+            auto prefetch_next = [&]() {
+                if (pf_t >= p.num_tiles) return;
+                int b, tm, tn;
+                umma_tile_coord(pf_t, p.tiles_m, p.tiles_n, b, tm, tn);
+                ptx::tma_prefetch_l2_3d(&tmA, pf_kb * BK, tm * 256 + static_cast<int>(rank) * PAIR_HALF, b);
+                if (++pf_kb == num_kb) { pf_kb = 0; pf_t += num_pairs; }
+            };
+            for (int i = 0; i < X3_PREFETCH; ++i) prefetch_next();
             for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
                 int b, tm, tn;
                 umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);
                 const int m0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF;
                 const int n0 = tn * PAIR_BN + static_cast<int>(rank) * PAIR_HALF;
                 for (int kb = 0; kb < num_kb; ++kb) {
+                    prefetch_next();
                     if (!x3_wait(&ctl->empty[stage], phase ^ 1, ctl, p.status, 1)) { ok = false; break; }
                     uint8_t* sa = smem + stage * X3_STAGE_BYTES;
                     uint8_t* sb = sa + 128 * 128;
@@ -192,29 +206,43 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         __syncwarp();
     } else if (warp >= 6) {
         // ------------------------------------------------------------ split warps: x -> (hi, lo)
-        const int tid = threadIdx.x - 6 * 32;  // 0..127
+        // the sets of four warps take stages in turn, so the fixed latencies of one stage's split
+        // (wait, store drain, proxy fence) overlap with the other set's work
+        const int set = (warp - 6) >> 2;
+        const int tid = (threadIdx.x - 6 * 32) & 127;  // 0..127 within the set
+        constexpr int NT = 128;
         int stage = 0;
         uint32_t phase = 0;
+        uint32_t turn = 0;
         bool ok = true;
         for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
-            for (int kb = 0; kb < num_kb; ++kb) {
+            for (int kb = 0; kb < num_kb; ++kb, ++turn) {
+                if (turn % X3_SPLIT_SETS != static_cast<uint32_t>(set)) {
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    continue;
+                }
                 if (!x3_wait(&ctl->full[stage], phase, ctl, p.status, 5)) { ok = false; break; }
                 uint8_t* base = smem + stage * X3_STAGE_BYTES;
-#pragma unroll 4
-                for (int it = 0; it < X3_STAGE_HI / (128 * 16); ++it) {
-                    const int off = (tid + 128 * it) * 16;
-                    const float4 v = *reinterpret_cast<const float4*>(base + off);
-                    const float x[4] = {v.x, v.y, v.z, v.w};
-                    uint32_t hi[4], lo[4];
+#pragma unroll 1
+                for (int it0 = 0; it0 < X3_STAGE_HI / (NT * 16); it0 += 4) {
+                    uint4 v[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        hi[e] = tf32_rna(x[e]);
-                        const float h = __uint_as_float(hi[e]);
-                        const float r = x[e] - h;                       // exact
-                        lo[e] = (fabsf(h) <= 3.0e38f) ? tf32_rna(r) : 0u;  // inf/NaN stay in the hi part only
+                    for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const uint4*>(base + (tid + NT * (it0 + u)) * 16);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                        uint32_t lo[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            // hi = x with the 13 low significand bits dropped: exactly what the tensor core reads
+                            // from the untouched fp32 tile.  inf/NaN stay in the hi part only.
+                            const uint32_t hi = x[e] & 0xFFFFE000u;
+                            const float r = __uint_as_float(x[e]) - __uint_as_float(hi);  // exact, below 2^-10 |x|
+                            lo[e] = ((x[e] & 0x7F800000u) == 0x7F800000u) ? 0u : tf32_round(__float_as_uint(r));
+                        }
+                        const int off = (tid + NT * (it0 + u)) * 16;
+                        *reinterpret_cast<uint4*>(base + X3_STAGE_HI + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                     }
-                    *reinterpret_cast<uint4*>(base + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<uint4*>(base + X3_STAGE_HI + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
                 ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
                 __syncwarp();
