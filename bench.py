@@ -383,19 +383,22 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--shape", default=None, help="M,N,K[,batch]: a smaller case of the workload's recipe (for profiling)")
+    ap.add_argument("--strict", action="store_true", help="set the fixed-k-order flag (fp32: the per-element FMA chain kernel)")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs (for profiling)")
     args = ap.parse_args()
     w = inputs.WORKLOADS[args.workload]
     if args.shape:
         dims = [int(x) for x in args.shape.split(",")]
         w = inputs.scaled(w, name=w.name + "@" + args.shape, M=dims[0], N=dims[1], K=dims[2], batch=dims[3] if len(dims) > 3 else w.batch)
+    if args.strict:
+        w = inputs.scaled(w, name=w.name + "+strict", fixed_k_order=True)
     if args.impl == "reference":
         if args.steps is None:
             args.steps = 3
         run_reference(args, w)
         return
     if args.steps is None:
-        args.steps = {"c1": 2000, "c2": 2000, "c3": 200, "c4": 1000, "c5": 1000}[w.name.split("@")[0]]
+        args.steps = {"c1": 2000, "c2": 2000, "c3": 200, "c4": 1000, "c5": 1000}[w.name.split("@")[0].split("+")[0]]
     run_ours(args, w)
 
 
