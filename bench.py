@@ -191,17 +191,15 @@ def describe(w):
 
 def run_ours(args, w):
     import torch
-    import torch.distributed as dist
     from paper_2511_09987_b200 import binding
+    from paper_2511_09987_b200.replicas import Replicas
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    reps = Replicas("nccl", torch.device("cuda", local))
+    world, rank = reps.world, reps.rank
     peaks, peak_kind = load_peaks()
 
     # ---- operands: generated once on the host, uploaded; several device copies rotate so that
@@ -231,8 +229,7 @@ def run_ours(args, w):
                                 sets[0][2].data_ptr(), b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        reps.barrier()
         torch.cuda.synchronize()
 
     for i in range(max(3, args.warmup)):
@@ -268,10 +265,7 @@ def run_ours(args, w):
     if extra_note:
         clocks["note"] = extra_note
 
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
+    ms = reps.max_over_ranks(ms)
     ms_per_step = ms / args.steps
     ops_step = 2.0 * w.macs
     value = world * ops_step / (ms_per_step * 1e-3) / 1e12
@@ -289,14 +283,10 @@ def run_ours(args, w):
     e1.record(stream)
     barrier()
     e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(1, e2e_steps)
-    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = world * ops_step / (float(t.item()) * 1e-3) / 1e12
+    e2e_value = world * ops_step / (reps.max_over_ranks(e2e_ms) * 1e-3) / 1e12
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        reps.close()
         return
 
     # ---- roofline of the dominant (only) kernel: one launch per step
@@ -342,8 +332,7 @@ def run_ours(args, w):
         "cpu_baseline": {"value": cpu_v, "unit": unit_of(w), "cores": cores, "kind": "oracle", "sample": sample},
     }
     print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    reps.close()
 
 
 def kernel_source_digest():

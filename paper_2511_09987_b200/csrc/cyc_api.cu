@@ -101,6 +101,15 @@ static int launch_simt(const Problem& q, cudaStream_t st) {
     p.tiles_n = static_cast<int>((q.N + SIMT_BN - 1) / SIMT_BN);
     const long long blocks = q.batch * p.tiles_m * p.tiles_n;
     if (blocks > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
+    if (blocks < 74) {  // too few large tiles to occupy even half the SMs: smaller tiles, shorter per-thread chains
+        p.tiles_m = static_cast<int>((q.M + SIMT_S_BM - 1) / SIMT_S_BM);
+        p.tiles_n = static_cast<int>((q.N + SIMT_S_BN - 1) / SIMT_S_BN);
+        const long long small_blocks = q.batch * p.tiles_m * p.tiles_n;
+        simt_recurrence_small_kernel<TIn, TAcc><<<static_cast<unsigned>(small_blocks), SIMT_THREADS, 0, st>>>(p);
+        CYC_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+        return CYC_OK;
+    }
     bool vec = false;
     if constexpr (sizeof(TIn) == 4) {
         vec = !colmajor && q.K % 4 == 0 && q.N % 4 == 0 && q.sA % 4 == 0 && q.sB % 4 == 0 && q.sC % 4 == 0 &&

@@ -205,4 +205,81 @@ __global__ void __launch_bounds__(SIMT_THREADS, 2) simt_recurrence_kernel(const 
     }
 }
 
+// Small problems (fewer 128 x 128 tiles than half the SMs): 64 x 64 tiles, 4 x 4 outputs per
+// thread, so that more SMs take part and the per-thread chain work shrinks.  Same chains, same
+// order, same bits; element-wise guarded loads (any shape, any alignment).
+constexpr int SIMT_S_BM = 64, SIMT_S_BN = 64, SIMT_S_BK = 16;
+
+template <typename TIn, typename TAcc>
+__global__ void __launch_bounds__(SIMT_THREADS) simt_recurrence_small_kernel(const SimtParams p) {
+    __shared__ __align__(16) TAcc As[SIMT_S_BK][SIMT_S_BM + 4];
+    __shared__ __align__(16) TAcc Bs[SIMT_S_BK][SIMT_S_BN + 4];
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    long long t = blockIdx.x;
+    const int tn = static_cast<int>(t % p.tiles_n);
+    t /= p.tiles_n;
+    const int tm = static_cast<int>(t % p.tiles_m);
+    const long long batch = t / p.tiles_m;
+    const int m0 = tm * SIMT_S_BM, n0 = tn * SIMT_S_BN;
+    const TIn* __restrict__ A = static_cast<const TIn*>(p.A) + batch * p.sA;
+    const TIn* __restrict__ B = static_cast<const TIn*>(p.B) + batch * p.sB;
+    TAcc* __restrict__ C = static_cast<TAcc*>(p.C) + batch * p.sC;
+    const int M = p.M, N = p.N, K = p.K;
+
+    TAcc acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = TAcc(0);  // [i,0-1]_C = 0
+
+    for (int k0 = 0; k0 < K; k0 += SIMT_S_BK) {
+        // 64 x 16 elements of A and 16 x 64 of B: four of each per thread
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = tid + e * SIMT_THREADS;
+            const int r = idx >> 4, kk = idx & 15;
+            TAcc v = TAcc(0);
+            if (m0 + r < M && k0 + kk < K) v = simt_widen<TIn, TAcc>(A[static_cast<long long>(m0 + r) * K + k0 + kk]);
+            As[kk][r] = v;
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = tid + e * SIMT_THREADS;
+            int kk, j;
+            if (p.b_sj == 1) { kk = idx >> 6; j = idx & 63; }
+            else { kk = idx & 15; j = idx >> 4; }
+            TAcc v = TAcc(0);
+            if (k0 + kk < K && n0 + j < N) v = simt_widen<TIn, TAcc>(B[static_cast<long long>(k0 + kk) * p.b_sk + static_cast<long long>(n0 + j) * p.b_sj]);
+            Bs[kk][j] = v;
+        }
+        __syncthreads();
+        const int kmax = min(SIMT_S_BK, K - k0);  // never run a chain past k_end
+        for (int kk = 0; kk < kmax; ++kk) {
+            TAcc a[4], b[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                a[q] = As[kk][ty * 4 + q];
+                b[q] = Bs[kk][tx * 4 + q];
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = simt_mac(acc[i][j], a[i], b[j]);
+        }
+        __syncthreads();
+    }
+    // C_ij <- [i,k_end]_C
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = m0 + ty * 4 + i;
+        if (r >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = n0 + tx * 4 + j;
+            if (c < N) C[static_cast<long long>(r) * N + c] = acc[i][j];
+        }
+    }
+}
+
 }  // namespace cyc
