@@ -112,8 +112,10 @@ int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, int64_t K, i
  */
 int cyc_last_device_status(void* stream, int* out);
 
-/* Name of the kernel family the dispatcher would pick ("simt", "tcgen05",
- * "tcgen05_3xtf32") for these arguments, or NULL if they are invalid.  Host only. */
+/* Name of the kernel the dispatcher would pick for these arguments -- "simt" (general
+ * kernel), "tcgen05" (one CTA per tile), "tcgen05_pair" (CTA pair, 256x256 tiles),
+ * "tcgen05_pair_tall" (CTA pair, 512x256 tiles), "tcgen05_3xtf32" (fp32 split into TF32
+ * parts) -- or NULL if the arguments are invalid.  Host only, makes no CUDA call. */
 const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
                            const void* C, unsigned flags);
 

@@ -14,6 +14,7 @@
 #include "simt_kernel.cuh"
 #include "umma_kernel.cuh"
 #include "umma_pair_kernel.cuh"
+#include "umma_pair_tall_kernel.cuh"
 #include "umma_pair_tf32x3_kernel.cuh"
 
 namespace cyc {
@@ -65,7 +66,8 @@ static int validate(const Problem& q) {
     return CYC_OK;
 }
 
-enum Family { FAM_SIMT = 0, FAM_UMMA = 1, FAM_UMMA_3XTF32 = 2 };
+enum Family { FAM_SIMT = 0, FAM_UMMA = 1, FAM_UMMA_3XTF32 = 2, FAM_UMMA_PAIR = 3, FAM_UMMA_TALL = 4 };
+constexpr long long kCtaPairs = 74;  // CTA pairs resident on a B200 (148 SMs); used by the tile-shape rule
 
 // the tensor-core kernels move tiles with TMA: 16-byte aligned bases and pitches
 static bool tma_ok(const Problem& q) {
@@ -84,7 +86,14 @@ static Family choose(const Problem& q) {
         if ((q.flags & CYC_FLAG_FIXED_K_ORDER) || !tma_ok(q) || q.M <= 128 || q.N <= 128) return FAM_SIMT;
         return FAM_UMMA_3XTF32;
     }
-    return tma_ok(q) ? FAM_UMMA : FAM_SIMT;
+    if (!tma_ok(q)) return FAM_SIMT;
+    const int bk = 128 / elem_bytes(q.dtype);
+    const long long nkb = (q.K + bk - 1) / bk;
+    const long long tall_tiles = q.batch * ((q.M + 511) / 512) * ((q.N + 255) / 256);
+    // 512 x 256 tiles need a long k loop (their export is not overlapped) and enough tiles to occupy every CTA pair
+    if (q.M > 256 && q.N > 128 && nkb >= 16 && tall_tiles >= kCtaPairs) return FAM_UMMA_TALL;
+    if (q.M > 128 && q.N > 128) return FAM_UMMA_PAIR;  // enough rows and columns for a CTA pair
+    return FAM_UMMA;
 }
 
 // ------------------------------------------------------------------ SIMT launch
@@ -273,6 +282,42 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms) {
     return CYC_OK;
 }
 
+// 512 x 256 tiles: selected when the k loop is long enough to amortise the unoverlapped export
+template <int KIND, bool B_MN>
+static int launch_pair_tall_cfg(const Problem& q, cudaStream_t st, int sms) {
+    constexpr int BK = 128 / UmmaTraits<KIND>::ELEM_BYTES;
+    constexpr int CH = 128 / UmmaTraits<KIND>::ELEM_BYTES;
+    CUtensorMap tmA, tmB, tmC;
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, q.K, q.sA, BK, PAIR_HALF);
+    if (rc) return rc;
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, PAIR_HALF);
+    if (rc) return rc;
+    PairParams p;
+    p.tma_store = (reinterpret_cast<uintptr_t>(q.C) % 16 == 0 && q.N % 4 == 0 && (q.batch == 1 || q.sC % 4 == 0)) ? 1 : 0;
+    if (p.tma_store) {
+        rc = make_c_map(&tmC, q.dtype, q.C, q.M, q.N, q.batch, q.sC);
+        if (rc) return rc;
+    } else {
+        tmC = tmA;  // never used
+    }
+    p.C = q.C;
+    p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
+    p.sC = q.sC;
+    p.tiles_m = static_cast<int>((q.M + 511) / 512);
+    p.tiles_n = static_cast<int>((q.N + PAIR_BN - 1) / PAIR_BN);
+    p.num_tiles = q.batch * p.tiles_m * p.tiles_n;
+    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    auto kern = umma_pair_tall_kernel<KIND, B_MN>;
+    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TALL_SMEM_BYTES));
+    const long long max_pairs = sms / 2;
+    const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
+    kern<<<static_cast<unsigned>(2 * pairs), TALL_THREADS, TALL_SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
+    CYC_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
 template <bool B_MN>
 static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
     CUtensorMap tmA, tmB, tmC;
@@ -328,7 +373,10 @@ static int launch_umma(const Problem& q, cudaStream_t st) {
         return CYC_ERR_UNSUPPORTED;
     }
     const bool b_mn = (q.flags & CYC_FLAG_B_COL_MAJOR) == 0;
-    if (q.M > 128 && q.N > 128)  // enough rows and columns for a CTA pair
+    const Family fam = choose(q);
+    if (fam == FAM_UMMA_TALL)
+        return b_mn ? launch_pair_tall_cfg<KIND, true>(q, st, di.sms) : launch_pair_tall_cfg<KIND, false>(q, st, di.sms);
+    if (fam == FAM_UMMA_PAIR)
         return b_mn ? launch_pair_cfg<KIND, true>(q, st, di.sms) : launch_pair_cfg<KIND, false>(q, st, di.sms);
     const bool wide = q.N > 128;
     if (b_mn) return wide ? launch_umma_cfg<KIND, true, 256, 4>(q, st, di.sms) : launch_umma_cfg<KIND, true, 128, 6>(q, st, di.sms);
@@ -340,6 +388,8 @@ static int dispatch(const Problem& q, cudaStream_t st) {
     if (rc) return rc;
     switch (choose(q)) {
         case FAM_UMMA:
+        case FAM_UMMA_PAIR:
+        case FAM_UMMA_TALL:
             return q.dtype == CYC_BF16_F32 ? launch_umma<KIND_BF16>(q, st) : launch_umma<KIND_I8>(q, st);
         case FAM_UMMA_3XTF32:
             return launch_tf32x3(q, st);
@@ -419,6 +469,8 @@ extern "C" const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64
     if (validate(q) != CYC_OK) return nullptr;
     switch (choose(q)) {
         case FAM_UMMA: return "tcgen05";
+        case FAM_UMMA_PAIR: return "tcgen05_pair";
+        case FAM_UMMA_TALL: return "tcgen05_pair_tall";
         case FAM_UMMA_3XTF32: return "tcgen05_3xtf32";
         default: return "simt";
     }

@@ -67,7 +67,7 @@ def check_workload(w, threads=8, rows_per_problem=None, fixed_k_order=None):
         else:
             rng = np.random.default_rng(1234 + (b or 0))
             # sampled rows, always including the first and last row of the problem and of a tile
-            fixed_rows = [r for r in (0, 127, 128, w.M - 129, w.M - 1) if 0 <= r < w.M]
+            fixed_rows = [r for r in (0, 127, 128, 255, 256, 383, 384, 511, 512, w.M - 129, w.M - 1) if 0 <= r < w.M]
             rows = np.unique(np.concatenate([fixed_rows, rng.integers(0, w.M, size=rows_per_problem)]))
         worst = max(worst, compare_rows(w, Ab, Bb, Cb[rows], rows, threads, exact))
     return worst

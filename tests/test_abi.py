@@ -66,9 +66,11 @@ def test_invalid_arguments_rejected_on_host(binding):
 def test_kernel_selection(binding):
     k = binding.kernel_for
     assert k(1, 64, 64, 64, "f32", fixed_k_order=True) == "simt"
-    assert k(1, 8192, 8192, 8192, "bf16") == "tcgen05"
-    assert k(1, 4096, 4096, 4096, "i8", b_col_major=True) == "tcgen05"
-    assert k(1024, 256, 256, 256, "bf16") == "tcgen05"
+    assert k(1, 8192, 8192, 8192, "bf16") == "tcgen05_pair_tall"
+    assert k(1, 4096, 4096, 4096, "i8", b_col_major=True) == "tcgen05_pair_tall"
+    assert k(1024, 256, 256, 256, "bf16") == "tcgen05_pair"
+    assert k(1, 4096, 4096, 64, "bf16") == "tcgen05_pair"        # k loop too short for the tall tiles
+    assert k(1, 128, 4096, 4096, "bf16") == "tcgen05"            # one row block: a single CTA per tile
     assert k(1, 65536, 256, 256, "f32") == "tcgen05_3xtf32"
     assert k(1, 65536, 256, 256, "f32", fixed_k_order=True) == "simt"
     assert k(1, 128, 256, 256, "f32") == "simt"

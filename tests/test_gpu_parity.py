@@ -67,7 +67,7 @@ UMMA_SHAPES = [(128, 128, 64), (128, 256, 64), (128, 256, 128), (256, 512, 256),
 @pytest.mark.parametrize("col", [False, True])
 def test_umma_bf16(shape, col):
     w = wl("bf16", *shape, seed=21, col=col)
-    assert family(w) == "tcgen05"
+    assert family(w).startswith("tcgen05")
     check_workload(w)
 
 
@@ -76,7 +76,7 @@ def test_umma_bf16(shape, col):
 @pytest.mark.parametrize("col", [True, False])
 def test_umma_int8_bit_exact(shape, col):
     w = wl("i8", *shape, seed=22, col=col)
-    assert family(w) == "tcgen05"
+    assert family(w).startswith("tcgen05")
     check_workload(w)
 
 
@@ -131,6 +131,24 @@ def test_umma_closed_forms_bf16():
     assert torch.equal(binding.recurrence_matmul(X, P, b_col_major=True), X.float()[:, perm])   # stored B^T = P
     ones = torch.ones((n, n), device="cuda", dtype=torch.bfloat16)
     assert (binding.recurrence_matmul(ones, ones) == n).all().item()
+
+
+def test_umma_tall_tiles_ragged():
+    # 512 x 256 tiles (long k loop, at least 74 tiles), ragged in every dimension
+    w = wl("bf16", 4100, 2600, 1032, seed=51)
+    assert family(w) == "tcgen05_pair_tall"
+    check_workload(w, rows_per_problem=64)
+    w = wl("bf16", 4100, 2600, 1032, seed=52, col=True)
+    check_workload(w, rows_per_problem=64)
+    w = wl("i8", 4100, 2320, 2064, seed=53, col=True)
+    assert family(w) == "tcgen05_pair_tall"
+    check_workload(w, rows_per_problem=64)
+    w = wl("i8", 4100, 2320, 2064, seed=54, col=False)
+    check_workload(w, rows_per_problem=64)
+    # batched: 40 problems of 600 x 304 x 1032 -> 2 x 2 tall tiles each
+    w = wl("bf16", 600, 304, 1032, seed=55, batch=40)
+    assert family(w) == "tcgen05_pair_tall"
+    check_workload(w, rows_per_problem=24)
 
 
 def test_umma_many_tiles_per_cta():
