@@ -67,7 +67,8 @@ def test_kernel_selection(binding):
     k = binding.kernel_for
     assert k(1, 64, 64, 64, "f32", fixed_k_order=True) == "simt"
     assert k(1, 8192, 8192, 8192, "bf16") == "tcgen05_pair_tall"
-    assert k(1, 4096, 4096, 4096, "i8", b_col_major=True) == "tcgen05_pair_tall"
+    assert k(1, 4096, 4096, 4096, "i8", b_col_major=True) == "tcgen05_pair"    # 32 k-blocks: 256x256 tiles
+    assert k(1, 4096, 4096, 16384, "i8", b_col_major=True) == "tcgen05_pair_tall"
     assert k(1024, 256, 256, 256, "bf16") == "tcgen05_pair"
     assert k(1, 4096, 4096, 64, "bf16") == "tcgen05_pair"        # k loop too short for the tall tiles
     assert k(1, 128, 4096, 4096, "bf16") == "tcgen05"            # one row block: a single CTA per tile

@@ -135,18 +135,18 @@ def test_umma_closed_forms_bf16():
 
 def test_umma_tall_tiles_ragged():
     # 512 x 256 tiles (long k loop, at least 74 tiles), ragged in every dimension
-    w = wl("bf16", 4100, 2600, 1032, seed=51)
+    w = wl("bf16", 4100, 2600, 6152, seed=51)
+    assert family(w) == "tcgen05_pair_tall"
+    check_workload(w, rows_per_problem=24)
+    w = wl("bf16", 4100, 2600, 6152, seed=52, col=True)
+    check_workload(w, rows_per_problem=64)
+    w = wl("i8", 4100, 2320, 12304, seed=53, col=True)
     assert family(w) == "tcgen05_pair_tall"
     check_workload(w, rows_per_problem=64)
-    w = wl("bf16", 4100, 2600, 1032, seed=52, col=True)
+    w = wl("i8", 4100, 2320, 12304, seed=54, col=False)
     check_workload(w, rows_per_problem=64)
-    w = wl("i8", 4100, 2320, 2064, seed=53, col=True)
-    assert family(w) == "tcgen05_pair_tall"
-    check_workload(w, rows_per_problem=64)
-    w = wl("i8", 4100, 2320, 2064, seed=54, col=False)
-    check_workload(w, rows_per_problem=64)
-    # batched: 40 problems of 600 x 304 x 1032 -> 2 x 2 tall tiles each
-    w = wl("bf16", 600, 304, 1032, seed=55, batch=40)
+    # batched: 20 problems of 600 x 304 x 6152 -> 2 x 2 tall tiles each
+    w = wl("bf16", 600, 304, 6152, seed=55, batch=20)
     assert family(w) == "tcgen05_pair_tall"
     check_workload(w, rows_per_problem=24)
 
