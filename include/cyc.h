@@ -33,9 +33,13 @@
  *                 into two TF32 parts and fp32 accumulation (error well inside
  *                 1e-5 * sum_k |A_ik||B_kj|).
  *   CYC_BF16_F32  A, B bfloat16; products exact; fp32 accumulation; C float.
- *                 k-blocks are accumulated in increasing order by one owner
- *                 per C_ij (never split-K, never atomics), so results are
- *                 run-to-run identical with or without the flag.
+ *                 k-blocks are accumulated in increasing order; results are
+ *                 run-to-run identical with or without the flag (no atomics).
+ *                 Without the flag, problems with few output tiles and a long k
+ *                 loop are cut into k-slices whose partial sums are added in
+ *                 slice order (split-K; needs a workspace from a stream-ordered
+ *                 pool the library owns); with the flag one CTA pair owns each
+ *                 C_ij for the whole k loop.
  *   CYC_I8_I32    A, B signed 8-bit; C int32; exact for K <= 131071.
  */
 #ifndef CYC_H_
@@ -114,8 +118,10 @@ int cyc_last_device_status(void* stream, int* out);
 
 /* Name of the kernel the dispatcher would pick for these arguments -- "simt" (general
  * kernel), "tcgen05" (one CTA per tile), "tcgen05_pair" (CTA pair, 256x256 tiles),
- * "tcgen05_pair_tall" (CTA pair, 512x256 tiles), "tcgen05_3xtf32" (fp32 split into TF32
- * parts) -- or NULL if the arguments are invalid.  Host only, makes no CUDA call. */
+ * "tcgen05_pair_tall" (CTA pair, 512x256 tiles), "tcgen05_pair_splitk" (few tiles, long k
+ * loop: k-slices on different CTA pairs, partial sums added in slice order by a second kernel),
+ * "tcgen05_3xtf32" (fp32 split into TF32 parts) -- or NULL if the arguments are invalid.
+ * Host only, makes no CUDA call. */
 const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
                            const void* C, unsigned flags);
 

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -15,6 +16,7 @@
 #include "umma_kernel.cuh"
 #include "umma_pair_kernel.cuh"
 #include "umma_pair_tall_kernel.cuh"
+#include "splitk_reduce_kernel.cuh"
 #include "umma_pair_tf32x3_kernel.cuh"
 
 namespace cyc {
@@ -66,7 +68,7 @@ static int validate(const Problem& q) {
     return CYC_OK;
 }
 
-enum Family { FAM_SIMT = 0, FAM_UMMA = 1, FAM_UMMA_3XTF32 = 2, FAM_UMMA_PAIR = 3, FAM_UMMA_TALL = 4 };
+enum Family { FAM_SIMT = 0, FAM_UMMA = 1, FAM_UMMA_3XTF32 = 2, FAM_UMMA_PAIR = 3, FAM_UMMA_TALL = 4, FAM_UMMA_SPLITK = 5 };
 constexpr long long kCtaPairs = 74;  // CTA pairs resident on a B200 (148 SMs); used by the tile-shape rule
 
 // the tensor-core kernels move tiles with TMA: 16-byte aligned bases and pitches
@@ -78,6 +80,28 @@ static bool tma_ok(const Problem& q) {
     if (!colmajor && (q.N * eb) % 16) return false;     // B pitch when stored [K][N]
     if (q.batch > 1 && ((q.sA * eb) % 16 || (q.sB * eb) % 16)) return false;
     return true;
+}
+
+// Split-K plan for problems with too few 256 x 256 tiles to occupy the CTA pairs but a long k loop:
+// S slices of kb_per_slice k-blocks (at least 8 each), so that tiles * S approaches the number of pairs.
+// Not used under CYC_FLAG_FIXED_K_ORDER (the flag promises one owner per C_ij).
+struct SplitPlan {
+    int S = 1, kb_per_slice = 0;
+};
+static SplitPlan plan_split_k(const Problem& q) {
+    SplitPlan sp;
+    if (q.flags & CYC_FLAG_FIXED_K_ORDER) return sp;
+    const int bk = 128 / elem_bytes(q.dtype);
+    const long long nkb = (q.K + bk - 1) / bk;
+    const long long tiles = q.batch * ((q.M + 255) / 256) * ((q.N + 255) / 256);
+    if (tiles * 2 > kCtaPairs || nkb < 16) return sp;
+    long long S = kCtaPairs / tiles;
+    if (S > nkb / 8) S = nkb / 8;
+    if (S < 2) return sp;
+    sp.kb_per_slice = static_cast<int>((nkb + S - 1) / S);
+    sp.S = static_cast<int>((nkb + sp.kb_per_slice - 1) / sp.kb_per_slice);  // no empty slice
+    if (sp.S < 2) sp = SplitPlan();
+    return sp;
 }
 
 static Family choose(const Problem& q) {
@@ -93,7 +117,8 @@ static Family choose(const Problem& q) {
     // 512 x 256 tiles need a long k loop (their export is not overlapped; measured break-even near 64 k-blocks,
     // a clear gain from 128) and enough tiles to occupy every CTA pair
     if (q.M > 256 && q.N > 128 && nkb >= 96 && tall_tiles >= kCtaPairs) return FAM_UMMA_TALL;
-    if (q.M > 128 && q.N > 128) return FAM_UMMA_PAIR;  // enough rows and columns for a CTA pair
+    if (q.M > 128 && q.N > 128)  // enough rows and columns for a CTA pair
+        return plan_split_k(q).S > 1 ? FAM_UMMA_SPLITK : FAM_UMMA_PAIR;
     return FAM_UMMA;
 }
 
@@ -246,8 +271,9 @@ static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
 }
 
 // ------------------------------------------------------------------ two-SM tensor-core launch
+// `ws` != nullptr: split-K -- the kernel writes plan.S planes of partial sums per problem into ws
 template <int KIND, bool B_MN>
-static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms) {
+static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws = nullptr, SplitPlan plan = SplitPlan()) {
     constexpr int STAGES = 6;
     constexpr int BK = 128 / UmmaTraits<KIND>::ELEM_BYTES;
     constexpr int CH = 128 / UmmaTraits<KIND>::ELEM_BYTES;
@@ -259,19 +285,26 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms) {
     else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, PAIR_HALF);
     if (rc) return rc;
     PairParams p;
-    p.tma_store = (reinterpret_cast<uintptr_t>(q.C) % 16 == 0 && q.N % 4 == 0 && (q.batch == 1 || q.sC % 4 == 0)) ? 1 : 0;
+    void* out = ws ? ws : q.C;
+    const long long out_planes = ws ? q.batch * plan.S : q.batch;
+    const long long out_stride = ws ? q.M * q.N : q.sC;
+    p.tma_store = (reinterpret_cast<uintptr_t>(out) % 16 == 0 && q.N % 4 == 0 && (out_planes == 1 || out_stride % 4 == 0)) ? 1 : 0;
     if (p.tma_store) {
-        rc = make_c_map(&tmC, q.dtype, q.C, q.M, q.N, q.batch, q.sC);
+        rc = make_c_map(&tmC, q.dtype, out, q.M, q.N, out_planes, out_stride);
         if (rc) return rc;
     } else {
         tmC = tmA;  // never used
     }
-    p.C = q.C;
+    p.C = out;
     p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
-    p.sC = q.sC;
+    p.sC = out_stride;
     p.tiles_m = static_cast<int>((q.M + 255) / 256);
     p.tiles_n = static_cast<int>((q.N + PAIR_BN - 1) / PAIR_BN);
-    p.num_tiles = q.batch * p.tiles_m * p.tiles_n;
+    p.num_tiles = out_planes * p.tiles_m * p.tiles_n;
+    if (ws) {
+        p.split_k = plan.S;
+        p.kb_per_slice = plan.kb_per_slice;
+    }
     CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
     auto kern = umma_pair_kernel<KIND, B_MN, STAGES>;
     CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
@@ -281,6 +314,65 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms) {
     CYC_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     return CYC_OK;
+}
+
+// ------------------------------------------------------------------ split-K
+// Workspace for the partial sums: stream-ordered allocations from a pool the library owns (one per device),
+// so that repeated calls reuse the same memory without a synchronising cudaMalloc.
+static int workspace_pool(cudaMemPool_t* out) {
+    static std::mutex mu;
+    static cudaMemPool_t pools[64] = {};
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!pools[dev]) {
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        CYC_CUDA(cudaMemPoolCreate(&pools[dev], &props));
+        unsigned long long keep = ~0ull;  // keep freed blocks for the next call instead of returning them to the driver
+        CYC_CUDA(cudaMemPoolSetAttribute(pools[dev], cudaMemPoolAttrReleaseThreshold, &keep));
+    }
+    *out = pools[dev];
+    return CYC_OK;
+}
+
+// partial sums of plan.S k-slices into the workspace (CTA-pair kernel), then their sum in slice order into C.
+// `ws` = nullptr: the workspace comes from the library's pool for the duration of the two kernels.
+template <int KIND>
+static int launch_splitk(const Problem& q, cudaStream_t st, int sms, void* ws, const SplitPlan& plan) {
+    using Out = typename UmmaTraits<KIND>::Out;
+    const long long plane = q.M * q.N;
+    const size_t bytes = static_cast<size_t>(q.batch) * plan.S * plane * sizeof(Out);
+    const bool pooled = ws == nullptr;
+    if (pooled) {
+        cudaMemPool_t pool;
+        int rc = workspace_pool(&pool);
+        if (rc) return rc;
+        CYC_CUDA(cudaMallocFromPoolAsync(&ws, bytes, pool, st));
+    }
+    const bool b_mn = (q.flags & CYC_FLAG_B_COL_MAJOR) == 0;
+    int rc = b_mn ? launch_pair_cfg<KIND, true>(q, st, sms, ws, plan) : launch_pair_cfg<KIND, false>(q, st, sms, ws, plan);
+    if (rc == CYC_OK) {
+        const int vec4 = (plane % 4 == 0 && q.sC % 4 == 0 && reinterpret_cast<uintptr_t>(q.C) % 16 == 0 &&
+                          reinterpret_cast<uintptr_t>(ws) % 16 == 0) ? 1 : 0;
+        const long long work = (vec4 ? plane / 4 : plane) * q.batch;
+        long long blocks = (work + 255) / 256;
+        if (blocks > 8ll * sms) blocks = 8ll * sms;
+        splitk_reduce_kernel<Out><<<static_cast<unsigned>(blocks), 256, 0, st>>>(static_cast<const Out*>(ws), static_cast<Out*>(q.C),
+                                                                                plane, q.sC, plan.S, q.batch, vec4);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) rc = cuda_fail(e, "splitk_reduce_kernel launch");
+        else g_launches.fetch_add(1);
+    }
+    if (pooled) {
+        cudaError_t e = cudaFreeAsync(ws, st);
+        if (e != cudaSuccess && rc == CYC_OK) rc = cuda_fail(e, "cudaFreeAsync");
+    }
+    return rc;
 }
 
 // 512 x 256 tiles: selected when the k loop is long enough to amortise the unoverlapped export
@@ -377,6 +469,7 @@ static int launch_umma(const Problem& q, cudaStream_t st) {
     const Family fam = choose(q);
     if (fam == FAM_UMMA_TALL)
         return b_mn ? launch_pair_tall_cfg<KIND, true>(q, st, di.sms) : launch_pair_tall_cfg<KIND, false>(q, st, di.sms);
+    if (fam == FAM_UMMA_SPLITK) return launch_splitk<KIND>(q, st, di.sms, nullptr, plan_split_k(q));
     if (fam == FAM_UMMA_PAIR)
         return b_mn ? launch_pair_cfg<KIND, true>(q, st, di.sms) : launch_pair_cfg<KIND, false>(q, st, di.sms);
     const bool wide = q.N > 128;
@@ -391,6 +484,7 @@ static int dispatch(const Problem& q, cudaStream_t st) {
         case FAM_UMMA:
         case FAM_UMMA_PAIR:
         case FAM_UMMA_TALL:
+        case FAM_UMMA_SPLITK:
             return q.dtype == CYC_BF16_F32 ? launch_umma<KIND_BF16>(q, st) : launch_umma<KIND_I8>(q, st);
         case FAM_UMMA_3XTF32:
             return launch_tf32x3(q, st);
@@ -472,6 +566,7 @@ extern "C" const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64
         case FAM_UMMA: return "tcgen05";
         case FAM_UMMA_PAIR: return "tcgen05_pair";
         case FAM_UMMA_TALL: return "tcgen05_pair_tall";
+        case FAM_UMMA_SPLITK: return "tcgen05_pair_splitk";
         case FAM_UMMA_3XTF32: return "tcgen05_3xtf32";
         default: return "simt";
     }

@@ -29,7 +29,21 @@ struct PairParams {
     long long num_tiles;
     int tma_store;  // 1: export through the C tensor map; 0: direct stores (unaligned C)
     int* status;
+    // split-K: the k loop of every tile is cut into `split_k` slices of `kb_per_slice` k-blocks; the tile list
+    // then runs over (batch * split_k) entries and entry e = b * split_k + s writes the partial sums of slice s
+    // to plane e of the output (a workspace that a second kernel adds up).  split_k = 1: the plain recurrence.
+    int split_k = 1;
+    int kb_per_slice = 0;
 };
+
+// k-block range [kb0, kb0 + nkb) of tile-list entry `e`, and the operand batch index it reads from
+__device__ __forceinline__ void pair_k_range(const PairParams& p, int num_kb, int e, int& b, int& kb0, int& nkb) {
+    if (p.split_k <= 1) { b = e; kb0 = 0; nkb = num_kb; return; }
+    b = e / p.split_k;
+    const int s = e - b * p.split_k;
+    kb0 = s * p.kb_per_slice;
+    nkb = min(p.kb_per_slice, num_kb - kb0);
+}
 
 constexpr int PAIR_BN = 256;        // columns of C per pair tile
 constexpr int PAIR_HALF = 128;      // B columns (and A rows) held by one CTA
@@ -101,11 +115,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             bool ok = true;
             const uint32_t full0 = ptx::mapa_u32(ptx::smem_u32(&ctl->full[0]), 0);  // the leader's full[] barriers
             for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
-                int b, tm, tn;
-                umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);
+                int e, tm, tn, b, kb0, nkb;
+                umma_tile_coord(t, p.tiles_m, p.tiles_n, e, tm, tn);
+                pair_k_range(p, num_kb, e, b, kb0, nkb);
                 const int m0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF;      // this CTA's 128 rows of cells
                 const int n0 = tn * PAIR_BN + static_cast<int>(rank) * PAIR_HALF;  // this CTA's half of the B tile
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = kb0; kb < kb0 + nkb; ++kb) {
                     if (!umma_wait(&ctl->empty[stage], phase ^ 1, ctl, p.status, 1)) { ok = false; break; }
                     uint8_t* sa = smem + stage * PAIR_STAGE_BYTES;
                     uint8_t* sb = sa + PAIR_STAGE_A;
@@ -149,7 +164,10 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!umma_wait(&ctl->acc_empty[ab], acc_phase ^ 1, ctl, p.status, 2)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * PAIR_BN);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                int e, tm, tn, b, kb0, nkb;
+                umma_tile_coord(t, p.tiles_m, p.tiles_n, e, tm, tn);
+                pair_k_range(p, num_kb, e, b, kb0, nkb);
+                for (int kb = 0; kb < nkb; ++kb) {  // the first k-block of the slice starts from zero
                     if (!umma_wait(&ctl->full[stage], phase, ctl, p.status, 3)) { ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t sa = ptx::smem_u32(smem + stage * PAIR_STAGE_BYTES);

@@ -72,6 +72,9 @@ def test_kernel_selection(binding):
     assert k(1024, 256, 256, 256, "bf16") == "tcgen05_pair"
     assert k(1, 4096, 4096, 64, "bf16") == "tcgen05_pair"        # k loop too short for the tall tiles
     assert k(1, 128, 4096, 4096, "bf16") == "tcgen05"            # one row block: a single CTA per tile
+    assert k(1, 256, 256, 8192, "bf16") == "tcgen05_pair_splitk" # one tile, 128 k-blocks
+    assert k(1, 256, 256, 8192, "bf16", fixed_k_order=True) == "tcgen05_pair"
+    assert k(1, 256, 256, 512, "bf16") == "tcgen05_pair"         # k loop too short to cut
     assert k(1, 65536, 256, 256, "f32") == "tcgen05_3xtf32"
     assert k(1, 65536, 256, 256, "f32", fixed_k_order=True) == "simt"
     assert k(1, 128, 256, 256, "f32") == "simt"

@@ -151,6 +151,22 @@ def test_umma_tall_tiles_ragged():
     check_workload(w, rows_per_problem=24)
 
 
+@pytest.mark.parametrize("case", [("bf16", 256, 256, 8192, False, 1), ("i8", 512, 256, 16400, True, 1), ("bf16", 300, 264, 4104, False, 1),
+                                  ("bf16", 300, 264, 4104, True, 1), ("i8", 260, 130, 4096, True, 1), ("bf16", 256, 256, 2048, False, 3),
+                                  ("i8", 384, 272, 8192, False, 2)])
+def test_split_k_few_tiles_long_k(case):
+    dtype, M, N, K, col, batch = case
+    w = wl(dtype, M, N, K, seed=61, col=col, batch=batch)
+    assert family(w) == "tcgen05_pair_splitk"
+    check_workload(w)
+    A, B = inputs.make_operands(w)
+    assert gpu_run(w, A, B).tobytes() == gpu_run(w, A, B).tobytes()      # slices are added in a fixed order
+    # with the fixed-order flag one CTA pair owns each output for the whole k loop
+    wf = wl(dtype, M, N, K, seed=61, col=col, batch=batch, fixed=True)
+    assert family(wf) == "tcgen05_pair"
+    check_workload(wf)
+
+
 def test_umma_many_tiles_per_cta():
     # 512 tiles on 148 SMs: every CTA walks 3-4 tiles, both TMEM accumulators and both barrier phases
     check_workload(wl("bf16", 4096, 4096, 64, seed=23), rows_per_problem=96)
