@@ -108,6 +108,40 @@ int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, int64_t K, i
                                const void* B_host, void* C_host, void* stream, unsigned flags);
 
 /*
+ * Split-K evaluation of ONE bf16 or int8 problem that never allocates (the paper has
+ * no counterpart; this is a service for hosts of the library).
+ *
+ * Who needs it: a program that gave all device memory to its own allocator at start-up,
+ * or a latency-critical loop that must never enter the driver's allocator (which may
+ * block, synchronise the device, or fail under memory pressure), cannot use the split-K
+ * path of cyc_recurrence_matmul, whose partial sums go through a stream-ordered pool.
+ * Here the partial sums go through a fixed array of CYC_STATIC_WORKSPACE_BYTES that is
+ * part of the library image: every device that loads the library holds it until the
+ * process exits, used or not.
+ *
+ *   A, B, C, stream, layouts, dtype: as for cyc_recurrence_matmul, restricted to
+ *   CYC_BF16_F32 and CYC_I8_I32, 16-byte aligned bases and row pitches, M > 128, N > 128.
+ *   flags: CYC_FLAG_B_COL_MAJOR or 0 (CYC_FLAG_FIXED_K_ORDER contradicts split-K:
+ *   CYC_ERR_INVALID_ARG).
+ * The k loop is cut into S >= 2 slices (as many as there are idle CTA pairs, >= 8
+ * k-blocks each) and S*M*N*4 bytes must fit the array; S is reduced to fit, and a
+ * problem for which not even two slices fit (2*M*N*4 > CYC_STATIC_WORKSPACE_BYTES), or
+ * whose k loop is shorter than 16 k-blocks, is refused with CYC_ERR_UNSUPPORTED and a
+ * message in cyc_last_cuda_error().  Results equal the split-K path of
+ * cyc_recurrence_matmul when both pick the same S, and stay within the usual tolerance
+ * otherwise (int8: exact).
+ * The first call on each device looks up the array's device address (a driver query, no
+ * allocation); make that first call outside any stream capture.  No call of this
+ * function allocates or frees memory.  Nothing in the array needs clearing: every
+ * element a call reads was written by the same call.  All calls share the one array, so
+ * two calls whose kernels can overlap on the GPU (different streams, no dependency) race
+ * on it: order them on one stream or with events.
+ */
+#define CYC_STATIC_WORKSPACE_BYTES (8u << 20)
+int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B, void* C,
+                                        void* stream, unsigned flags);
+
+/*
  * Synchronise `stream` and report whether a kernel enqueued by this library on
  * the current device since the previous call of this function gave up on a
  * bounded wait.  *out (HOST pointer, may be NULL) receives CYC_OK or

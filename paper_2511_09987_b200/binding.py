@@ -26,6 +26,7 @@ SYMBOLS = {
     "cyc_recurrence_matmul": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_recurrence_matmul_batched": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _i64, _ptr, _i64, _ptr, _i64, _ptr, _u32]),
     "cyc_recurrence_matmul_host": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
+    "cyc_recurrence_matmul_splitk_static": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_last_device_status": (_int, [_ptr, ctypes.POINTER(ctypes.c_int)]),
     "cyc_kernel_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
     "cyc_launch_count": (_i64, []),
@@ -57,7 +58,9 @@ _lib = _load()
 cyc_recurrence_matmul = _lib.cyc_recurrence_matmul
 cyc_recurrence_matmul_batched = _lib.cyc_recurrence_matmul_batched
 cyc_recurrence_matmul_host = _lib.cyc_recurrence_matmul_host
+cyc_recurrence_matmul_splitk_static = _lib.cyc_recurrence_matmul_splitk_static
 cyc_last_device_status = _lib.cyc_last_device_status
+CYC_STATIC_WORKSPACE_BYTES = 8 << 20
 cyc_kernel_for = _lib.cyc_kernel_for
 cyc_launch_count = _lib.cyc_launch_count
 cyc_last_cuda_error = _lib.cyc_last_cuda_error
@@ -67,7 +70,7 @@ cyc_version = _lib.cyc_version
 
 def check(status: int) -> None:
     if status != CYC_OK:
-        raise CycError(status, cyc_last_cuda_error().decode() if status == CYC_ERR_CUDA else "")
+        raise CycError(status, cyc_last_cuda_error().decode() if status in (CYC_ERR_CUDA, CYC_ERR_UNSUPPORTED) else "")
 
 
 def _flags(b_col_major: bool, fixed_k_order: bool) -> int:
@@ -135,6 +138,27 @@ def recurrence_matmul_host(A, B, C, *, b_col_major: bool = False, fixed_k_order:
         raise ValueError("bad result shape or non-contiguous tensors")
     check(cyc_recurrence_matmul_host(batch, M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(),
                                      _flags(b_col_major, fixed_k_order)))
+    return C
+
+
+def recurrence_matmul_splitk_static(A, B, C=None, *, b_col_major: bool = False):
+    """Split-K evaluation through the library's fixed workspace: the call itself allocates nothing.
+
+    For hosts that must not allocate device memory at call time; pass ``C`` to keep torch from allocating
+    the result as well.  bf16 or int8 CUDA matrices with M, N > 128; see ``include/cyc.h`` for the size limit.
+    Calls share one workspace: keep them ordered on a stream."""
+    import torch
+    if not (A.is_cuda and B.is_cuda and A.is_contiguous() and B.is_contiguous() and A.dim() == 2 and B.dim() == 2):
+        raise ValueError("A and B must be contiguous CUDA matrices")
+    code = _torch_dtype_code(A)
+    M, K = A.shape
+    N = B.shape[0] if b_col_major else B.shape[1]
+    if (B.shape[1] if b_col_major else B.shape[0]) != K or B.dtype != A.dtype:
+        raise ValueError("operand shapes or dtypes differ")
+    if C is None:
+        C = torch.empty((M, N), dtype=torch.int32 if code == CYC_I8_I32 else torch.float32, device=A.device)
+    check(cyc_recurrence_matmul_splitk_static(M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(),
+                                              _flags(b_col_major, False)))
     return C
 
 

@@ -24,6 +24,10 @@ namespace cyc {
 // raised by a kernel whose bounded wait ran out; one word per device (module scope)
 __device__ int g_device_status = 0;
 
+// Fixed workspace of cyc_recurrence_matmul_splitk_static: lives in every device that loads the library, from load
+// to exit.  In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.
+static __device__ __align__(256) unsigned char g_static_workspace[CYC_STATIC_WORKSPACE_BYTES];
+
 static std::atomic<long long> g_launches{0};
 static thread_local char g_err[512] = "";
 
@@ -542,6 +546,66 @@ extern "C" int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, i
     cudaFreeAsync(d, st);
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess && !rc) rc = cuda_fail(e, "cudaStreamSynchronize");
     return rc;
+}
+
+// Device address of the fixed workspace on the current device, looked up once per device.
+static int static_workspace_address(void** out) {
+    static std::mutex mu;
+    static void* addr[64] = {};
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        CYC_CUDA(cudaGetSymbolAddress(&p, g_static_workspace));  // the current device's copy of the array
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return CYC_OK;
+}
+
+extern "C" int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
+                                                   void* C, void* stream, unsigned flags) {
+    if (M <= 0 || N <= 0 || K <= 0) return CYC_ERR_INVALID_ARG;
+    if (flags & CYC_FLAG_FIXED_K_ORDER) return CYC_ERR_INVALID_ARG;  // the flag asks for one owner per C_ij; this schedule has several
+    Problem q{1, M, N, K, dtype, A, B, C, M * K, K * N, M * N, flags};
+    int rc = validate(q);
+    if (rc) return rc;
+    if (dtype == CYC_F32 || !tma_ok(q) || M <= 128 || N <= 128) {
+        snprintf(g_err, sizeof g_err, "split-K needs bf16 or int8 operands, 16-byte aligned bases and pitches, M > 128 and N > 128");
+        return CYC_ERR_UNSUPPORTED;
+    }
+    // as many k-slices as there are idle CTA pairs, at least 8 k-blocks each, and no more than fit the fixed array
+    const int bk = 128 / elem_bytes(dtype);
+    const long long nkb = (K + bk - 1) / bk;
+    const long long tiles = ((M + 255) / 256) * ((N + 255) / 256);
+    const long long plane_bytes = M * N * 4;
+    long long S = kCtaPairs / tiles;
+    if (S > nkb / 8) S = nkb / 8;
+    if (S > static_cast<long long>(CYC_STATIC_WORKSPACE_BYTES) / plane_bytes) S = static_cast<long long>(CYC_STATIC_WORKSPACE_BYTES) / plane_bytes;
+    if (S < 2) {
+        snprintf(g_err, sizeof g_err,
+                 "no split-K plan fits: need >= 2 slices of >= 8 k-blocks, at most %lld CTA pairs' worth of tiles, and "
+                 "2*M*N*4 bytes <= the fixed workspace of %lld bytes",
+                 static_cast<long long>(kCtaPairs), static_cast<long long>(CYC_STATIC_WORKSPACE_BYTES));
+        return CYC_ERR_UNSUPPORTED;
+    }
+    SplitPlan plan;
+    plan.kb_per_slice = static_cast<int>((nkb + S - 1) / S);
+    plan.S = static_cast<int>((nkb + plan.kb_per_slice - 1) / plan.kb_per_slice);
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc) return rc;
+    if (di.cc_major != 10) {
+        snprintf(g_err, sizeof g_err, "tensor-core kernels need an sm_100 device");
+        return CYC_ERR_UNSUPPORTED;
+    }
+    void* ws = nullptr;
+    rc = static_workspace_address(&ws);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return dtype == CYC_BF16_F32 ? launch_splitk<KIND_BF16>(q, st, di.sms, ws, plan) : launch_splitk<KIND_I8>(q, st, di.sms, ws, plan);
 }
 
 extern "C" int cyc_last_device_status(void* stream, int* out) {
