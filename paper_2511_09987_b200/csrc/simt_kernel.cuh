@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(SIMT_THREADS, 2) simt_recurrence_kernel(const 
 // Small problems (fewer 128 x 128 tiles than half the SMs): 64 x 64 tiles, 4 x 4 outputs per
 // thread, so that more SMs take part and the per-thread chain work shrinks.  Same chains, same
 // order, same bits; element-wise guarded loads (any shape, any alignment).
-constexpr int SIMT_S_BM = 64, SIMT_S_BN = 64, SIMT_S_BK = 16;
+constexpr int SIMT_S_BM = 64, SIMT_S_BN = 64, SIMT_S_BK = 64;  // a deep slab: one round trip to memory per 64 k
 
 template <typename TIn, typename TAcc>
 __global__ void __launch_bounds__(SIMT_THREADS) simt_recurrence_small_kernel(const SimtParams p) {
@@ -234,24 +234,30 @@ __global__ void __launch_bounds__(SIMT_THREADS) simt_recurrence_small_kernel(con
         for (int j = 0; j < 4; ++j) acc[i][j] = TAcc(0);  // [i,0-1]_C = 0
 
     for (int k0 = 0; k0 < K; k0 += SIMT_S_BK) {
-        // 64 x 16 elements of A and 16 x 64 of B: four of each per thread
+        // 64 x 64 elements of A and of B: sixteen of each per thread, all loads issued before the first use
+        TAcc ra[16], rb[16];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < 16; ++e) {
             const int idx = tid + e * SIMT_THREADS;
-            const int r = idx >> 4, kk = idx & 15;
-            TAcc v = TAcc(0);
-            if (m0 + r < M && k0 + kk < K) v = simt_widen<TIn, TAcc>(A[static_cast<long long>(m0 + r) * K + k0 + kk]);
-            As[kk][r] = v;
+            const int r = idx >> 6, kk = idx & 63;
+            ra[e] = TAcc(0);
+            if (m0 + r < M && k0 + kk < K) ra[e] = simt_widen<TIn, TAcc>(A[static_cast<long long>(m0 + r) * K + k0 + kk]);
         }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < 16; ++e) {
             const int idx = tid + e * SIMT_THREADS;
             int kk, j;
             if (p.b_sj == 1) { kk = idx >> 6; j = idx & 63; }
-            else { kk = idx & 15; j = idx >> 4; }
-            TAcc v = TAcc(0);
-            if (k0 + kk < K && n0 + j < N) v = simt_widen<TIn, TAcc>(B[static_cast<long long>(k0 + kk) * p.b_sk + static_cast<long long>(n0 + j) * p.b_sj]);
-            Bs[kk][j] = v;
+            else { kk = idx & 63; j = idx >> 6; }
+            rb[e] = TAcc(0);
+            if (k0 + kk < K && n0 + j < N) rb[e] = simt_widen<TIn, TAcc>(B[static_cast<long long>(k0 + kk) * p.b_sk + static_cast<long long>(n0 + j) * p.b_sj]);
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const int idx = tid + e * SIMT_THREADS;
+            As[idx & 63][idx >> 6] = ra[e];
+            if (p.b_sj == 1) Bs[idx >> 6][idx & 63] = rb[e];
+            else Bs[idx & 63][idx >> 6] = rb[e];
         }
         __syncthreads();
         const int kmax = min(SIMT_S_BK, K - k0);  // never run a chain past k_end
