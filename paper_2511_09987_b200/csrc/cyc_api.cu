@@ -519,6 +519,9 @@ extern "C" int cyc_recurrence_matmul_batched(int64_t batch, int64_t M, int64_t N
     return dispatch(q, static_cast<cudaStream_t>(stream));
 }
 
+// Host-buffer evaluation.  Device buffers come from the library's pool; for large problems the rows of A and C (or the
+// problems of a batch) are cut into chunks so that the upload of chunk i+1, the kernel of chunk i and the download of
+// chunk i-1 overlap (two helper streams, ordered against the caller's stream by events).
 extern "C" int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A_host,
                                           const void* B_host, void* C_host, void* stream, unsigned flags) {
     if (batch <= 0 || M <= 0 || N <= 0 || K <= 0 || !A_host || !B_host || !C_host) return CYC_ERR_INVALID_ARG;
@@ -530,19 +533,94 @@ extern "C" int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, i
                  nc = static_cast<size_t>(batch) * M * N * 4;
     // one allocation, three 256-byte aligned regions
     const size_t oa = 0, ob = (na + 255) & ~static_cast<size_t>(255), oc = ob + ((nb + 255) & ~static_cast<size_t>(255));
+    cudaMemPool_t pool;
+    int rc = workspace_pool(&pool);
+    if (rc) return rc;
     uint8_t* d = nullptr;
-    CYC_CUDA(cudaMallocAsync(reinterpret_cast<void**>(&d), oc + nc, st));
-    int rc = CYC_OK;
-    cudaError_t e;
-    if ((e = cudaMemcpyAsync(d + oa, A_host, na, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(d + ob, B_host, nb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-        rc = cuda_fail(e, "cudaMemcpyAsync(host to device)");
-    if (!rc) {
-        Problem q{batch, M, N, K, dtype, d + oa, d + ob, d + oc, M * K, K * N, M * N, flags};
-        rc = dispatch(q, st);
+    CYC_CUDA(cudaMallocFromPoolAsync(reinterpret_cast<void**>(&d), oc + nc, pool, st));
+    const uint8_t* hA = static_cast<const uint8_t*>(A_host);
+    const uint8_t* hB = static_cast<const uint8_t*>(B_host);
+    uint8_t* hC = static_cast<uint8_t*>(C_host);
+    cudaError_t e = cudaSuccess;
+
+    // chunks: rows of one problem (multiples of 512), or whole problems of a batch
+    const bool by_rows = batch == 1;
+    const long long units = by_rows ? M : batch;
+    long long nch = (na + nc) > (16u << 20) ? 4 : 1;
+    long long per = (units + nch - 1) / nch;
+    if (by_rows) per = (per + 511) / 512 * 512;
+    if (per < 1) per = 1;
+    nch = (units + per - 1) / per;
+
+    if (nch <= 1) {
+        if ((e = cudaMemcpyAsync(d + oa, hA, na, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(d + ob, hB, nb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+            rc = cuda_fail(e, "cudaMemcpyAsync(host to device)");
+        if (!rc) {
+            Problem q{batch, M, N, K, dtype, d + oa, d + ob, d + oc, M * K, K * N, M * N, flags};
+            rc = dispatch(q, st);
+        }
+        if (!rc && (e = cudaMemcpyAsync(hC, d + oc, nc, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+            rc = cuda_fail(e, "cudaMemcpyAsync(device to host)");
+    } else {
+        cudaStream_t up = nullptr, down = nullptr;
+        cudaEvent_t ev_start = nullptr, ev_up[8] = {}, ev_done[8] = {}, ev_down = nullptr;
+        auto ok = [&](cudaError_t err, const char* what) {
+            if (err != cudaSuccess && !rc) rc = cuda_fail(err, what);
+            return rc == CYC_OK;
+        };
+        ok(cudaStreamCreateWithFlags(&up, cudaStreamNonBlocking), "cudaStreamCreateWithFlags");
+        ok(cudaStreamCreateWithFlags(&down, cudaStreamNonBlocking), "cudaStreamCreateWithFlags");
+        ok(cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming), "cudaEventCreateWithFlags");
+        ok(cudaEventCreateWithFlags(&ev_down, cudaEventDisableTiming), "cudaEventCreateWithFlags");
+        for (long long c = 0; c < nch && !rc; ++c) {
+            ok(cudaEventCreateWithFlags(&ev_up[c], cudaEventDisableTiming), "cudaEventCreateWithFlags");
+            ok(cudaEventCreateWithFlags(&ev_done[c], cudaEventDisableTiming), "cudaEventCreateWithFlags");
+        }
+        if (!rc) {
+            // the helper streams start after whatever the caller's stream holds (the allocation included)
+            ok(cudaEventRecord(ev_start, st), "cudaEventRecord");
+            ok(cudaStreamWaitEvent(up, ev_start, 0), "cudaStreamWaitEvent");
+            ok(cudaStreamWaitEvent(down, ev_start, 0), "cudaStreamWaitEvent");
+            if (by_rows) ok(cudaMemcpyAsync(d + ob, hB, nb, cudaMemcpyHostToDevice, up), "cudaMemcpyAsync(B)");
+        }
+        for (long long c = 0; c < nch && !rc; ++c) {
+            const long long u0 = c * per, un = (u0 + per <= units ? per : units - u0);
+            // element offsets of this chunk in A, B, C
+            const size_t a_off = static_cast<size_t>(u0) * (by_rows ? K : M * K) * eb, a_len = static_cast<size_t>(un) * (by_rows ? K : M * K) * eb;
+            const size_t c_off = static_cast<size_t>(u0) * (by_rows ? N : M * N) * 4, c_len = static_cast<size_t>(un) * (by_rows ? N : M * N) * 4;
+            const size_t b_off = by_rows ? 0 : static_cast<size_t>(u0) * K * N * eb, b_len = by_rows ? 0 : static_cast<size_t>(un) * K * N * eb;
+            ok(cudaMemcpyAsync(d + oa + a_off, hA + a_off, a_len, cudaMemcpyHostToDevice, up), "cudaMemcpyAsync(A chunk)");
+            if (b_len) ok(cudaMemcpyAsync(d + ob + b_off, hB + b_off, b_len, cudaMemcpyHostToDevice, up), "cudaMemcpyAsync(B chunk)");
+            ok(cudaEventRecord(ev_up[c], up), "cudaEventRecord");
+            ok(cudaStreamWaitEvent(st, ev_up[c], 0), "cudaStreamWaitEvent");
+            if (!rc) {
+                Problem q{by_rows ? 1 : un, by_rows ? un : M, N, K, dtype, d + oa + a_off, d + ob + b_off, d + oc + c_off, (by_rows ? un : M) * K, K * N,
+                          (by_rows ? un : M) * N, flags};
+                rc = dispatch(q, st);
+            }
+            ok(cudaEventRecord(ev_done[c], st), "cudaEventRecord");
+            ok(cudaStreamWaitEvent(down, ev_done[c], 0), "cudaStreamWaitEvent");
+            ok(cudaMemcpyAsync(hC + c_off, d + oc + c_off, c_len, cudaMemcpyDeviceToHost, down), "cudaMemcpyAsync(C chunk)");
+        }
+        // the caller's stream continues (and the buffer is freed) only after the last download
+        if (down) {
+            if (ev_down && cudaEventRecord(ev_down, down) == cudaSuccess) cudaStreamWaitEvent(st, ev_down, 0);
+            else cudaStreamSynchronize(down);
+        }
+        if (up && rc) cudaStreamSynchronize(up);
+        cudaFreeAsync(d, st);
+        if ((e = cudaStreamSynchronize(st)) != cudaSuccess && !rc) rc = cuda_fail(e, "cudaStreamSynchronize");
+        if (up) { cudaStreamSynchronize(up); cudaStreamDestroy(up); }
+        if (down) { cudaStreamSynchronize(down); cudaStreamDestroy(down); }
+        if (ev_start) cudaEventDestroy(ev_start);
+        if (ev_down) cudaEventDestroy(ev_down);
+        for (int c = 0; c < 8; ++c) {
+            if (ev_up[c]) cudaEventDestroy(ev_up[c]);
+            if (ev_done[c]) cudaEventDestroy(ev_done[c]);
+        }
+        return rc;
     }
-    if (!rc && (e = cudaMemcpyAsync(C_host, d + oc, nc, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-        rc = cuda_fail(e, "cudaMemcpyAsync(device to host)");
     cudaFreeAsync(d, st);
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess && !rc) rc = cuda_fail(e, "cudaStreamSynchronize");
     return rc;

@@ -232,6 +232,38 @@ def test_host_entry_point():
     assert hC.numpy().tobytes() == gpu_run(w, A, B).tobytes()
 
 
+@pytest.mark.parametrize("case", [("bf16", 3000, 1024, 2048, 1, False), ("i8", 256, 256, 1024, 40, True), ("f32", 2500, 512, 1024, 1, False)])
+def test_host_entry_point_chunked_pipeline(case):
+    # large enough (> 16 MB of A and C) for the chunked upload / compute / download pipeline; ragged last chunk
+    import torch
+    from paper_2511_09987_b200 import binding
+    dtype, M, N, K, batch, col = case
+    w = wl(dtype, M, N, K, seed=32, batch=batch, col=col)
+    A, B = inputs.make_operands(w)
+    hA, hB = torch.from_numpy(A), torch.from_numpy(B)
+    if dtype == "bf16":
+        hA, hB = hA.view(torch.bfloat16), hB.view(torch.bfloat16)
+    hA, hB = hA.pin_memory(), hB.pin_memory()
+    shape = (batch, M, N) if batch > 1 else (M, N)
+    hC = torch.full(shape, 7, dtype=torch.int32 if dtype == "i8" else torch.float32).pin_memory()
+    binding.recurrence_matmul_host(hA, hB, hC, b_col_major=col)
+    want = gpu_run(w, A, B)
+    got = hC.numpy()
+    if dtype == "i8":
+        assert (got == want).all()
+    else:
+        # a chunk of rows may be served by another kernel than the whole problem: compare within the tolerance
+        prob = range(batch) if batch > 1 else [None]
+        for b in prob:
+            Ab, Bb, g, wv = (A, B, got, want) if b is None else (A[b], B[b], got[b], want[b])
+            rows = np.unique(np.concatenate([[0, M - 1], np.random.default_rng(3).integers(0, M, 40)]))
+            S, _ = oracle.abs_sum_rows(dtype, Ab, Bb, b_col_major=col, rows=rows, threads=8)
+            tol = 4e-3 if dtype == "bf16" else 1e-5
+            assert (np.abs(g[rows].astype(np.float64) - wv[rows]) <= 2 * tol * S).all()
+            ref = oracle.collapsed(dtype, Ab, Bb, b_col_major=col, rows=rows, threads=8)
+            assert (np.abs(g[rows].astype(np.float64) - ref) <= tol * S).all()
+
+
 def test_device_status_is_clean():
     from paper_2511_09987_b200 import binding
     assert binding.last_device_status() == binding.CYC_OK
