@@ -364,9 +364,9 @@ static int launch_splitk(const Problem& q, cudaStream_t st, int sms, void* ws, c
         const int vec4 = (plane % 4 == 0 && q.sC % 4 == 0 && reinterpret_cast<uintptr_t>(q.C) % 16 == 0 &&
                           reinterpret_cast<uintptr_t>(ws) % 16 == 0) ? 1 : 0;
         const long long work = (vec4 ? plane / 4 : plane) * q.batch;
-        long long blocks = (work + 255) / 256;
-        if (blocks > 8ll * sms) blocks = 8ll * sms;
-        splitk_reduce_kernel<Out><<<static_cast<unsigned>(blocks), 256, 0, st>>>(static_cast<const Out*>(ws), static_cast<Out*>(q.C),
+        long long blocks = (work + 127) / 128;  // short kernel: spread the work over as many SMs as possible
+        if (blocks > 16ll * sms) blocks = 16ll * sms;
+        splitk_reduce_kernel<Out><<<static_cast<unsigned>(blocks), 128, 0, st>>>(static_cast<const Out*>(ws), static_cast<Out*>(q.C),
                                                                                 plane, q.sC, plan.S, q.batch, vec4);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) rc = cuda_fail(e, "splitk_reduce_kernel launch");

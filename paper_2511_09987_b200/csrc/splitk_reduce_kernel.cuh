@@ -9,7 +9,7 @@ namespace cyc {
 
 // ws: [batch][S][plane] ; C: [batch] planes with stride sC ; plane = M*N elements
 template <typename T>
-__global__ void __launch_bounds__(256) splitk_reduce_kernel(const T* __restrict__ ws, T* __restrict__ C, long long plane,
+__global__ void __launch_bounds__(128) splitk_reduce_kernel(const T* __restrict__ ws, T* __restrict__ C, long long plane,
                                                             long long sC, int S, long long batch, int vec4) {
     const long long per_batch = vec4 ? plane / 4 : plane;
     const long long total = per_batch * batch;
@@ -20,7 +20,15 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const T* __restrict_
         if (vec4) {
             using V = typename std::conditional<sizeof(T) == 4 && std::is_floating_point<T>::value, float4, int4>::type;
             V acc = reinterpret_cast<const V*>(src)[r];
-            for (int s = 1; s < S; ++s) {
+            int s = 1;
+            for (; s + 8 <= S; s += 8) {  // eight loads in flight, added in slice order
+                V v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = reinterpret_cast<const V*>(src + static_cast<long long>(s + u) * plane)[r];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+            }
+            for (; s < S; ++s) {
                 const V v = reinterpret_cast<const V*>(src + static_cast<long long>(s) * plane)[r];
                 acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
             }
