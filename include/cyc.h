@@ -150,6 +150,15 @@ int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t K, int dty
  */
 int cyc_last_device_status(void* stream, int* out);
 
+/*
+ * Self-test of the failure path (no counterpart in the paper): enqueue a one-CTA kernel whose
+ * only wait can never be satisfied and which gives up after `budget_cycles` SM clocks
+ * (1 .. 2^24, i.e. at most about ten milliseconds), exactly as the bounded waits of the real
+ * kernels do.  The kernel ends normally; the next cyc_last_device_status reports
+ * CYC_ERR_TIMEOUT once and the device stays usable.
+ */
+int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles);
+
 /* Name of the kernel the dispatcher would pick for these arguments -- "simt" (general
  * kernel), "tcgen05" (one CTA per tile), "tcgen05_pair" (CTA pair, 256x256 tiles),
  * "tcgen05_pair_tall" (CTA pair, 512x256 tiles), "tcgen05_pair_splitk" (few tiles, long k

@@ -27,6 +27,7 @@ SYMBOLS = {
     "cyc_recurrence_matmul_batched": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _i64, _ptr, _i64, _ptr, _i64, _ptr, _u32]),
     "cyc_recurrence_matmul_host": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_recurrence_matmul_splitk_static": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
+    "cyc_selftest_bounded_wait": (_int, [_ptr, _i64]),
     "cyc_last_device_status": (_int, [_ptr, ctypes.POINTER(ctypes.c_int)]),
     "cyc_kernel_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
     "cyc_launch_count": (_i64, []),
@@ -59,6 +60,7 @@ cyc_recurrence_matmul = _lib.cyc_recurrence_matmul
 cyc_recurrence_matmul_batched = _lib.cyc_recurrence_matmul_batched
 cyc_recurrence_matmul_host = _lib.cyc_recurrence_matmul_host
 cyc_recurrence_matmul_splitk_static = _lib.cyc_recurrence_matmul_splitk_static
+cyc_selftest_bounded_wait = _lib.cyc_selftest_bounded_wait
 cyc_last_device_status = _lib.cyc_last_device_status
 CYC_STATIC_WORKSPACE_BYTES = 8 << 20
 cyc_kernel_for = _lib.cyc_kernel_for

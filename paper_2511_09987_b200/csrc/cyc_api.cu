@@ -28,6 +28,34 @@ __device__ int g_device_status = 0;
 // to exit.  In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.
 static __device__ __align__(256) unsigned char g_static_workspace[CYC_STATIC_WORKSPACE_BYTES];
 
+// Self-test of the bounded-wait path: one CTA waits on an mbarrier that nothing ever arrives on, with a
+// caller-chosen clock budget, and reports through the same status word and abort flag as the real kernels.
+__global__ void bounded_wait_selftest_kernel(long long budget_cycles, int* status) {
+    __shared__ uint64_t bar;
+    __shared__ volatile int abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(&bar, 0)) {
+            if (clock64() - t0 > budget_cycles) {
+                abort_flag = 1;
+                atomicExch(status, 0x7f0);
+                break;
+            }
+        }
+    } else {
+        // the other role polls the abort flag the way the kernels' roles do, with its own (larger) budget
+        const long long t0 = clock64();
+        while (!abort_flag && clock64() - t0 < 64 * budget_cycles) {}
+    }
+    __syncthreads();
+}
+
 static std::atomic<long long> g_launches{0};
 static thread_local char g_err[512] = "";
 
@@ -684,6 +712,16 @@ extern "C" int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == CYC_BF16_F32 ? launch_splitk<KIND_BF16>(q, st, di.sms, ws, plan) : launch_splitk<KIND_I8>(q, st, di.sms, ws, plan);
+}
+
+extern "C" int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles) {
+    if (budget_cycles < 1 || budget_cycles > (1ll << 24)) return CYC_ERR_INVALID_ARG;  // at most ~10 ms
+    int* status = nullptr;
+    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_device_status));
+    bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(budget_cycles, status);
+    CYC_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return CYC_OK;
 }
 
 extern "C" int cyc_last_device_status(void* stream, int* out) {

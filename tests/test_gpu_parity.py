@@ -264,6 +264,58 @@ def test_host_entry_point_chunked_pipeline(case):
             assert (np.abs(g[rows].astype(np.float64) - ref) <= tol * S).all()
 
 
+def test_bounded_wait_reports_timeout_and_device_stays_usable():
+    # a wait that nothing satisfies runs out of its (short) budget: the kernel returns, the status word says so once,
+    # and the next evaluation on the same device is correct
+    import torch
+    from paper_2511_09987_b200 import binding
+    assert binding.last_device_status() == binding.CYC_OK
+    stream = torch.cuda.current_stream().cuda_stream
+    assert binding.cyc_selftest_bounded_wait(stream, 0) == binding.CYC_ERR_INVALID_ARG
+    assert binding.cyc_selftest_bounded_wait(stream, 1 << 30) == binding.CYC_ERR_INVALID_ARG
+    assert binding.cyc_selftest_bounded_wait(stream, 100000) == binding.CYC_OK
+    assert binding.last_device_status() == binding.CYC_ERR_TIMEOUT
+    assert b"wait ran out" in binding.cyc_last_cuda_error()
+    assert binding.last_device_status() == binding.CYC_OK          # reported once, then cleared
+    check_workload(wl("bf16", 300, 520, 200, seed=33))
+
+
+def test_two_host_threads_on_two_streams():
+    import threading
+    import torch
+    from paper_2511_09987_b200 import binding
+    results, errors = {}, []
+    cases = {0: wl("bf16", 512, 512, 512, seed=34), 1: wl("i8", 384, 528, 400, seed=35, col=True)}
+    ops = {k: inputs.make_operands(w) for k, w in cases.items()}
+
+    def work(k):
+        try:
+            w = cases[k]
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                dA, dB = to_device(ops[k][0], w.dtype), to_device(ops[k][1], w.dtype)
+                outs = [binding.recurrence_matmul(dA, dB, b_col_major=w.b_col_major) for _ in range(20)]
+                s.synchronize()
+            results[k] = [o.cpu().numpy() for o in (outs[0], outs[-1])]
+        except Exception as exc:  # noqa: BLE001
+            errors.append(exc)
+
+    threads = [threading.Thread(target=work, args=(k,)) for k in cases]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for k, w in cases.items():
+        ref = oracle.collapsed(w.dtype, ops[k][0], ops[k][1], b_col_major=w.b_col_major, threads=4)
+        for got in results[k]:
+            if w.dtype == "i8":
+                assert (got == ref).all()
+            else:
+                S, _ = oracle.abs_sum_rows(w.dtype, ops[k][0], ops[k][1], threads=4)
+                assert (np.abs(got.astype(np.float64) - ref) <= 4e-3 * S).all()
+
+
 def test_device_status_is_clean():
     from paper_2511_09987_b200 import binding
     assert binding.last_device_status() == binding.CYC_OK
