@@ -315,7 +315,7 @@ def run_ours(args, w):
     # ---- roofline of the dominant (only) kernel: one launch per step
     kernel_s = ms_per_step * 1e-3
     bound = bound_of(w, family)
-    traffic = load_traffic(w)
+    traffic = load_traffic(w, family)
     if bound == "hbm":
         achieved, peak, runit = w.algorithmic_bytes / kernel_s / 1e9, float(peaks["hbm_gbs"]), "GB/s"
         peak_note = "%s STREAM-style copy" % peak_kind
@@ -360,27 +360,38 @@ def run_ours(args, w):
     reps.close()
 
 
-def kernel_source_digest():
-    """sha256 over the CUDA sources: ties a stored DRAM-traffic figure to the kernels it was taken from."""
+# CUDA sources each kernel family is built from (host-side launch code is not part of a kernel's identity)
+KERNEL_SOURCES = {
+    "simt": ["simt_kernel.cuh"],
+    "tcgen05": ["ptx.cuh", "umma_kernel.cuh"],
+    "tcgen05_pair": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh"],
+    "tcgen05_pair_tall": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "umma_pair_tall_kernel.cuh"],
+    "tcgen05_pair_splitk": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "splitk_reduce_kernel.cuh"],
+    "tcgen05_3xtf32": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "umma_pair_tf32x3_kernel.cuh"],
+}
+
+
+def kernel_source_digest(family):
+    """sha256 over the CUDA sources of one kernel family: ties a stored DRAM-traffic figure to the kernel it was taken from."""
     import hashlib
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2511_09987_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
+    for name in KERNEL_SOURCES.get(family, sorted(os.listdir(csrc))):
         with open(os.path.join(csrc, name), "rb") as f:
             h.update(name.encode())
             h.update(f.read())
     return h.hexdigest()[:16]
 
 
-def load_traffic(w):
+def load_traffic(w, family):
     """DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) for this workload's kernel.
 
     Read from profiles/dram_traffic.txt, lines `workload bytes digest`; a figure whose digest does not match the
-    current kernel sources is stale and reported as null."""
+    current sources of the kernel is stale and reported as null."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     if not os.path.exists(path):
         return None
-    digest = kernel_source_digest()
+    digest = kernel_source_digest(family)
     with open(path) as f:
         for line in f:
             parts = line.split()
