@@ -271,7 +271,7 @@ def run_ours(args, w):
     ms = e0.elapsed_time(e1)
     launches = args.steps if graph is not None else binding.cyc_launch_count() - launches0
     if binding.last_device_status() != binding.CYC_OK:
-        raise SystemExit("a device-side wait timed out during the benchmark")
+        raise SystemExit("a device-side wait timed out during the benchmark: " + binding.cyc_last_cuda_error().decode())
     # keep the GPU loaded a little longer if the timed region was too short to catch a clock sample
     extra_note = None
     if len(sampler.samples) < 3:

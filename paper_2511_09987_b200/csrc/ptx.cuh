@@ -28,17 +28,16 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// arrive on the barrier at the same offset in CTA `cta` of this cluster.  Default semantics (release at CTA scope), as
-// for a local arrive: a release at CLUSTER scope was measured to hold the arriving thread for about 1300 clocks, which
-// turns any per-k-block cross-CTA signal into the bottleneck.  What the arrivals here publish to the other CTA is either
-// data written by TMA (complete before the arriving thread saw its own barrier flip), shared-memory writes already made
-// visible to the async proxy by fence.proxy.async, or the fact that TMEM has been read.
+// arrive on the barrier at the same offset in CTA `cta` of this cluster, releasing at CLUSTER scope: what the arrival
+// publishes (shared-memory writes of this CTA, the fact that TMEM has been read) must be ordered for a thread of
+// another CTA.  It is expensive -- the arriving thread is held for about 1300 clocks -- but a CTA-scope release here was
+// measured to stall the 3xTF32 pipeline now and then (caught by the bounded waits), so the cost is paid.
 __device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t cta) {
     asm volatile(
         "{\n"
         ".reg .b32 ra;\n"
         "mapa.shared::cluster.u32 ra, %0, %1;\n"
-        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n"
         "}" ::"r"(smem_u32(bar)),
         "r"(cta)
         : "memory");
