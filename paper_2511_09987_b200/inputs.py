@@ -170,3 +170,67 @@ def scaled(w: Workload, **kw) -> Workload:
              fixed_k_order=w.fixed_k_order, a_dist=w.a_dist, b_dist=w.b_dist)
     d.update(kw)
     return Workload(**d)
+
+
+# ---------------------------------------------------------------------- block triangular solve
+TENSOR_L = 2
+TENSOR_L_DIAG = 3
+TENSOR_RHS = 4
+
+
+@dataclass(frozen=True)
+class TrsmWorkload:
+    """Synthetic ``L X = B``: ``L`` lower triangular ``[n][n]``, ``B`` ``[n][m]`` (``m`` right-hand sides), fp32.
+
+    ``coupling`` selects the strictly-lower part (``u`` uniform in ``[-1,1)``):
+
+    * ``"dominant"``: ``L_ij = 0.5 * u_ij / i`` -- every row is diagonally dominant (off-diagonal absolute row sum
+      below 0.5, diagonal magnitude in ``[1,2)``), so the inverse is bounded by 2 in the infinity norm;
+    * ``"sqrt"``: ``L_ij = u_ij / sqrt(n)`` -- the off-diagonal sum of a row is of order one.
+
+    The diagonal is ``+-(1 + v)``, ``v`` uniform in ``[0,1)``, the sign from one more bit.  The strictly upper part is
+    filled with ``upper`` (NaN by default: it must never be read).
+    """
+    name: str
+    n: int
+    m: int
+    tile: int
+    seed: int
+    coupling: str = "dominant"
+    upper: float = float("nan")
+
+    @property
+    def flops(self) -> int:
+        """Multiply-adds of the substitution counted as two operations: ``n (n+1) m``."""
+        return self.n * (self.n + 1) * self.m
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        """Lower triangle of L and B read once, X written once."""
+        return (self.n * (self.n + 1) // 2 + 2 * self.n * self.m) * 4
+
+
+TRSM_WORKLOADS = {
+    "t1": TrsmWorkload("t1", 512, 96, 64, seed=10),
+    "t2": TrsmWorkload("t2", 8192, 4096, 256, seed=11),
+}
+
+
+def make_trsm_operands(w: TrsmWorkload):
+    """Host arrays ``(L, B)`` (float32) for a triangular-solve workload."""
+    n, m = w.n, w.m
+    u = uniform_f32(w.seed, TENSOR_L, n * n, -1.0, 1.0).reshape(n, n)
+    if w.coupling == "dominant":
+        scale = (0.5 / np.maximum(np.arange(n, dtype=np.float64), 1.0)).astype(np.float32)[:, None]
+    elif w.coupling == "sqrt":
+        scale = np.float32(1.0 / np.sqrt(float(n)))
+    else:
+        raise ValueError("unknown coupling %r" % (w.coupling,))
+    L = (u * scale).astype(np.float32)
+    v = uniform_f32(w.seed, TENSOR_L_DIAG, n, 0.0, 1.0)
+    sign = np.where((_bits(w.seed, TENSOR_L_DIAG, n, n) >> np.uint64(63)).astype(bool), np.float32(-1.0), np.float32(1.0))
+    rows, cols = np.indices((n, n), sparse=True)
+    L[rows < cols] = np.float32(w.upper)
+    L[np.arange(n), np.arange(n)] = sign * (np.float32(1.0) + v)
+    B = uniform_f32(w.seed, TENSOR_RHS, n * m, -1.0, 1.0).reshape(n, m)
+    return L, B
