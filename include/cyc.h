@@ -142,6 +142,40 @@ int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t K, int dty
                                         void* stream, unsigned flags);
 
 /*
+ * Block lower-triangular solve  L X = B  (Section "Multiple Iteration Spaces":
+ *     X_i = TRSM( L_ii , B_i - sum_{j<i} GEMM(L_ij, X_j) ),
+ * recurrences of Figure "deps-tri-solve"): a triangular iteration space of tile products
+ * whose accumulators run along j, and a diagonal space of small triangular solves that
+ * consume the end of each row and seed the next block column.
+ *
+ *   n      order of L;  m  number of right-hand sides (columns of B and X);  n, m >= 1
+ *   tile   edge T of the square tiles of both spaces, 1 .. 256; 0 selects 256.  The last
+ *          tile may be ragged.  T changes only the grouping of the additions (results
+ *          differ by roundings), not the mathematical result.
+ *   dtype  CYC_F32 (fp32 in, fp32 arithmetic, fp32 out); the other types are refused
+ *          with CYC_ERR_UNSUPPORTED
+ *   L      DEVICE, [n][n] row-major; only entries on and below the diagonal are read
+ *          (the rest may hold anything, NaN included).  A zero on the diagonal gives
+ *          infinities or NaN in X, as the division does; it is not an error.
+ *   B      DEVICE, [n][m] row-major
+ *   X      DEVICE, [n][m] row-major, fully overwritten.  X may be the very same buffer as
+ *          B (in place); any other overlap of X with B or L is CYC_ERR_INVALID_ARG.
+ *   stream cudaStream_t; every kernel is enqueued there, the call does not synchronise
+ *   flags  0, or CYC_FLAG_FIXED_K_ORDER: the tile products then run as per-element fp32
+ *          fused-multiply-add chains in increasing k (bit-reproducible, slower); without
+ *          it they may run on the tensor cores (fp32 split into TF32 parts).
+ * The tile products of the triangular space are evaluated by the same kernels as
+ * cyc_recurrence_matmul (operand A = a sub-block of L, row pitch n); their partial sums
+ * pass through a workspace of ceil(log2(ceil(n/T))) * n * m * 4 bytes taken from the
+ * library's stream-ordered pool for the duration of the call.  The diagonal tiles are
+ * solved by forward substitution in fp32 (x_k = s_k * (1 / L_kk)).  Caller owns L, B, X;
+ * the library keeps no reference after the kernels complete.  Errors as for
+ * cyc_recurrence_matmul.
+ */
+int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, const void* L, const void* B, void* X, void* stream,
+                   unsigned flags);
+
+/*
  * Synchronise `stream` and report whether a kernel enqueued by this library on
  * the current device since the previous call of this function gave up on a
  * bounded wait.  *out (HOST pointer, may be NULL) receives CYC_OK or

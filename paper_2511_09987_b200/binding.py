@@ -27,6 +27,7 @@ SYMBOLS = {
     "cyc_recurrence_matmul_batched": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _i64, _ptr, _i64, _ptr, _i64, _ptr, _u32]),
     "cyc_recurrence_matmul_host": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_recurrence_matmul_splitk_static": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
+    "cyc_block_trsm": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_selftest_bounded_wait": (_int, [_ptr, _i64]),
     "cyc_last_device_status": (_int, [_ptr, ctypes.POINTER(ctypes.c_int)]),
     "cyc_kernel_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
@@ -60,6 +61,7 @@ cyc_recurrence_matmul = _lib.cyc_recurrence_matmul
 cyc_recurrence_matmul_batched = _lib.cyc_recurrence_matmul_batched
 cyc_recurrence_matmul_host = _lib.cyc_recurrence_matmul_host
 cyc_recurrence_matmul_splitk_static = _lib.cyc_recurrence_matmul_splitk_static
+cyc_block_trsm = _lib.cyc_block_trsm
 cyc_selftest_bounded_wait = _lib.cyc_selftest_bounded_wait
 cyc_last_device_status = _lib.cyc_last_device_status
 CYC_STATIC_WORKSPACE_BYTES = 8 << 20
@@ -162,6 +164,25 @@ def recurrence_matmul_splitk_static(A, B, C=None, *, b_col_major: bool = False):
     check(cyc_recurrence_matmul_splitk_static(M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(),
                                               _flags(b_col_major, False)))
     return C
+
+
+def block_trsm(L, B, X=None, *, tile: int = 0, fixed_k_order: bool = False):
+    """Solve ``L X = B`` for contiguous fp32 CUDA tensors ``L[n,n]`` (lower triangle read) and ``B[n,m]``.
+
+    ``X`` defaults to a new tensor; pass ``X=B`` to solve in place."""
+    import torch
+    if not (L.is_cuda and B.is_cuda and L.is_contiguous() and B.is_contiguous() and L.dim() == 2 and B.dim() == 2):
+        raise ValueError("L and B must be contiguous CUDA matrices")
+    n, m = B.shape
+    if L.shape[0] != n or L.shape[1] != n or L.dtype != B.dtype:
+        raise ValueError("L must be [n,n] and B [n,m] of one dtype")
+    if X is None:
+        X = torch.empty_like(B)
+    elif not (X.is_cuda and X.is_contiguous() and X.shape == B.shape and X.dtype == B.dtype):
+        raise ValueError("X must be a contiguous CUDA tensor shaped like B")
+    check(cyc_block_trsm(n, m, tile, _torch_dtype_code(L), L.data_ptr(), B.data_ptr(), X.data_ptr(), _stream(),
+                         _flags(False, fixed_k_order)))
+    return X
 
 
 def last_device_status() -> int:

@@ -18,6 +18,7 @@
 #include "umma_pair_tall_kernel.cuh"
 #include "splitk_reduce_kernel.cuh"
 #include "umma_pair_tf32x3_kernel.cuh"
+#include "trsm_diag_kernel.cuh"
 
 namespace cyc {
 
@@ -78,7 +79,9 @@ struct Problem {
     void* C;
     long long sA, sB, sC;
     unsigned flags;
+    long long lda = 0;  // row pitch of A in elements; 0 = dense (K).  Only internal callers set it (sub-blocks of L).
 };
+static long long lda_of(const Problem& q) { return q.lda ? q.lda : q.K; }
 
 // host-side validation; no CUDA call
 static int validate(const Problem& q) {
@@ -108,7 +111,8 @@ static bool tma_ok(const Problem& q) {
     const int eb = elem_bytes(q.dtype);
     const bool colmajor = (q.flags & CYC_FLAG_B_COL_MAJOR) != 0;
     if (reinterpret_cast<uintptr_t>(q.A) % 16 || reinterpret_cast<uintptr_t>(q.B) % 16) return false;
-    if ((q.K * eb) % 16) return false;                  // A pitch (and B pitch when stored [N][K])
+    if ((lda_of(q) * eb) % 16) return false;            // A pitch
+    if (colmajor && (q.K * eb) % 16) return false;      // B pitch when stored [N][K]
     if (!colmajor && (q.N * eb) % 16) return false;     // B pitch when stored [K][N]
     if (q.batch > 1 && ((q.sA * eb) % 16 || (q.sB * eb) % 16)) return false;
     return true;
@@ -161,6 +165,7 @@ static int launch_simt(const Problem& q, cudaStream_t st) {
     p.A = q.A; p.B = q.B; p.C = q.C;
     p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
     p.sA = q.sA; p.sB = q.sB; p.sC = q.sC;
+    p.lda = lda_of(q);
     const bool colmajor = (q.flags & CYC_FLAG_B_COL_MAJOR) != 0;
     p.b_sk = colmajor ? 1 : q.N;
     p.b_sj = colmajor ? q.K : 1;
@@ -179,7 +184,7 @@ static int launch_simt(const Problem& q, cudaStream_t st) {
     }
     bool vec = false;
     if constexpr (sizeof(TIn) == 4) {
-        vec = !colmajor && q.K % 4 == 0 && q.N % 4 == 0 && q.sA % 4 == 0 && q.sB % 4 == 0 && q.sC % 4 == 0 &&
+        vec = !colmajor && q.K % 4 == 0 && lda_of(q) % 4 == 0 && q.N % 4 == 0 && q.sA % 4 == 0 && q.sB % 4 == 0 && q.sC % 4 == 0 &&
               reinterpret_cast<uintptr_t>(q.A) % 16 == 0 && reinterpret_cast<uintptr_t>(q.B) % 16 == 0 &&
               reinterpret_cast<uintptr_t>(q.C) % 16 == 0;
     }
@@ -278,7 +283,7 @@ static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
     constexpr int BK = Sm::BK;
     constexpr int CH = 128 / UmmaTraits<KIND>::ELEM_BYTES;
     CUtensorMap tmA, tmB;
-    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, q.K, q.sA, BK, UMMA_BM);
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, BK, UMMA_BM);
     if (rc) return rc;
     if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
     else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, BN);
@@ -311,7 +316,7 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws 
     constexpr int CH = 128 / UmmaTraits<KIND>::ELEM_BYTES;
     constexpr int SMEM = pair_smem_bytes<STAGES>();
     CUtensorMap tmA, tmB, tmC;
-    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, q.K, q.sA, BK, PAIR_HALF);
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, BK, PAIR_HALF);
     if (rc) return rc;
     if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
     else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, PAIR_HALF);
@@ -413,7 +418,7 @@ static int launch_pair_tall_cfg(const Problem& q, cudaStream_t st, int sms) {
     constexpr int BK = 128 / UmmaTraits<KIND>::ELEM_BYTES;
     constexpr int CH = 128 / UmmaTraits<KIND>::ELEM_BYTES;
     CUtensorMap tmA, tmB, tmC;
-    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, q.K, q.sA, BK, PAIR_HALF);
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, BK, PAIR_HALF);
     if (rc) return rc;
     if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
     else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, PAIR_HALF);
@@ -446,7 +451,7 @@ static int launch_pair_tall_cfg(const Problem& q, cudaStream_t st, int sms) {
 template <bool B_MN>
 static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
     CUtensorMap tmA, tmB, tmC;
-    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, q.K, q.sA, 32, PAIR_HALF);
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, 32, PAIR_HALF);
     if (rc) return rc;
     // fp32 B stored [K][N] feeds the MMA column-contiguous: 32-byte-chunk swizzle (see umma_smem_desc)
     if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
@@ -509,9 +514,8 @@ static int launch_umma(const Problem& q, cudaStream_t st) {
     return wide ? launch_umma_cfg<KIND, false, 256, 4>(q, st, di.sms) : launch_umma_cfg<KIND, false, 128, 6>(q, st, di.sms);
 }
 
-static int dispatch(const Problem& q, cudaStream_t st) {
-    int rc = validate(q);
-    if (rc) return rc;
+// kernel selection and launch for a validated problem (also used for the sub-problems the library builds itself)
+static int route(const Problem& q, cudaStream_t st) {
     switch (choose(q)) {
         case FAM_UMMA:
         case FAM_UMMA_PAIR:
@@ -525,6 +529,56 @@ static int dispatch(const Problem& q, cudaStream_t st) {
             if (q.dtype == CYC_BF16_F32) return launch_simt<__nv_bfloat16, float>(q, st);
             return launch_simt<int8_t, int>(q, st);
     }
+}
+
+static int dispatch(const Problem& q, cudaStream_t st) {
+    int rc = validate(q);
+    if (rc) return rc;
+    return route(q, st);
+}
+
+// ------------------------------------------------------------------ block lower-triangular solve
+// X_i = TRSM(L_ii, B_i - sum_{j<i} GEMM(L_ij, X_j)).  The block rows are split recursively: solve the upper part,
+// form the partial sums of the lower part's rows over the solved block columns with one recurrence-matmul launch
+// (triangular space; written to the plane of this recursion level), solve the lower part.  A diagonal tile subtracts
+// the planes of every level that covered its rows (its end-of-row accumulator) and solves (diagonal space).
+struct TrsmPlan {
+    long long n, m, T;
+    const float* L;
+    const float* B;
+    float* X;
+    float* W;
+    long long plane;
+    unsigned flags;
+    cudaStream_t st;
+};
+
+static int trsm_diag(const TrsmPlan& t, long long b, unsigned mask) {
+    TrsmDiagParams p;
+    p.L = t.L; p.B = t.B; p.X = t.X; p.W = t.W;
+    p.plane = t.plane;
+    p.n = static_cast<int>(t.n); p.m = static_cast<int>(t.m);
+    p.r0 = static_cast<int>(b * t.T);
+    p.rows = static_cast<int>(t.n - b * t.T < t.T ? t.n - b * t.T : t.T);
+    p.mask = mask;
+    const long long blocks = (t.m + TRSM_CW - 1) / TRSM_CW;
+    trsm_diag_kernel<<<static_cast<unsigned>(blocks), TRSM_THREADS, TRSM_SMEM_BYTES, t.st>>>(p);
+    CYC_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
+static int trsm_range(const TrsmPlan& t, long long b0, long long b1, unsigned mask, int level) {
+    if (b1 - b0 == 1) return trsm_diag(t, b0, mask);
+    const long long mid = b0 + (b1 - b0 + 1) / 2;
+    int rc = trsm_range(t, b0, mid, mask, level + 1);
+    if (rc) return rc;
+    const long long r0 = mid * t.T, r1 = b1 * t.T < t.n ? b1 * t.T : t.n, k0 = b0 * t.T, k1 = mid * t.T;
+    Problem q{1, r1 - r0, t.m, k1 - k0, CYC_F32, t.L + r0 * t.n + k0, t.X + k0 * t.m, t.W + level * t.plane + r0 * t.m,
+              (r1 - r0) * t.n, (k1 - k0) * t.m, (r1 - r0) * t.m, t.flags & CYC_FLAG_FIXED_K_ORDER, t.n};
+    rc = route(q, t.st);
+    if (rc) return rc;
+    return trsm_range(t, mid, b1, mask | (1u << level), level + 1);
 }
 
 }  // namespace cyc
@@ -712,6 +766,43 @@ extern "C" int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == CYC_BF16_F32 ? launch_splitk<KIND_BF16>(q, st, di.sms, ws, plan) : launch_splitk<KIND_I8>(q, st, di.sms, ws, plan);
+}
+
+extern "C" int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, const void* L, const void* B, void* X,
+                              void* stream, unsigned flags) {
+    if (n <= 0 || m <= 0 || tile < 0 || tile > TRSM_T_MAX || !L || !B || !X) return CYC_ERR_INVALID_ARG;
+    if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
+    if (flags & ~CYC_FLAG_FIXED_K_ORDER) return CYC_ERR_INVALID_ARG;
+    const uintptr_t l0 = reinterpret_cast<uintptr_t>(L), b0 = reinterpret_cast<uintptr_t>(B), x0 = reinterpret_cast<uintptr_t>(X);
+    if ((l0 | b0 | x0) % 4) return CYC_ERR_INVALID_ARG;
+    if (n > 0x7fffffffll || m > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
+    if (dtype != CYC_F32) return CYC_ERR_UNSUPPORTED;  // the solve is defined for fp32 only
+    const uintptr_t lbytes = static_cast<uintptr_t>(n) * n * 4, xbytes = static_cast<uintptr_t>(n) * m * 4;
+    if (x0 < l0 + lbytes && l0 < x0 + xbytes) return CYC_ERR_INVALID_ARG;                // X over L
+    if (x0 != b0 && x0 < b0 + xbytes && b0 < x0 + xbytes) return CYC_ERR_INVALID_ARG;    // X over B, other than in place
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    TrsmPlan t;
+    t.n = n; t.m = m; t.T = tile ? tile : TRSM_T_MAX;
+    t.L = static_cast<const float*>(L); t.B = static_cast<const float*>(B); t.X = static_cast<float*>(X);
+    t.W = nullptr; t.plane = n * m; t.flags = flags; t.st = st;
+    const long long nb = (n + t.T - 1) / t.T;
+    int levels = 0;
+    while ((1ll << levels) < nb) ++levels;
+    CYC_CUDA(cudaFuncSetAttribute(trsm_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TRSM_SMEM_BYTES));
+    if (levels) {
+        cudaMemPool_t pool;
+        int rc = workspace_pool(&pool);
+        if (rc) return rc;
+        void* ws = nullptr;
+        CYC_CUDA(cudaMallocFromPoolAsync(&ws, static_cast<size_t>(levels) * t.plane * sizeof(float), pool, st));
+        t.W = static_cast<float*>(ws);
+    }
+    int rc = trsm_range(t, 0, nb, 0u, 0);
+    if (t.W) {
+        cudaError_t e = cudaFreeAsync(t.W, st);
+        if (e != cudaSuccess && rc == CYC_OK) rc = cuda_fail(e, "cudaFreeAsync");
+    }
+    return rc;
 }
 
 extern "C" int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles) {

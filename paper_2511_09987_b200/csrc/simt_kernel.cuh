@@ -23,6 +23,7 @@ struct SimtParams {
     void* C;
     int M, N, K;
     long long sA, sB, sC;  // batch strides, elements
+    long long lda;         // row pitch of A, elements (K when A is dense)
     long long b_sk, b_sj;  // element B_kj at B[k*b_sk + j*b_sj]
     int tiles_m, tiles_n;
 };
@@ -71,7 +72,7 @@ __global__ void __launch_bounds__(SIMT_THREADS, 2) simt_recurrence_kernel(const 
             for (int h = 0; h < 2; ++h) {
                 const int r = (tid >> 2) + 64 * h, kq = (tid & 3) * 4;
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (m0 + r < M && k0 + kq < K) v = *reinterpret_cast<const float4*>(A + static_cast<long long>(m0 + r) * K + k0 + kq);
+                if (m0 + r < M && k0 + kq < K) v = *reinterpret_cast<const float4*>(A + static_cast<long long>(m0 + r) * p.lda + k0 + kq);
                 ra[4 * h + 0] = v.x; ra[4 * h + 1] = v.y; ra[4 * h + 2] = v.z; ra[4 * h + 3] = v.w;
             }
             // B: 16 k x 128 j = 512 float4; thread -> k rows (tid>>5) and (tid>>5)+8, j quad (tid&31)
@@ -89,7 +90,7 @@ __global__ void __launch_bounds__(SIMT_THREADS, 2) simt_recurrence_kernel(const 
                 const int idx = tid + e * SIMT_THREADS;
                 const int r = idx >> 4, kk = idx & 15;
                 TAcc v = TAcc(0);
-                if (m0 + r < M && k0 + kk < K) v = simt_widen<TIn, TAcc>(A[static_cast<long long>(m0 + r) * K + k0 + kk]);
+                if (m0 + r < M && k0 + kk < K) v = simt_widen<TIn, TAcc>(A[static_cast<long long>(m0 + r) * p.lda + k0 + kk]);
                 ra[e] = v;
             }
 #pragma unroll
@@ -241,7 +242,7 @@ __global__ void __launch_bounds__(SIMT_THREADS) simt_recurrence_small_kernel(con
             const int idx = tid + e * SIMT_THREADS;
             const int r = idx >> 6, kk = idx & 63;
             ra[e] = TAcc(0);
-            if (m0 + r < M && k0 + kk < K) ra[e] = simt_widen<TIn, TAcc>(A[static_cast<long long>(m0 + r) * K + k0 + kk]);
+            if (m0 + r < M && k0 + kk < K) ra[e] = simt_widen<TIn, TAcc>(A[static_cast<long long>(m0 + r) * p.lda + k0 + kk]);
         }
 #pragma unroll
         for (int e = 0; e < 16; ++e) {

@@ -63,6 +63,27 @@ def test_invalid_arguments_rejected_on_host(binding):
     assert h(1, 4, 4, 4, 9, A, B, C, None, 0) == b.CYC_ERR_INVALID_ARG
 
 
+def test_block_trsm_arguments_rejected_on_host(binding):
+    b = binding
+    L, B, X = 1 << 20, 1 << 30, 1 << 40   # never dereferenced: validation comes first
+    t = b.cyc_block_trsm
+    assert t(0, 4, 0, 0, L, B, X, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert t(4, 0, 0, 0, L, B, X, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert t(4, 4, 257, 0, L, B, X, None, 0) == b.CYC_ERR_INVALID_ARG         # tile edge above 256
+    assert t(4, 4, -1, 0, L, B, X, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert t(4, 4, 0, 5, L, B, X, None, 0) == b.CYC_ERR_INVALID_ARG           # unknown dtype
+    assert t(4, 4, 0, 1, L, B, X, None, 0) == b.CYC_ERR_UNSUPPORTED           # bf16: the solve is fp32 only
+    assert t(4, 4, 0, 2, L, B, X, None, 0) == b.CYC_ERR_UNSUPPORTED
+    assert t(4, 4, 0, 0, L, B, X, None, 2) == b.CYC_ERR_INVALID_ARG           # no column-major flag here
+    assert t(4, 4, 0, 0, None, B, X, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert t(4, 4, 0, 0, L, None, X, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert t(4, 4, 0, 0, L, B, None, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert t(4, 4, 0, 0, L, B + 2, X, None, 0) == b.CYC_ERR_INVALID_ARG       # not 4-byte aligned
+    assert t(4, 4, 0, 0, L, B, L + 32, None, 0) == b.CYC_ERR_INVALID_ARG      # X over L
+    assert t(4, 4, 0, 0, L, B, B + 16, None, 0) == b.CYC_ERR_INVALID_ARG      # X over B, not in place
+    assert t(1 << 31, 4, 0, 0, L, B, X, None, 0) == b.CYC_ERR_UNSUPPORTED
+
+
 def test_kernel_selection(binding):
     k = binding.kernel_for
     assert k(1, 64, 64, 64, "f32", fixed_k_order=True) == "simt"
