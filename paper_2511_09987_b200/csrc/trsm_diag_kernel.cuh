@@ -41,6 +41,10 @@ __device__ __forceinline__ void trsm_cp_async4(float* dst_smem, const float* src
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem))), "l"(src)
                  : "memory");
 }
+__device__ __forceinline__ void trsm_cp_async16(float* dst_smem, const float* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem))), "l"(src)
+                 : "memory");
+}
 __device__ __forceinline__ void trsm_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void trsm_cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
@@ -55,34 +59,60 @@ __global__ void __launch_bounds__(TRSM_THREADS) trsm_diag_kernel(const TrsmDiagP
     const int c = blockIdx.x * TRSM_CW + lane;
     const bool col_ok = c < p.m;
 
-    // panel of sub-block sb: rows [s0, s0+32) of the tile, tile columns [0, s0+32); rows past the tile are zero
+    // panel of sub-block sb: rows [s0, s0+32) of the tile, tile columns [0, s0+32); rows past the tile are zero.
+    // Warp w fetches rows w, w+8, w+16, w+24; 16-byte copies when every row of L starts on a 16-byte boundary.
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(p.L) % 16 == 0) && (p.n % 4 == 0) && (p.r0 % 4 == 0);
     auto issue_panel = [&](int s0, int buf) {
         float* Lp = Lp_base + buf * TRSM_SB * TRSM_LP_PITCH;
         const int width = s0 + TRSM_SB;
-        for (int idx = tid; idx < TRSM_SB * width; idx += TRSM_THREADS) {
-            const int r = idx / width, k = idx - r * width;
-            float* dst = Lp + r * TRSM_LP_PITCH + k;
-            if (s0 + r < p.rows && k < p.rows)
-                trsm_cp_async4(dst, p.L + static_cast<long long>(p.r0 + s0 + r) * p.n + p.r0 + k);
-            else
-                *dst = 0.f;
+#pragma unroll
+        for (int i = 0; i < TRSM_SB / 8; ++i) {
+            const int r = warp + 8 * i;
+            float* dst = Lp + r * TRSM_LP_PITCH;
+            const float* src = p.L + static_cast<long long>(p.r0 + s0 + r) * p.n + p.r0;
+            const bool row_ok = s0 + r < p.rows;
+            for (int k = 4 * lane; k < width; k += 128) {
+                if (row_ok && vec_ok && k + 4 <= p.rows) {
+                    trsm_cp_async16(dst + k, src + k);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if (row_ok && k + q < p.rows) trsm_cp_async4(dst + k + q, src + k + q);
+                        else dst[k + q] = 0.f;
+                    }
+                }
+            }
         }
         trsm_cp_async_commit();
     };
     issue_panel(0, 0);
 
-    // right-hand side of the tile: B_ii - Xa, Xa = the partial-sum planes in increasing level
-    for (int r = warp; r < TRSM_T_MAX; r += TRSM_THREADS / 32) {
-        float v = 0.f;
-        if (r < p.rows && col_ok) {
-            const long long at = static_cast<long long>(p.r0 + r) * p.m + c;
-            float xa = 0.f;
-            unsigned mk = p.mask;
-            for (int l = 0; mk; ++l, mk >>= 1)
-                if (mk & 1u) xa += p.W[l * p.plane + at];
-            v = p.B[at] - xa;
+    // right-hand side of the tile: B_ii - Xa, Xa = the partial-sum planes in increasing level.  Eight rows per warp
+    // at a time, all their loads in flight together.
+    for (int rb = 0; rb < TRSM_T_MAX; rb += 64) {
+        float v[8], xa[8];
+        long long at[8];
+        bool ok[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = rb + 8 * i + warp;
+            ok[i] = r < p.rows && col_ok;
+            at[i] = static_cast<long long>(p.r0 + r) * p.m + c;
+            v[i] = ok[i] ? __ldg(p.B + at[i]) : 0.f;
+            xa[i] = 0.f;
         }
-        Xs[r][lane] = v;
+        unsigned mk = p.mask;
+        for (int l = 0; mk; ++l, mk >>= 1) {
+            if (!(mk & 1u)) continue;
+            const float* Wl = p.W + l * p.plane;
+            float w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w[i] = ok[i] ? __ldg(Wl + at[i]) : 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) xa[i] += w[i];
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) Xs[rb + 8 * i + warp][lane] = v[i] - xa[i];
     }
 
     for (int s0 = 0, sb = 0; s0 < p.rows; s0 += TRSM_SB, ++sb) {
@@ -101,7 +131,7 @@ __global__ void __launch_bounds__(TRSM_THREADS) trsm_diag_kernel(const TrsmDiagP
 
         // update: rows s0 + 4*warp .. +3  -=  L[row][0..s0) . X[0..s0)
         if (s0 > 0) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            float acc[4][2] = {};  // two partial sums per row (even and odd pairs of k): eight independent chains
             const float* lrow = Lp + (4 * warp) * TRSM_LP_PITCH;
 #pragma unroll 2
             for (int k = 0; k < s0; k += 4) {
@@ -109,14 +139,14 @@ __global__ void __launch_bounds__(TRSM_THREADS) trsm_diag_kernel(const TrsmDiagP
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const float4 l = *reinterpret_cast<const float4*>(lrow + i * TRSM_LP_PITCH + k);
-                    acc[i] = fmaf(l.x, x0, acc[i]);
-                    acc[i] = fmaf(l.y, x1, acc[i]);
-                    acc[i] = fmaf(l.z, x2, acc[i]);
-                    acc[i] = fmaf(l.w, x3, acc[i]);
+                    acc[i][0] = fmaf(l.x, x0, acc[i][0]);
+                    acc[i][1] = fmaf(l.y, x1, acc[i][1]);
+                    acc[i][0] = fmaf(l.z, x2, acc[i][0]);
+                    acc[i][1] = fmaf(l.w, x3, acc[i][1]);
                 }
             }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) Xs[s0 + 4 * warp + i][lane] -= acc[i];
+            for (int i = 0; i < 4; ++i) Xs[s0 + 4 * warp + i][lane] -= acc[i][0] + acc[i][1];
         }
         __syncthreads();  // updated right-hand side, Lt and dinv visible to warp 0
 
@@ -124,17 +154,27 @@ __global__ void __launch_bounds__(TRSM_THREADS) trsm_diag_kernel(const TrsmDiagP
             float s[TRSM_SB];
 #pragma unroll
             for (int r = 0; r < TRSM_SB; ++r) s[r] = Xs[s0 + r][lane];
+            const float my_dinv = dinv[lane];
+            float4 lnext[TRSM_SB / 4];  // column k+1 of the triangle (row k+1 of Lt), fetched while column k is applied
+#pragma unroll
+            for (int g = 0; g < TRSM_SB / 4; ++g) lnext[g] = *reinterpret_cast<const float4*>(&Lt[0][4 * g]);
 #pragma unroll
             for (int k = 0; k < TRSM_SB; ++k) {
-                const float xk = s[k] * dinv[k];
+                float4 l[TRSM_SB / 4];
+#pragma unroll
+                for (int g = 0; g < TRSM_SB / 4; ++g) l[g] = lnext[g];
+                if (k + 1 < TRSM_SB) {
+#pragma unroll
+                    for (int g = (k + 2) / 4; g < TRSM_SB / 4; ++g) lnext[g] = *reinterpret_cast<const float4*>(&Lt[k + 1][4 * g]);
+                }
+                const float xk = s[k] * __shfl_sync(0xffffffffu, my_dinv, k);
                 s[k] = xk;
 #pragma unroll
-                for (int g = (k + 1) / 4; g < TRSM_SB / 4; ++g) {
-                    const float4 l = *reinterpret_cast<const float4*>(&Lt[k][4 * g]);  // zero where r <= k
-                    if (4 * g + 0 > k) s[4 * g + 0] = fmaf(-l.x, xk, s[4 * g + 0]);
-                    if (4 * g + 1 > k) s[4 * g + 1] = fmaf(-l.y, xk, s[4 * g + 1]);
-                    if (4 * g + 2 > k) s[4 * g + 2] = fmaf(-l.z, xk, s[4 * g + 2]);
-                    if (4 * g + 3 > k) s[4 * g + 3] = fmaf(-l.w, xk, s[4 * g + 3]);
+                for (int g = (k + 1) / 4; g < TRSM_SB / 4; ++g) {  // entries with r <= k are zero in Lt and skipped here
+                    if (4 * g + 0 > k) s[4 * g + 0] = fmaf(-l[g].x, xk, s[4 * g + 0]);
+                    if (4 * g + 1 > k) s[4 * g + 1] = fmaf(-l[g].y, xk, s[4 * g + 1]);
+                    if (4 * g + 2 > k) s[4 * g + 2] = fmaf(-l[g].z, xk, s[4 * g + 2]);
+                    if (4 * g + 3 > k) s[4 * g + 3] = fmaf(-l[g].w, xk, s[4 * g + 3]);
                 }
             }
 #pragma unroll
