@@ -168,7 +168,8 @@ int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t K, int dty
  * cyc_recurrence_matmul (operand A = a sub-block of L, row pitch n); their partial sums
  * pass through a workspace of ceil(log2(ceil(n/T))) * n * m * 4 bytes taken from the
  * library's stream-ordered pool for the duration of the call.  The diagonal tiles are
- * solved by forward substitution in fp32 (x_k = s_k * (1 / L_kk)).  Caller owns L, B, X;
+ * solved by forward substitution in fp32 (rows scaled by the correctly rounded reciprocal
+ * of their diagonal entry).  Caller owns L, B, X;
  * the library keeps no reference after the kernels complete.  Errors as for
  * cyc_recurrence_matmul.
  */

@@ -9,11 +9,15 @@
 //
 // One CTA solves one diagonal tile (rows <= 256) for 32 right-hand-side columns; lane = column, so every shared-memory
 // access of the right-hand side is conflict-free and every global access of B, W, X is a 128-byte row segment.
-// The tile is processed in sub-blocks of 32 rows:
-//   update   rows of the sub-block  -=  L[sub-block rows][earlier rows of the tile] * X[earlier rows]   (8 warps x 4 rows)
-//   solve    the 32 x 32 triangle by a column sweep in registers (warp 0): x_k = s_k / L_kk, s_r -= L_rk x_k for r > k
-// The L panel of the next sub-block is fetched with cp.async while the current one is processed.  Entries of L above
-// the diagonal are never used.  x_k is formed as s_k * (1 / L_kk) with a correctly rounded reciprocal.
+// The lower triangle of the tile is brought into shared memory once, as 32 x 32 blocks (cp.async; 144 KB for a full
+// tile).  The tile is then processed in sub-blocks of 32 rows, with one step of look-ahead so that the sequential part
+// overlaps the bulk of the arithmetic:
+//   solve(s)     warp 0: the 32 x 32 triangle of sub-block s by a column sweep in registers, rows pre-scaled by the
+//                reciprocal of their diagonal entry: x_r = s_r / L_rr - sum_{k<r} (L_rk / L_rr) x_k
+//   trailing(s)  twelve other warps, at the same time: rows below sub-block s  -=  L[rows][sub-block s-1] * x_(s-1)
+//                (a warp takes 16 rows x 32 columns, a 4 x 4 patch per lane)
+//   next(s+1)    two warps: rows of sub-block s+1  -=  L[rows][sub-block s] * x_s; eight warps prepare its triangle
+// Every row receives its updates in increasing column order.  Entries of L above the diagonal are never used.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -31,11 +35,13 @@ struct TrsmDiagParams {
     unsigned mask;    // bit l set: plane l holds a partial sum for these rows
 };
 
-constexpr int TRSM_T_MAX = 256, TRSM_CW = 32, TRSM_SB = 32, TRSM_THREADS = 256;
-constexpr int TRSM_LP_PITCH = TRSM_T_MAX + 4;  // floats; rows stay 16-byte aligned, row starts fall in different banks
+constexpr int TRSM_T_MAX = 256, TRSM_CW = 32, TRSM_SB = 32, TRSM_THREADS = 512, TRSM_WARPS = TRSM_THREADS / 32;
+constexpr int TRSM_NSB = TRSM_T_MAX / TRSM_SB;            // sub-blocks per tile
+constexpr int TRSM_BLK = TRSM_SB * TRSM_SB;               // floats per 32 x 32 block of L
+constexpr int TRSM_NBLK = TRSM_NSB * (TRSM_NSB + 1) / 2;  // blocks on and below the diagonal
 constexpr int TRSM_LT_PITCH = TRSM_SB + 4;
 constexpr int TRSM_SMEM_BYTES =
-    (TRSM_T_MAX * TRSM_CW + 2 * TRSM_SB * TRSM_LP_PITCH + TRSM_SB * TRSM_LT_PITCH + TRSM_SB) * static_cast<int>(sizeof(float));
+    (TRSM_T_MAX * TRSM_CW + TRSM_NBLK * TRSM_BLK + TRSM_SB * TRSM_LT_PITCH + TRSM_SB) * static_cast<int>(sizeof(float));
 
 __device__ __forceinline__ void trsm_cp_async4(float* dst_smem, const float* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem))), "l"(src)
@@ -46,56 +52,106 @@ __device__ __forceinline__ void trsm_cp_async16(float* dst_smem, const float* sr
                  : "memory");
 }
 __device__ __forceinline__ void trsm_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void trsm_cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void trsm_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-__global__ void __launch_bounds__(TRSM_THREADS) trsm_diag_kernel(const TrsmDiagParams p) {
+// block (bi, bj), bj <= bi, of the tile's lower triangle; element (r, k) of a block at [r * 32 + k]
+__device__ __forceinline__ int trsm_block(int bi, int bj) { return (bi * (bi + 1) / 2 + bj) * TRSM_BLK; }
+
+// One warp:  xdst[0..4R)[0..32)  -=  Lrows[0..4R)[0..32) . xsrc[0..32)[0..32)
+// (Lrows: 4R consecutive rows of one 32 x 32 block; xsrc: the 32 solved rows; xdst: the 4R rows to update).
+// Each lane owns an R x 4 patch (rows R*(lane/8).., columns 4*(lane%8)..): the eight lanes that share a row group read
+// the same address of L (broadcast), the eight column groups read one contiguous 128-byte row of x.
+template <int R>
+__device__ __forceinline__ void trsm_apply(const float* __restrict__ lrows, float (*xsrc)[TRSM_CW], float (*xdst)[TRSM_CW], int lane) {
+    const int tr = lane >> 3, tc = lane & 7;
+    float acc[R][4] = {};
+#pragma unroll 2
+    for (int k = 0; k < TRSM_SB; k += 4) {
+        float4 xv[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) xv[j] = *reinterpret_cast<const float4*>(&xsrc[k + j][4 * tc]);
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const float4 l = *reinterpret_cast<const float4*>(lrows + (R * tr + i) * TRSM_SB + k);
+            acc[i][0] = fmaf(l.x, xv[0].x, acc[i][0]); acc[i][1] = fmaf(l.x, xv[0].y, acc[i][1]);
+            acc[i][2] = fmaf(l.x, xv[0].z, acc[i][2]); acc[i][3] = fmaf(l.x, xv[0].w, acc[i][3]);
+            acc[i][0] = fmaf(l.y, xv[1].x, acc[i][0]); acc[i][1] = fmaf(l.y, xv[1].y, acc[i][1]);
+            acc[i][2] = fmaf(l.y, xv[1].z, acc[i][2]); acc[i][3] = fmaf(l.y, xv[1].w, acc[i][3]);
+            acc[i][0] = fmaf(l.z, xv[2].x, acc[i][0]); acc[i][1] = fmaf(l.z, xv[2].y, acc[i][1]);
+            acc[i][2] = fmaf(l.z, xv[2].z, acc[i][2]); acc[i][3] = fmaf(l.z, xv[2].w, acc[i][3]);
+            acc[i][0] = fmaf(l.w, xv[3].x, acc[i][0]); acc[i][1] = fmaf(l.w, xv[3].y, acc[i][1]);
+            acc[i][2] = fmaf(l.w, xv[3].z, acc[i][2]); acc[i][3] = fmaf(l.w, xv[3].w, acc[i][3]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        float4* dst = reinterpret_cast<float4*>(&xdst[R * tr + i][4 * tc]);
+        float4 cur = *dst;
+        cur.x -= acc[i][0]; cur.y -= acc[i][1]; cur.z -= acc[i][2]; cur.w -= acc[i][3];
+        *dst = cur;
+    }
+}
+
+// wait until at most `pending` of this thread's cp.async groups are still in flight (pending = 0 .. TRSM_NSB - 1)
+__device__ __forceinline__ void trsm_wait_pending(int pending) {
+    switch (pending) {
+        case 0: trsm_cp_async_wait<0>(); break;
+        case 1: trsm_cp_async_wait<1>(); break;
+        case 2: trsm_cp_async_wait<2>(); break;
+        case 3: trsm_cp_async_wait<3>(); break;
+        case 4: trsm_cp_async_wait<4>(); break;
+        case 5: trsm_cp_async_wait<5>(); break;
+        case 6: trsm_cp_async_wait<6>(); break;
+        default: trsm_cp_async_wait<7>(); break;
+    }
+}
+
+__global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDiagParams p) {
     extern __shared__ __align__(16) float trsm_smem[];
-    float(*Xs)[TRSM_CW] = reinterpret_cast<float(*)[TRSM_CW]>(trsm_smem);                     // right-hand side, then X
-    float* Lp_base = trsm_smem + TRSM_T_MAX * TRSM_CW;                                        // two panels
-    float(*Lt)[TRSM_LT_PITCH] = reinterpret_cast<float(*)[TRSM_LT_PITCH]>(Lp_base + 2 * TRSM_SB * TRSM_LP_PITCH);
+    float(*Xs)[TRSM_CW] = reinterpret_cast<float(*)[TRSM_CW]>(trsm_smem);  // right-hand side, then X
+    float* Lb = trsm_smem + TRSM_T_MAX * TRSM_CW;                          // the blocks of L
+    float(*Lt)[TRSM_LT_PITCH] = reinterpret_cast<float(*)[TRSM_LT_PITCH]>(Lb + TRSM_NBLK * TRSM_BLK);
     float* dinv = reinterpret_cast<float*>(Lt) + TRSM_SB * TRSM_LT_PITCH;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c = blockIdx.x * TRSM_CW + lane;
     const bool col_ok = c < p.m;
+    const int nsb = (p.rows + TRSM_SB - 1) / TRSM_SB;
 
-    // panel of sub-block sb: rows [s0, s0+32) of the tile, tile columns [0, s0+32); rows past the tile are zero.
-    // Warp w fetches rows w, w+8, w+16, w+24; 16-byte copies when every row of L starts on a 16-byte boundary.
+    // Column block j of the triangle (tile rows [32 j, 32 nsb), tile columns [32 j, 32 j + 32)) is one cp.async group:
+    // step s of the loop below needs the column blocks up to s only, so the later ones arrive behind the arithmetic.
+    // Rows and columns past the tile are zero.  16-byte copies when every row of L starts on a 16-byte boundary.
     const bool vec_ok = (reinterpret_cast<uintptr_t>(p.L) % 16 == 0) && (p.n % 4 == 0) && (p.r0 % 4 == 0);
-    auto issue_panel = [&](int s0, int buf) {
-        float* Lp = Lp_base + buf * TRSM_SB * TRSM_LP_PITCH;
-        const int width = s0 + TRSM_SB;
+    for (int j = 0; j < nsb; ++j) {
+        const int chunks = (nsb - j) * TRSM_SB * (TRSM_SB / 4);
+        for (int idx = tid; idx < chunks; idx += TRSM_THREADS) {
+            const int t = j * TRSM_SB + (idx >> 3), k = j * TRSM_SB + 4 * (idx & 7);
+            float* dst = Lb + trsm_block(t >> 5, j) + (t & 31) * TRSM_SB + 4 * (idx & 7);
+            const float* src = p.L + static_cast<long long>(p.r0 + t) * p.n + p.r0 + k;
+            const bool row_ok = t < p.rows;
+            if (row_ok && vec_ok && k + 4 <= p.rows) {
+                trsm_cp_async16(dst, src);
+            } else {
 #pragma unroll
-        for (int i = 0; i < TRSM_SB / 8; ++i) {
-            const int r = warp + 8 * i;
-            float* dst = Lp + r * TRSM_LP_PITCH;
-            const float* src = p.L + static_cast<long long>(p.r0 + s0 + r) * p.n + p.r0;
-            const bool row_ok = s0 + r < p.rows;
-            for (int k = 4 * lane; k < width; k += 128) {
-                if (row_ok && vec_ok && k + 4 <= p.rows) {
-                    trsm_cp_async16(dst + k, src + k);
-                } else {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        if (row_ok && k + q < p.rows) trsm_cp_async4(dst + k + q, src + k + q);
-                        else dst[k + q] = 0.f;
-                    }
+                for (int q = 0; q < 4; ++q) {
+                    if (row_ok && k + q < p.rows) trsm_cp_async4(dst + q, src + q);
+                    else dst[q] = 0.f;
                 }
             }
         }
         trsm_cp_async_commit();
-    };
-    issue_panel(0, 0);
+    }
 
     // right-hand side of the tile: B_ii - Xa, Xa = the partial-sum planes in increasing level.  Eight rows per warp
     // at a time, all their loads in flight together.
-    for (int rb = 0; rb < TRSM_T_MAX; rb += 64) {
+    for (int rb = 0; rb < TRSM_T_MAX; rb += 8 * TRSM_WARPS) {
         float v[8], xa[8];
         long long at[8];
         bool ok[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int r = rb + 8 * i + warp;
+            const int r = rb + TRSM_WARPS * i + warp;
             ok[i] = r < p.rows && col_ok;
             at[i] = static_cast<long long>(p.r0 + r) * p.m + c;
             v[i] = ok[i] ? __ldg(p.B + at[i]) : 0.f;
@@ -112,49 +168,44 @@ __global__ void __launch_bounds__(TRSM_THREADS) trsm_diag_kernel(const TrsmDiagP
             for (int i = 0; i < 8; ++i) xa[i] += w[i];
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) Xs[rb + 8 * i + warp][lane] = v[i] - xa[i];
+        for (int i = 0; i < 8; ++i) Xs[rb + TRSM_WARPS * i + warp][lane] = v[i] - xa[i];
     }
 
-    for (int s0 = 0, sb = 0; s0 < p.rows; s0 += TRSM_SB, ++sb) {
-        const int buf = sb & 1;
-        float* Lp = Lp_base + buf * TRSM_SB * TRSM_LP_PITCH;
-        trsm_cp_async_wait_all();
-        __syncthreads();  // panel sb complete; rows < s0 of Xs final; the other panel buffer and Lt free again
-        if (s0 + TRSM_SB < p.rows) issue_panel(s0 + TRSM_SB, buf ^ 1);
-
-        // diagonal 32 x 32 block transposed (strictly lower part only) and the reciprocals of its diagonal
-        for (int idx = tid; idx < TRSM_SB * TRSM_SB; idx += TRSM_THREADS) {
-            const int r = idx >> 5, k = idx & 31;
-            Lt[k][r] = (r > k) ? Lp[r * TRSM_LP_PITCH + s0 + k] : 0.f;
-        }
-        if (tid < TRSM_SB) dinv[tid] = (s0 + tid < p.rows) ? 1.0f / Lp[tid * TRSM_LP_PITCH + s0 + tid] : 1.0f;
-
-        // update: rows s0 + 4*warp .. +3  -=  L[row][0..s0) . X[0..s0)
-        if (s0 > 0) {
-            float acc[4][2] = {};  // two partial sums per row (even and odd pairs of k): eight independent chains
-            const float* lrow = Lp + (4 * warp) * TRSM_LP_PITCH;
-#pragma unroll 2
-            for (int k = 0; k < s0; k += 4) {
-                const float x0 = Xs[k][lane], x1 = Xs[k + 1][lane], x2 = Xs[k + 2][lane], x3 = Xs[k + 3][lane];
+    // Diagonal block s prepared for the column sweep: every row r scaled by 1 / L_rr (so that the sweep needs no
+    // multiplication by the reciprocal inside its dependent chain), strictly lower part, transposed; dinv = 1 / L_rr.
+    // Done by the upper half of the warps.
+    auto build_lt = [&](int s) {
+        if (warp < TRSM_WARPS / 2) return;
+        const float* d = Lb + trsm_block(s, s);
+        const int k = lane;
+        float diag[4], low[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float4 l = *reinterpret_cast<const float4*>(lrow + i * TRSM_LP_PITCH + k);
-                    acc[i][0] = fmaf(l.x, x0, acc[i][0]);
-                    acc[i][1] = fmaf(l.y, x1, acc[i][1]);
-                    acc[i][0] = fmaf(l.z, x2, acc[i][0]);
-                    acc[i][1] = fmaf(l.w, x3, acc[i][1]);
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) Xs[s0 + 4 * warp + i][lane] -= acc[i][0] + acc[i][1];
+        for (int i = 0; i < 4; ++i) {  // rows (warp - 8) + 8 i: one row per warp and pass, lane = column
+            const int r = warp - TRSM_WARPS / 2 + (TRSM_WARPS / 2) * i;
+            diag[i] = d[r * TRSM_SB + r];
+            low[i] = d[r * TRSM_SB + k];
         }
-        __syncthreads();  // updated right-hand side, Lt and dinv visible to warp 0
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = warp - TRSM_WARPS / 2 + (TRSM_WARPS / 2) * i;
+            const float rinv = (s * TRSM_SB + r < p.rows) ? 1.0f / diag[i] : 1.0f;
+            Lt[k][r] = (r > k) ? low[i] * rinv : 0.f;
+            if (k == 0) dinv[r] = rinv;
+        }
+    };
 
+    trsm_wait_pending(nsb - 1);  // column block 0 (this thread's copies; the barrier below covers the other threads')
+    __syncthreads();
+    build_lt(0);
+    __syncthreads();
+
+    for (int s = 0; s < nsb; ++s) {
+        const int s0 = s * TRSM_SB;
         if (warp == 0) {
-            float s[TRSM_SB];
+            // ---- solve(s): x_r = (s_r - sum_{k<r} L_rk x_k) / L_rr evaluated as s_r/L_rr - sum_k (L_rk/L_rr) x_k
+            float sv[TRSM_SB];
 #pragma unroll
-            for (int r = 0; r < TRSM_SB; ++r) s[r] = Xs[s0 + r][lane];
-            const float my_dinv = dinv[lane];
+            for (int r = 0; r < TRSM_SB; ++r) sv[r] = Xs[s0 + r][lane] * dinv[r];
             float4 lnext[TRSM_SB / 4];  // column k+1 of the triangle (row k+1 of Lt), fetched while column k is applied
 #pragma unroll
             for (int g = 0; g < TRSM_SB / 4; ++g) lnext[g] = *reinterpret_cast<const float4*>(&Lt[0][4 * g]);
@@ -167,21 +218,39 @@ __global__ void __launch_bounds__(TRSM_THREADS) trsm_diag_kernel(const TrsmDiagP
 #pragma unroll
                     for (int g = (k + 2) / 4; g < TRSM_SB / 4; ++g) lnext[g] = *reinterpret_cast<const float4*>(&Lt[k + 1][4 * g]);
                 }
-                const float xk = s[k] * __shfl_sync(0xffffffffu, my_dinv, k);
-                s[k] = xk;
+                const float xk = sv[k];
 #pragma unroll
                 for (int g = (k + 1) / 4; g < TRSM_SB / 4; ++g) {  // entries with r <= k are zero in Lt and skipped here
-                    if (4 * g + 0 > k) s[4 * g + 0] = fmaf(-l[g].x, xk, s[4 * g + 0]);
-                    if (4 * g + 1 > k) s[4 * g + 1] = fmaf(-l[g].y, xk, s[4 * g + 1]);
-                    if (4 * g + 2 > k) s[4 * g + 2] = fmaf(-l[g].z, xk, s[4 * g + 2]);
-                    if (4 * g + 3 > k) s[4 * g + 3] = fmaf(-l[g].w, xk, s[4 * g + 3]);
+                    if (4 * g + 0 > k) sv[4 * g + 0] = fmaf(-l[g].x, xk, sv[4 * g + 0]);
+                    if (4 * g + 1 > k) sv[4 * g + 1] = fmaf(-l[g].y, xk, sv[4 * g + 1]);
+                    if (4 * g + 2 > k) sv[4 * g + 2] = fmaf(-l[g].z, xk, sv[4 * g + 2]);
+                    if (4 * g + 3 > k) sv[4 * g + 3] = fmaf(-l[g].w, xk, sv[4 * g + 3]);
                 }
             }
 #pragma unroll
             for (int r = 0; r < TRSM_SB; ++r) {
-                Xs[s0 + r][lane] = s[r];
-                if (s0 + r < p.rows && col_ok) p.X[static_cast<long long>(p.r0 + s0 + r) * p.m + c] = s[r];
+                Xs[s0 + r][lane] = sv[r];
+                if (s0 + r < p.rows && col_ok) p.X[static_cast<long long>(p.r0 + s0 + r) * p.m + c] = sv[r];
             }
+        } else if ((warp & 3) != 0 && s >= 1 && s + 1 < nsb) {
+            // ---- trailing(s): rows below sub-block s, sixteen per warp at a time, with x of sub-block s-1.  Twelve
+            // warps: those that share warp 0's scheduler stay out of its way.
+            const int tasks = (nsb - s - 1) * (TRSM_SB / 16);
+            for (int g = warp - 1 - (warp >> 2); g < tasks; g += 12) {
+                const int t = s0 + TRSM_SB + 16 * g;  // first tile row of the task
+                trsm_apply<4>(Lb + trsm_block(t >> 5, s - 1) + (t & 31) * TRSM_SB, &Xs[s0 - TRSM_SB], &Xs[t], lane);
+            }
+        }
+        if (s + 1 < nsb) trsm_wait_pending(nsb - 2 - s);  // column block s+1
+        __syncthreads();  // x of sub-block s final; rows below it carry every update up to x of s-1
+        if (s + 1 < nsb) {
+            // ---- next(s+1): the 32 rows of the next sub-block with x of sub-block s (warps 1 and 2, sixteen rows each:
+            // every warp that takes part reads all of x, so few warps with large patches cost the least shared-memory
+            // bandwidth); its triangle is prepared by warps 8-15 meanwhile
+            if (warp == 1 || warp == 2)
+                trsm_apply<4>(Lb + trsm_block(s + 1, s) + (16 * (warp - 1)) * TRSM_SB, &Xs[s0], &Xs[s0 + TRSM_SB + 16 * (warp - 1)], lane);
+            build_lt(s + 1);
+            __syncthreads();
         }
     }
 }
