@@ -3,6 +3,9 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
 
+Workloads c1..c5 are the matrix-multiply recurrence (the default, c2, is the headline); t1 and t2 are the block
+lower-triangular solve built on it.
+
 One step = one evaluation of the whole recurrence (weight load, B injection, the
 multiply-accumulate chain along k, export of C) for one workload.  Prints ONE JSON
 line.  `value` is throughput with operands resident in HBM; `e2e` is the same metric
@@ -360,6 +363,148 @@ def run_ours(args, w):
     reps.close()
 
 
+def run_trsm(args, w):
+    """Block lower-triangular solve L X = B (workloads t1, t2): one step = one whole solve (every tile product of the
+    triangular space and every diagonal solve)."""
+    import torch
+    from paper_2511_09987_b200 import binding
+    from paper_2511_09987_b200.replicas import Replicas
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    reps = Replicas("nccl", torch.device("cuda", local))
+    world, rank = reps.world, reps.rank
+    peaks, peak_kind = load_peaks()
+    L, B = inputs.make_trsm_operands(w)
+    hL, hB = torch.from_numpy(L).pin_memory(), torch.from_numpy(B).pin_memory()
+    hX = torch.empty_like(hB).pin_memory()
+    dL, dB = hL.cuda(), hB.cuda()
+    dX = torch.empty_like(dB)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        reps.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        binding.block_trsm(dL, dB, dX, tile=w.tile)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = binding.cyc_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        binding.block_trsm(dL, dB, dX, tile=w.tile)
+    e1.record(stream)
+    barrier()
+    launches = binding.cyc_launch_count() - launches0
+    if binding.last_device_status() != binding.CYC_OK:
+        raise SystemExit("a device-side wait timed out during the benchmark: " + binding.cyc_last_cuda_error().decode())
+    clocks = sampler.stop()
+    ms_per_step = reps.max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+
+    # end to end: pinned host L and B up, solve, X down, every step
+    e2e_steps = 0 if args.kernel_only else max(3, min(args.steps, 10))
+
+    def e2e_step():
+        dL.copy_(hL, non_blocking=True)
+        dB.copy_(hB, non_blocking=True)
+        binding.block_trsm(dL, dB, dX, tile=w.tile)
+        hX.copy_(dX, non_blocking=True)
+
+    for _ in range(0 if args.kernel_only else 2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(1, e2e_steps)
+    e2e_value = None if args.kernel_only else world * w.flops / (reps.max_over_ranks(e2e_ms) * 1e-3) / 1e12
+    if rank != 0:
+        reps.close()
+        return
+    step_s = ms_per_step * 1e-3
+    base = float(peaks["bf16_tflops"]) if args.steps * step_s < 1.0 else float(peaks["bf16_tflops_sustained"])
+    which = "burst" if args.steps * step_s < 1.0 else "sustained"
+    peak = base * NOMINAL_RATIO["tf32"]
+    roofline = {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s", "frac": value / world / peak,
+                "traffic": None,
+                "peak_source": "%s bf16 cuBLAS %s x nominal tf32/bf16 ratio %.1f; the whole step is rated (n(n+1)m flop, the three "
+                               "TF32 products of each fp32 product counted once): %d launches per solve"
+                               % (peak_kind, which, NOMINAL_RATIO["tf32"], launches // max(1, args.steps)),
+                "kernel": "tcgen05_3xtf32 (tile products) + trsm_diag (diagonal tiles)", "kernel_us": step_s * 1e6}
+    if args.kernel_only:
+        cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
+    else:
+        cpu_v, cores, sample = cpu_trsm_rate(w, L, B)
+    line = {
+        "metric": "block_trsm_throughput", "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": describe_trsm(w), "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "L, B, X and the partial-sum planes (%.0f MB) exceed the 126 MB L2" % (
+                       (w.n * w.n + 2 * w.n * w.m) * 4 / 1e6) if (w.n * w.n + 2 * w.n * w.m) * 4 > 2 * L2_BYTES
+                   else "working set below L2: latency-bound, no DRAM figure claimed",
+                   "launch": "one library call per step"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "TFLOPS", "h2d_bytes_per_step": int((hL.numel() + hB.numel()) * 4),
+                "d2h_bytes_per_step": int(hX.numel() * 4), "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_v, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": sample},
+    }
+    print(json.dumps(line))
+    reps.close()
+
+
+def describe_trsm(w):
+    return "%s: block lower-triangular solve f32 n=%d m=%d tile=%d seed=%d coupling=%s" % (w.name, w.n, w.m, w.tile, w.seed, w.coupling)
+
+
+def cpu_trsm_rate(w, L, B, target_seconds=12.0, threads=None):
+    """Time the triangular-solve oracle (collapsed form, as it stands) on a prefix of the right-hand-side columns."""
+    from oracle import trsm as otrsm
+    threads = threads or os.cpu_count() or 1
+    cols = min(w.m, threads)
+    while True:
+        t0 = time.perf_counter()
+        otrsm.block_trsm(L, np.ascontiguousarray(B[:, :cols]), w.tile, threads=threads)
+        dt = time.perf_counter() - t0
+        if dt >= 0.5 * target_seconds or cols >= w.m:
+            break
+        cols = int(min(w.m, cols * min(8.0, max(2.0, 0.9 * target_seconds / max(dt, 1e-3)))))
+    rate = w.n * (w.n + 1) * cols / dt / 1e12
+    return rate, threads, "columns 0..%d of %s (n=%d), collapsed form, %d threads, %.1f s" % (cols - 1, w.name, w.n, threads, dt)
+
+
+def run_trsm_reference(args, w):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    L, B = inputs.make_trsm_operands(w)
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, sample, threads = [], "", os.cpu_count() or 1
+    for s in range(args.warmup + args.steps):
+        v, threads, sample = cpu_trsm_rate(w, L, B, target_seconds=per_step)
+        if s >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    print(json.dumps({
+        "impl": "reference", "metric": "block_trsm_throughput", "value": value, "unit": "TFLOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": w.flops / (value * 1e12) * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": describe_trsm(w), "note": "ms_per_step extrapolated from the sampled rate"},
+        "cpu_baseline": {"value": value, "unit": "TFLOPS", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
+
+
 # CUDA sources each kernel family is built from (host-side launch code is not part of a kernel's identity)
 KERNEL_SOURCES = {
     "simt": ["simt_kernel.cuh"],
@@ -405,14 +550,24 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--shape", default=None, help="M,N,K[,batch]: a smaller case of the workload's recipe (for profiling)")
+    ap.add_argument("--shape", default=None, help="M,N,K[,batch] (c1..c5) or n,m[,tile] (t1, t2): a smaller case of the workload's recipe (for profiling)")
     ap.add_argument("--strict", action="store_true", help="set the fixed-k-order flag (fp32: the per-element FMA chain kernel)")
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="replay the timed steps from a CUDA graph (auto: only for launch-bound workloads)")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs (for profiling)")
     args = ap.parse_args()
+    if args.workload in inputs.TRSM_WORKLOADS:
+        w = inputs.TRSM_WORKLOADS[args.workload]
+        if args.shape:  # n,m[,tile]: a smaller case of the same recipe (for profiling)
+            dims = [int(x) for x in args.shape.split(",")]
+            w = inputs.TrsmWorkload(w.name + "@" + args.shape, dims[0], dims[1], dims[2] if len(dims) > 2 else w.tile, seed=w.seed,
+                                    coupling=w.coupling)
+        if args.steps is None:
+            args.steps = 3 if args.impl == "reference" else {"t1": 500, "t2": 50}[w.name.split("@")[0]]
+        (run_trsm_reference if args.impl == "reference" else run_trsm)(args, w)
+        return
     w = inputs.WORKLOADS[args.workload]
     if args.shape:
         dims = [int(x) for x in args.shape.split(",")]
