@@ -234,3 +234,49 @@ def make_trsm_operands(w: TrsmWorkload):
     L[np.arange(n), np.arange(n)] = sign * (np.float32(1.0) + v)
     B = uniform_f32(w.seed, TENSOR_RHS, n * m, -1.0, 1.0).reshape(n, m)
     return L, B
+
+
+# ---------------------------------------------------------------------- FlashAttention-2 recurrence
+TENSOR_Q = 5
+TENSOR_K = 6
+TENSOR_V = 7
+
+
+@dataclass(frozen=True)
+class AttentionWorkload:
+    """Synthetic attention problem: ``batch`` independent (Q, K, V) triples, bf16, ``Q`` ``[N][d]``, ``K``/``V`` ``[M][d]``.
+
+    ``Q`` and ``K`` are normal(0, ``qk_std``), ``V`` uniform in ``[-1, 1)``: with unit ``qk_std`` the scaled scores
+    ``Q K^T / sqrt(d)`` have unit variance, the regime of a trained attention layer's logits.
+    """
+    name: str
+    batch: int
+    N: int
+    M: int
+    d: int
+    seed: int
+    qk_std: float = 1.0
+
+    @property
+    def flops(self) -> int:
+        """Two matrix products per (query, key) pair: ``4 N M d`` per problem."""
+        return 4 * self.batch * self.N * self.M * self.d
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        """Q, K, V read once (bf16), O written once (fp32)."""
+        return self.batch * ((self.N + 2 * self.M) * self.d * 2 + self.N * self.d * 4)
+
+
+ATTENTION_WORKLOADS = {
+    "a1": AttentionWorkload("a1", 2, 300, 500, 64, seed=20),
+    "a2": AttentionWorkload("a2", 32, 4096, 4096, 128, seed=21),
+}
+
+
+def make_attention_operands(w: AttentionWorkload):
+    """Host arrays ``(Q, K, V)`` as bf16 bit patterns (uint16), shapes ``[batch][N][d]`` and ``[batch][M][d]``."""
+    Q = f32_to_bf16_bits(normal_f32(w.seed, TENSOR_Q, w.batch * w.N * w.d, w.qk_std)).reshape(w.batch, w.N, w.d)
+    K = f32_to_bf16_bits(normal_f32(w.seed, TENSOR_K, w.batch * w.M * w.d, w.qk_std)).reshape(w.batch, w.M, w.d)
+    V = f32_to_bf16_bits(uniform_f32(w.seed, TENSOR_V, w.batch * w.M * w.d, -1.0, 1.0)).reshape(w.batch, w.M, w.d)
+    return Q, K, V
