@@ -177,6 +177,26 @@ int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, const void* L,
                    unsigned flags);
 
 /*
+ * FlashAttention-2 recurrence (Section "Simulated Cholesky and Flash Attention"): for every
+ * query row i, over key tiles J_t,
+ *     S = alpha Q_i K_{J_t}^T,  mh = max(m, max S),  l <- e^(m-mh) l + sum_j e^(S_j-mh),
+ *     o <- e^(m-mh) o + sum_j e^(S_j-mh) V_j,  m <- mh;      O_i = o / l,  alpha = 1/sqrt(d),
+ * which equals softmax(alpha Q K^T) V.  `batch` independent problems (batch x heads, flattened).
+ *
+ *   Q      DEVICE, [batch][N][d] bf16, row-major, 16-byte aligned
+ *   K, V   DEVICE, [batch][M][d] bf16
+ *   O      DEVICE, [batch][N][d] fp32, fully overwritten, 16-byte aligned, must not overlap an input
+ *   dtype  CYC_BF16_F32 (bf16 in; scores, normaliser and output accumulated in fp32; the
+ *          exponentials enter the second product rounded to bf16); d = 64 or 128.  Anything
+ *          else is refused with CYC_ERR_UNSUPPORTED.
+ *   flags  0 (the paper's recurrence has no mask and no other scale)
+ * N, M >= 1 need not be multiples of the tile sizes (128 queries, 128 keys).  Asynchronous on
+ * `stream`; the caller owns all buffers; errors as for cyc_recurrence_matmul.
+ */
+int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t d, int dtype, const void* Q, const void* K, const void* V,
+                        void* O, void* stream, unsigned flags);
+
+/*
  * Synchronise `stream` and report whether a kernel enqueued by this library on
  * the current device since the previous call of this function gave up on a
  * bounded wait.  *out (HOST pointer, may be NULL) receives CYC_OK or

@@ -28,6 +28,7 @@ SYMBOLS = {
     "cyc_recurrence_matmul_host": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_recurrence_matmul_splitk_static": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_block_trsm": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
+    "cyc_flash_attention": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_selftest_bounded_wait": (_int, [_ptr, _i64]),
     "cyc_last_device_status": (_int, [_ptr, ctypes.POINTER(ctypes.c_int)]),
     "cyc_kernel_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
@@ -62,6 +63,7 @@ cyc_recurrence_matmul_batched = _lib.cyc_recurrence_matmul_batched
 cyc_recurrence_matmul_host = _lib.cyc_recurrence_matmul_host
 cyc_recurrence_matmul_splitk_static = _lib.cyc_recurrence_matmul_splitk_static
 cyc_block_trsm = _lib.cyc_block_trsm
+cyc_flash_attention = _lib.cyc_flash_attention
 cyc_selftest_bounded_wait = _lib.cyc_selftest_bounded_wait
 cyc_last_device_status = _lib.cyc_last_device_status
 CYC_STATIC_WORKSPACE_BYTES = 8 << 20
@@ -183,6 +185,28 @@ def block_trsm(L, B, X=None, *, tile: int = 0, fixed_k_order: bool = False):
     check(cyc_block_trsm(n, m, tile, _torch_dtype_code(L), L.data_ptr(), B.data_ptr(), X.data_ptr(), _stream(),
                          _flags(False, fixed_k_order)))
     return X
+
+
+def flash_attention(Q, K, V, O=None):
+    """``softmax(Q K^T / sqrt(d)) V`` by the FlashAttention-2 recurrence for contiguous bf16 CUDA tensors
+    ``Q[batch,N,d]``, ``K[batch,M,d]``, ``V[batch,M,d]`` (or rank 2 for one problem); fp32 result shaped like ``Q``."""
+    import torch
+    if Q.dim() == 2:
+        Q, K, V = Q.unsqueeze(0), K.unsqueeze(0), V.unsqueeze(0)
+        squeeze = True
+    else:
+        squeeze = False
+    if not all(t.is_cuda and t.is_contiguous() and t.dim() == 3 for t in (Q, K, V)):
+        raise ValueError("Q, K, V must be contiguous CUDA tensors of rank 2 or 3")
+    batch, N, d = Q.shape
+    M = K.shape[1]
+    if K.shape != (batch, M, d) or V.shape != (batch, M, d) or K.dtype != Q.dtype or V.dtype != Q.dtype:
+        raise ValueError("operand shapes or dtypes differ")
+    if O is None:
+        O = torch.empty((batch, N, d), dtype=torch.float32, device=Q.device)
+    check(cyc_flash_attention(batch, N, M, d, _torch_dtype_code(Q), Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(),
+                              _stream(), 0))
+    return O[0] if squeeze else O
 
 
 def last_device_status() -> int:

@@ -1,0 +1,296 @@
+// FlashAttention-2 recurrence (Section "Simulated Cholesky and Flash Attention"):
+//
+//   S_{i,J_t} = alpha Q_i K_{J_t}^T,  mh = max(m, max S),  l <- e^{m-mh} l + sum_j e^{S_ij-mh},
+//   o <- e^{m-mh} o + sum_j e^{S_ij-mh} V_j,  m <- mh,   O_i = o / l,     alpha = 1/sqrt(d)
+//
+// "Each processing element holds a query tile and computes a series of matrix multiplications followed by elementwise
+// activations in place": here a CTA holds a 128-row query tile in shared memory for its whole life and walks the key
+// tiles J_t (128 keys each):
+//   warp 0      TMA producer: Q once, then K_t and V_t into a two-stage ring
+//   warp 1      one thread issues tcgen05 MMAs:  S_t = Q K_t^T  (fp32, in tensor memory, two buffers) and
+//               U_t = P_t V_t (fp32, tensor memory), P_t = e^{S_t - mh} in bf16 read from shared memory
+//   warps 2-5   one thread per query row (= one TMEM lane): running maximum, P_t, normaliser, and the running output
+//               o <- e^{m-mh} o + U_t in registers
+// S_{t+1} is issued before U_t, so the tensor core works on the next scores while the row threads exponentiate.
+// Exponentials are 2^x on the scores scaled by alpha*log2(e).  bf16 inputs, fp32 output.  Every wait is bounded.
+#pragma once
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "ptx.cuh"
+#include "umma_kernel.cuh"
+
+namespace cyc {
+
+constexpr int FA2_THREADS = 192, FA2_BM = 128, FA2_BN = 128;
+
+struct Fa2Params {
+    float* O;          // [batch][N][D] fp32
+    int N, M;          // queries, keys
+    int tiles_q;       // ceil(N / 128)
+    float scale_log2;  // alpha * log2(e)
+    int* status;       // device status word
+};
+
+struct Fa2Ctl {
+    uint64_t q_full;
+    uint64_t kv_full[2], kv_empty[2];
+    uint64_t s_full[2], s_empty[2];
+    uint64_t p_ready, pv_done;
+    uint32_t tmem_base;
+    volatile int abort;
+};
+
+template <int D>
+struct Fa2Smem {
+    static constexpr int SLAB = 128 * 128;            // 128 rows x 128 bytes (64 bf16)
+    static constexpr int Q_BYTES = (D / 64) * SLAB;   // K-major A operand of S
+    static constexpr int K_BYTES = (D / 64) * SLAB;   // K-major B operand of S
+    static constexpr int V_BYTES = (D / 64) * SLAB;   // MN-major B operand of U: D/64 chunks of 128 keys x 128 bytes of d
+    static constexpr int STAGE_BYTES = K_BYTES + V_BYTES;
+    static constexpr int P_BYTES = 2 * SLAB;          // K-major A operand of U: two slabs of 64 keys
+    static constexpr int TOTAL = Q_BYTES + 2 * STAGE_BYTES + P_BYTES + 1024 + 1024;
+};
+
+__device__ __forceinline__ bool fa2_wait(uint64_t* bar, uint32_t parity, Fa2Ctl* ctl, int* status, int where) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if (ctl->abort) return false;
+        if (clock64() - t0 > UMMA_WAIT_CYCLES) {
+            ctl->abort = 1;
+            atomicExch(status, 0x300 | where);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ float fa2_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int D>
+__global__ void __launch_bounds__(FA2_THREADS, 1)
+fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+           const Fa2Params p) {
+    using Sm = Fa2Smem<D>;
+    static_assert(D == 64 || D == 128, "head dimension 64 or 128");
+    constexpr uint32_t TMEM_COLS = 512;                 // S0 | S1 | U  (128 + 128 + D columns)
+    constexpr uint32_t COL_S0 = 0, COL_U = 256;
+    constexpr uint32_t IDESC_S = umma_instr_desc(1, 1, false, FA2_BM, FA2_BN);
+    constexpr uint32_t IDESC_U = umma_instr_desc(1, 1, true, FA2_BM, D);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* sQ = smem;
+    uint8_t* sKV = sQ + Sm::Q_BYTES;
+    uint8_t* sP = sKV + 2 * Sm::STAGE_BYTES;
+    Fa2Ctl* ctl = reinterpret_cast<Fa2Ctl*>(sP + Sm::P_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x / p.tiles_q, qt = blockIdx.x - b * p.tiles_q;
+    const int n0 = qt * FA2_BM;
+    const int T = (p.M + FA2_BN - 1) / FA2_BN;  // key tiles
+
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&ctl->q_full, 1);
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(&ctl->kv_full[s], 1);
+            ptx::mbar_init(&ctl->kv_empty[s], 1);
+            ptx::mbar_init(&ctl->s_full[s], 1);
+            ptx::mbar_init(&ctl->s_empty[s], 4);
+        }
+        ptx::mbar_init(&ctl->p_ready, 4);
+        ptx::mbar_init(&ctl->pv_done, 1);
+        ctl->abort = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmQ);
+        ptx::prefetch_tensormap(&tmK);
+        ptx::prefetch_tensormap(&tmV);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc<1>(&ctl->tmem_base, TMEM_COLS);
+        ptx::tmem_relinquish<1>();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(&ctl->q_full, Sm::Q_BYTES);
+#pragma unroll
+            for (int kb = 0; kb < D / 64; ++kb) ptx::tma_load_3d(sQ + kb * Sm::SLAB, &tmQ, &ctl->q_full, kb * 64, n0, b);
+            int issued = 0;
+            bool ok = true;
+            for (int t = 0; t < T; ++t) {
+                const int st = t & 1;
+                if (!fa2_wait(&ctl->kv_empty[st], ((t >> 1) & 1) ^ 1, ctl, p.status, 1)) { ok = false; break; }
+                uint8_t* sK = sKV + st * Sm::STAGE_BYTES;
+                uint8_t* sV = sK + Sm::K_BYTES;
+                ptx::mbar_arrive_expect_tx(&ctl->kv_full[st], Sm::STAGE_BYTES);
+#pragma unroll
+                for (int kb = 0; kb < D / 64; ++kb) {
+                    ptx::tma_load_3d(sK + kb * Sm::SLAB, &tmK, &ctl->kv_full[st], kb * 64, t * FA2_BN, b);  // keys x 64 of d
+                    ptx::tma_load_3d(sV + kb * Sm::SLAB, &tmV, &ctl->kv_full[st], kb * 64, t * FA2_BN, b);  // keys x d-chunk kb
+                }
+                ++issued;
+            }
+            if (!ok) {
+                // leave no copy in flight: wait (bounded) for the loads already issued
+                const long long t0 = clock64();
+                while (!ptx::mbar_try_wait(&ctl->q_full, 0) && clock64() - t0 < UMMA_WAIT_CYCLES) {}
+                for (int u = issued - 1; u >= 0 && u >= issued - 2; --u) {
+                    const long long t1 = clock64();
+                    while (!ptx::mbar_try_wait(&ctl->kv_full[u & 1], (u >> 1) & 1) && clock64() - t1 < UMMA_WAIT_CYCLES) {}
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t aQ = ptx::smem_u32(sQ), aP = ptx::smem_u32(sP);
+            bool ok = fa2_wait(&ctl->q_full, 0, ctl, p.status, 2);
+            // U_u = P_u V_u : A = P (K-major, two slabs of 64 keys), B = V (MN-major: 128-byte rows of d, 8-key groups
+            // 1024 B apart, next 64 columns of d one slab on)
+            auto issue_u = [&](int u) -> bool {
+                if (!fa2_wait(&ctl->p_ready, u & 1, ctl, p.status, 3)) return false;
+                ptx::tc_fence_after();
+                const uint32_t aV = ptx::smem_u32(sKV + (u & 1) * Sm::STAGE_BYTES + Sm::K_BYTES);
+#pragma unroll
+                for (int k = 0; k < FA2_BN / 16; ++k) {
+                    const uint64_t adesc = umma_smem_desc(aP + (k >> 2) * Sm::SLAB + (k & 3) * 32, 16, 1024);
+                    const uint64_t bdesc = umma_smem_desc(aV + k * (16 * 128), Sm::SLAB, 1024);
+                    ptx::umma<KIND_BF16, 1>(tmem_base + COL_U, adesc, bdesc, IDESC_U, k != 0 ? 1u : 0u);
+                }
+                ptx::umma_commit(&ctl->pv_done);
+                ptx::umma_commit(&ctl->kv_empty[u & 1]);
+                return true;
+            };
+            for (int t = 0; t < T && ok; ++t) {
+                const int st = t & 1;
+                const uint32_t ph = (t >> 1) & 1;
+                if (!fa2_wait(&ctl->kv_full[st], ph, ctl, p.status, 4)) { ok = false; break; }
+                if (!fa2_wait(&ctl->s_empty[st], ph ^ 1, ctl, p.status, 5)) { ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t aK = ptx::smem_u32(sKV + st * Sm::STAGE_BYTES);
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {  // S_t = Q K_t^T, both K-major
+                    const uint32_t off = (k >> 2) * Sm::SLAB + (k & 3) * 32;
+                    ptx::umma<KIND_BF16, 1>(tmem_base + COL_S0 + st * FA2_BN, umma_smem_desc(aQ + off, 16, 1024),
+                                            umma_smem_desc(aK + off, 16, 1024), IDESC_S, k != 0 ? 1u : 0u);
+                }
+                ptx::umma_commit(&ctl->s_full[st]);
+                if (t > 0) ok = issue_u(t - 1);
+            }
+            if (ok) issue_u(T - 1);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ row threads: one query row per thread
+        const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int r = q * 32 + lane;            // row of the query tile
+        const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        float m = -INFINITY, l = 0.f, carry_prev = 0.f;
+        float o[D];
+#pragma unroll
+        for (int c = 0; c < D; ++c) o[c] = 0.f;
+        bool ok = true;
+        // o <- carry o + U_u  (U_u in tensor memory once pv_done has completed phase u & 1)
+        auto fold = [&](int u) -> bool {
+            if (!fa2_wait(&ctl->pv_done, u & 1, ctl, p.status, 6)) return false;
+            ptx::tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(lane_addr + COL_U + c0, v);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int g = 0; g < 32; ++g) o[c0 + g] = fmaf(o[c0 + g], carry_prev, __uint_as_float(v[g]));
+            }
+            return true;
+        };
+        for (int t = 0; t < T && ok; ++t) {
+            const int st = t & 1;
+            if (!fa2_wait(&ctl->s_full[st], (t >> 1) & 1, ctl, p.status, 7)) { ok = false; break; }
+            ptx::tc_fence_after();
+            const uint32_t s_addr = lane_addr + COL_S0 + st * FA2_BN;
+            const int valid = min(FA2_BN, p.M - t * FA2_BN);  // keys of this tile that exist
+            // running maximum (of the raw dot products; the positive scale commutes with max)
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < FA2_BN; c0 += 32) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(s_addr + c0, v);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int g = 0; g < 32; ++g)
+                    if (c0 + g < valid) mx = fmaxf(mx, __uint_as_float(v[g]));
+            }
+            const float m_new = fmaxf(m, mx * p.scale_log2);
+            const float carry = fa2_exp2(m - m_new);  // 2^(-inf) = 0 on the first tile
+            // previous tile's product must be complete before P is overwritten; fold it into the running output
+            if (t > 0 && !fold(t - 1)) { ok = false; break; }
+            // P_t = 2^(S scale - m_new) as bf16 into shared memory (K-major, 128-byte swizzle), row sum in fp32
+            float lsum = 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < FA2_BN; c0 += 32) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(s_addr + c0, v);
+                ptx::tmem_ld_wait();
+                uint32_t packed[16];
+#pragma unroll
+                for (int g = 0; g < 32; g += 2) {
+                    float p0 = (c0 + g < valid) ? fa2_exp2(fmaf(__uint_as_float(v[g]), p.scale_log2, -m_new)) : 0.f;
+                    float p1 = (c0 + g + 1 < valid) ? fa2_exp2(fmaf(__uint_as_float(v[g + 1]), p.scale_log2, -m_new)) : 0.f;
+                    lsum += p0 + p1;
+                    __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                    packed[g >> 1] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                uint8_t* slab = sP + (c0 >> 6) * Sm::SLAB + r * 128;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    const int chunk = ((c0 & 32) >> 3) + g;  // 16-byte chunk of the 128-byte row
+                    *reinterpret_cast<uint4*>(slab + ((chunk ^ (r & 7)) << 4)) =
+                        make_uint4(packed[4 * g], packed[4 * g + 1], packed[4 * g + 2], packed[4 * g + 3]);
+                }
+            }
+            l = fmaf(l, carry, lsum);
+            m = m_new;
+            carry_prev = carry;
+            ptx::tc_fence_before();
+            ptx::fence_proxy_async_smem();  // the MMA reads P through the async proxy
+            __syncwarp();
+            if (lane == 0) {
+                ptx::mbar_arrive(&ctl->p_ready);
+                ptx::mbar_arrive(&ctl->s_empty[st]);
+            }
+        }
+        if (ok) ok = fold(T - 1);
+        if (ok && n0 + r < p.N) {
+            const float inv = 1.0f / l;
+            float* dst = p.O + (static_cast<long long>(b) * p.N + n0 + r) * D;
+#pragma unroll
+            for (int c = 0; c < D; c += 4)
+                *reinterpret_cast<float4*>(dst + c) = make_float4(o[c] * inv, o[c + 1] * inv, o[c + 2] * inv, o[c + 3] * inv);
+        }
+        ptx::tc_fence_before();
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc<1>(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace cyc

@@ -84,6 +84,24 @@ def test_block_trsm_arguments_rejected_on_host(binding):
     assert t(1 << 31, 4, 0, 0, L, B, X, None, 0) == b.CYC_ERR_UNSUPPORTED
 
 
+def test_flash_attention_arguments_rejected_on_host(binding):
+    b = binding
+    Q, K, V, O = 1 << 20, 1 << 30, 1 << 34, 1 << 40   # never dereferenced: validation comes first
+    f = b.cyc_flash_attention
+    assert f(0, 8, 8, 64, 1, Q, K, V, O, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(1, 0, 8, 64, 1, Q, K, V, O, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(1, 8, -3, 64, 1, Q, K, V, O, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(1, 8, 8, 64, 9, Q, K, V, O, None, 0) == b.CYC_ERR_INVALID_ARG          # unknown dtype
+    assert f(1, 8, 8, 64, 1, Q, K, V, O, None, 1) == b.CYC_ERR_INVALID_ARG          # no flag applies
+    assert f(1, 8, 8, 64, 1, None, K, V, O, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(1, 8, 8, 64, 1, Q, K, V, None, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(1, 8, 8, 64, 1, Q + 1, K, V, O, None, 0) == b.CYC_ERR_INVALID_ARG      # bf16 operand not 2-byte aligned
+    assert f(1, 8, 8, 64, 1, Q, K, V, Q + 64, None, 0) == b.CYC_ERR_INVALID_ARG     # O over Q
+    assert f(1, 8, 8, 64, 0, Q, K, V, O, None, 0) == b.CYC_ERR_UNSUPPORTED          # fp32 inputs
+    assert f(1, 8, 8, 96, 1, Q, K, V, O, None, 0) == b.CYC_ERR_UNSUPPORTED          # head dimension
+    assert f(1, 8, 8, 64, 1, Q + 2, K, V, O, None, 0) == b.CYC_ERR_UNSUPPORTED      # not 16-byte aligned
+
+
 def test_kernel_selection(binding):
     k = binding.kernel_for
     assert k(1, 64, 64, 64, "f32", fixed_k_order=True) == "simt"
