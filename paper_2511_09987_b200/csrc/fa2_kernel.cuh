@@ -6,11 +6,12 @@
 // "Each processing element holds a query tile and computes a series of matrix multiplications followed by elementwise
 // activations in place": here a CTA holds a 128-row query tile in shared memory for its whole life and walks the key
 // tiles J_t (128 keys each):
-//   warp 0      TMA producer: Q once, then K_t and V_t into a two-stage ring
+//   warp 0      TMA producer: Q once, then K_t and V_t into two buffers each (K_t is released as soon as S_t is done)
 //   warp 1      one thread issues tcgen05 MMAs:  S_t = Q K_t^T  (fp32, in tensor memory, two buffers) and
 //               U_t = P_t V_t (fp32, tensor memory), P_t = e^{S_t - mh} in bf16 read from shared memory
-//   warps 2-5   one thread per query row (= one TMEM lane): running maximum, P_t, normaliser, and the running output
-//               o <- e^{m-mh} o + U_t in registers
+//   warps 2-9   two threads per query row (= one TMEM lane; warps 2-5 take keys 0-63 of the tile and the first half of
+//               the d columns, warps 6-9 the rest): running maximum (the two partial maxima meet through shared memory),
+//               P_t, partial normaliser, and the running output o <- e^{m-mh} o + U_t in registers
 // S_{t+1} is issued before U_t, so the tensor core works on the next scores while the row threads exponentiate.
 // Exponentials are 2^x on the scores scaled by alpha*log2(e).  bf16 inputs, fp32 output.  Every wait is bounded.
 #pragma once
@@ -24,7 +25,7 @@
 
 namespace cyc {
 
-constexpr int FA2_THREADS = 192, FA2_BM = 128, FA2_BN = 128;
+constexpr int FA2_THREADS = 320, FA2_BM = 128, FA2_BN = 128;
 
 struct Fa2Params {
     float* O;          // [batch][N][D] fp32
@@ -36,11 +37,13 @@ struct Fa2Params {
 
 struct Fa2Ctl {
     uint64_t q_full;
-    uint64_t kv_full[2], kv_empty[2];
+    uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
     uint64_t s_full[2], s_empty[2];
     uint64_t p_ready, pv_done;
     uint32_t tmem_base;
     volatile int abort;
+    float row_max[2][2][FA2_BM];  // [tile parity][half][row]: partial maxima of the two threads of a row
+    float row_sum[2][FA2_BM];     // [half][row]: partial normalisers, exchanged once at the end
 };
 
 template <int D>
@@ -51,7 +54,7 @@ struct Fa2Smem {
     static constexpr int V_BYTES = (D / 64) * SLAB;   // MN-major B operand of U: D/64 chunks of 128 keys x 128 bytes of d
     static constexpr int STAGE_BYTES = K_BYTES + V_BYTES;
     static constexpr int P_BYTES = 2 * SLAB;          // K-major A operand of U: two slabs of 64 keys
-    static constexpr int TOTAL = Q_BYTES + 2 * STAGE_BYTES + P_BYTES + 1024 + 1024;
+    static constexpr int TOTAL = Q_BYTES + 2 * STAGE_BYTES + P_BYTES + 4096 + 1024;  // + control block + alignment slack
 };
 
 __device__ __forceinline__ bool fa2_wait(uint64_t* bar, uint32_t parity, Fa2Ctl* ctl, int* status, int where) {
@@ -100,12 +103,14 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (threadIdx.x == 0) {
         ptx::mbar_init(&ctl->q_full, 1);
         for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(&ctl->kv_full[s], 1);
-            ptx::mbar_init(&ctl->kv_empty[s], 1);
+            ptx::mbar_init(&ctl->k_full[s], 1);
+            ptx::mbar_init(&ctl->k_empty[s], 1);
+            ptx::mbar_init(&ctl->v_full[s], 1);
+            ptx::mbar_init(&ctl->v_empty[s], 1);
             ptx::mbar_init(&ctl->s_full[s], 1);
-            ptx::mbar_init(&ctl->s_empty[s], 4);
+            ptx::mbar_init(&ctl->s_empty[s], 8);
         }
-        ptx::mbar_init(&ctl->p_ready, 4);
+        ptx::mbar_init(&ctl->p_ready, 8);
         ptx::mbar_init(&ctl->pv_done, 1);
         ctl->abort = 0;
         ptx::fence_mbar_init();
@@ -128,28 +133,39 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ptx::mbar_arrive_expect_tx(&ctl->q_full, Sm::Q_BYTES);
 #pragma unroll
             for (int kb = 0; kb < D / 64; ++kb) ptx::tma_load_3d(sQ + kb * Sm::SLAB, &tmQ, &ctl->q_full, kb * 64, n0, b);
-            int issued = 0;
+            // K_t is free again as soon as S_t has been computed, V_t only after U_t: separate barriers, so that the
+            // next keys are on their way one whole tile earlier than the next values
+            int issued_k = 0, issued_v = 0;
             bool ok = true;
             for (int t = 0; t < T; ++t) {
                 const int st = t & 1;
-                if (!fa2_wait(&ctl->kv_empty[st], ((t >> 1) & 1) ^ 1, ctl, p.status, 1)) { ok = false; break; }
+                const uint32_t ph = (t >> 1) & 1;
                 uint8_t* sK = sKV + st * Sm::STAGE_BYTES;
                 uint8_t* sV = sK + Sm::K_BYTES;
-                ptx::mbar_arrive_expect_tx(&ctl->kv_full[st], Sm::STAGE_BYTES);
+                if (!fa2_wait(&ctl->k_empty[st], ph ^ 1, ctl, p.status, 1)) { ok = false; break; }
+                ptx::mbar_arrive_expect_tx(&ctl->k_full[st], Sm::K_BYTES);
 #pragma unroll
-                for (int kb = 0; kb < D / 64; ++kb) {
-                    ptx::tma_load_3d(sK + kb * Sm::SLAB, &tmK, &ctl->kv_full[st], kb * 64, t * FA2_BN, b);  // keys x 64 of d
-                    ptx::tma_load_3d(sV + kb * Sm::SLAB, &tmV, &ctl->kv_full[st], kb * 64, t * FA2_BN, b);  // keys x d-chunk kb
-                }
-                ++issued;
+                for (int kb = 0; kb < D / 64; ++kb)
+                    ptx::tma_load_3d(sK + kb * Sm::SLAB, &tmK, &ctl->k_full[st], kb * 64, t * FA2_BN, b);  // keys x 64 of d
+                ++issued_k;
+                if (!fa2_wait(&ctl->v_empty[st], ph ^ 1, ctl, p.status, 8)) { ok = false; break; }
+                ptx::mbar_arrive_expect_tx(&ctl->v_full[st], Sm::V_BYTES);
+#pragma unroll
+                for (int kb = 0; kb < D / 64; ++kb)
+                    ptx::tma_load_3d(sV + kb * Sm::SLAB, &tmV, &ctl->v_full[st], kb * 64, t * FA2_BN, b);  // keys x d-chunk kb
+                ++issued_v;
             }
             if (!ok) {
                 // leave no copy in flight: wait (bounded) for the loads already issued
                 const long long t0 = clock64();
                 while (!ptx::mbar_try_wait(&ctl->q_full, 0) && clock64() - t0 < UMMA_WAIT_CYCLES) {}
-                for (int u = issued - 1; u >= 0 && u >= issued - 2; --u) {
+                for (int u = issued_k - 1; u >= 0 && u >= issued_k - 2; --u) {
                     const long long t1 = clock64();
-                    while (!ptx::mbar_try_wait(&ctl->kv_full[u & 1], (u >> 1) & 1) && clock64() - t1 < UMMA_WAIT_CYCLES) {}
+                    while (!ptx::mbar_try_wait(&ctl->k_full[u & 1], (u >> 1) & 1) && clock64() - t1 < UMMA_WAIT_CYCLES) {}
+                }
+                for (int u = issued_v - 1; u >= 0 && u >= issued_v - 2; --u) {
+                    const long long t1 = clock64();
+                    while (!ptx::mbar_try_wait(&ctl->v_full[u & 1], (u >> 1) & 1) && clock64() - t1 < UMMA_WAIT_CYCLES) {}
                 }
             }
         }
@@ -162,6 +178,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // U_u = P_u V_u : A = P (K-major, two slabs of 64 keys), B = V (MN-major: 128-byte rows of d, 8-key groups
             // 1024 B apart, next 64 columns of d one slab on)
             auto issue_u = [&](int u) -> bool {
+                if (!fa2_wait(&ctl->v_full[u & 1], (u >> 1) & 1, ctl, p.status, 9)) return false;
                 if (!fa2_wait(&ctl->p_ready, u & 1, ctl, p.status, 3)) return false;
                 ptx::tc_fence_after();
                 const uint32_t aV = ptx::smem_u32(sKV + (u & 1) * Sm::STAGE_BYTES + Sm::K_BYTES);
@@ -172,13 +189,13 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     ptx::umma<KIND_BF16, 1>(tmem_base + COL_U, adesc, bdesc, IDESC_U, k != 0 ? 1u : 0u);
                 }
                 ptx::umma_commit(&ctl->pv_done);
-                ptx::umma_commit(&ctl->kv_empty[u & 1]);
+                ptx::umma_commit(&ctl->v_empty[u & 1]);
                 return true;
             };
             for (int t = 0; t < T && ok; ++t) {
                 const int st = t & 1;
                 const uint32_t ph = (t >> 1) & 1;
-                if (!fa2_wait(&ctl->kv_full[st], ph, ctl, p.status, 4)) { ok = false; break; }
+                if (!fa2_wait(&ctl->k_full[st], ph, ctl, p.status, 4)) { ok = false; break; }
                 if (!fa2_wait(&ctl->s_empty[st], ph ^ 1, ctl, p.status, 5)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t aK = ptx::smem_u32(sKV + st * Sm::STAGE_BYTES);
@@ -189,60 +206,76 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                                             umma_smem_desc(aK + off, 16, 1024), IDESC_S, k != 0 ? 1u : 0u);
                 }
                 ptx::umma_commit(&ctl->s_full[st]);
+                ptx::umma_commit(&ctl->k_empty[st]);
                 if (t > 0) ok = issue_u(t - 1);
             }
             if (ok) issue_u(T - 1);
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------ row threads: one query row per thread
+        // ------------------------------------------------------------ row threads: two per query row
+        constexpr int HD = D / 2;               // d columns of the running output per thread
+        constexpr int HN = FA2_BN / 2;          // keys of a tile per thread
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;       // 0: keys 0-63, d columns 0..HD ; 1: the rest
         const int r = q * 32 + lane;            // row of the query tile
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
         float m = -INFINITY, l = 0.f, carry_prev = 0.f;
-        float o[D];
+        float o[HD];
 #pragma unroll
-        for (int c = 0; c < D; ++c) o[c] = 0.f;
+        for (int c = 0; c < HD; ++c) o[c] = 0.f;
         bool ok = true;
+        // the two warps that share a lane quarter meet at a named barrier of their own
+        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory"); };
         // o <- carry o + U_u  (U_u in tensor memory once pv_done has completed phase u & 1)
         auto fold = [&](int u) -> bool {
             if (!fa2_wait(&ctl->pv_done, u & 1, ctl, p.status, 6)) return false;
             ptx::tc_fence_after();
 #pragma unroll
-            for (int c0 = 0; c0 < D; c0 += 32) {
+            for (int c0 = 0; c0 < HD; c0 += 32) {
                 uint32_t v[32];
-                ptx::tmem_ld_32x32(lane_addr + COL_U + c0, v);
+                ptx::tmem_ld_32x32(lane_addr + COL_U + half * HD + c0, v);
                 ptx::tmem_ld_wait();
 #pragma unroll
                 for (int g = 0; g < 32; ++g) o[c0 + g] = fmaf(o[c0 + g], carry_prev, __uint_as_float(v[g]));
             }
             return true;
         };
-        for (int t = 0; t < T && ok; ++t) {
+        // Both threads of a row pass the named barrier exactly once per key tile and once after the loop, whatever
+        // happens: a thread whose wait ran out keeps walking the loop (doing nothing else) so that its partner is never
+        // left alone at the barrier.
+        for (int t = 0; t < T; ++t) {
             const int st = t & 1;
-            if (!fa2_wait(&ctl->s_full[st], (t >> 1) & 1, ctl, p.status, 7)) { ok = false; break; }
+            if (ok) ok = fa2_wait(&ctl->s_full[st], (t >> 1) & 1, ctl, p.status, 7);
             ptx::tc_fence_after();
-            const uint32_t s_addr = lane_addr + COL_S0 + st * FA2_BN;
-            const int valid = min(FA2_BN, p.M - t * FA2_BN);  // keys of this tile that exist
+            const uint32_t s_addr = lane_addr + COL_S0 + st * FA2_BN + half * HN;
+            const int valid = min(FA2_BN, p.M - t * FA2_BN) - half * HN;  // keys of this thread's half that exist
             // running maximum (of the raw dot products; the positive scale commutes with max)
             float mx = -INFINITY;
+            if (ok) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < FA2_BN; c0 += 32) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(s_addr + c0, v);
-                ptx::tmem_ld_wait();
+                for (int c0 = 0; c0 < HN; c0 += 32) {
+                    uint32_t v[32];
+                    ptx::tmem_ld_32x32(s_addr + c0, v);
+                    ptx::tmem_ld_wait();
 #pragma unroll
-                for (int g = 0; g < 32; ++g)
-                    if (c0 + g < valid) mx = fmaxf(mx, __uint_as_float(v[g]));
+                    for (int g = 0; g < 32; ++g)
+                        if (c0 + g < valid) mx = fmaxf(mx, __uint_as_float(v[g]));
+                }
             }
+            ctl->row_max[st][half][r] = mx;
+            pair_sync();
+            if (ctl->abort) ok = false;
+            if (!ok) continue;
+            mx = fmaxf(mx, ctl->row_max[st][half ^ 1][r]);
             const float m_new = fmaxf(m, mx * p.scale_log2);
             const float carry = fa2_exp2(m - m_new);  // 2^(-inf) = 0 on the first tile
             // previous tile's product must be complete before P is overwritten; fold it into the running output
-            if (t > 0 && !fold(t - 1)) { ok = false; break; }
+            if (t > 0 && !fold(t - 1)) { ok = false; continue; }
             // P_t = 2^(S scale - m_new) as bf16 into shared memory (K-major, 128-byte swizzle), row sum in fp32
             float lsum = 0.f;
 #pragma unroll 1
-            for (int c0 = 0; c0 < FA2_BN; c0 += 32) {
+            for (int c0 = 0; c0 < HN; c0 += 32) {
                 uint32_t v[32];
                 ptx::tmem_ld_32x32(s_addr + c0, v);
                 ptx::tmem_ld_wait();
@@ -255,10 +288,10 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                     packed[g >> 1] = *reinterpret_cast<uint32_t*>(&h);
                 }
-                uint8_t* slab = sP + (c0 >> 6) * Sm::SLAB + r * 128;
+                uint8_t* slab = sP + half * Sm::SLAB + r * 128;  // this half's 64 keys are one 128-byte row of slab `half`
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
-                    const int chunk = ((c0 & 32) >> 3) + g;  // 16-byte chunk of the 128-byte row
+                    const int chunk = (c0 >> 3) + g;  // 16-byte chunk of the 128-byte row
                     *reinterpret_cast<uint4*>(slab + ((chunk ^ (r & 7)) << 4)) =
                         make_uint4(packed[4 * g], packed[4 * g + 1], packed[4 * g + 2], packed[4 * g + 3]);
                 }
@@ -275,11 +308,14 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
         }
         if (ok) ok = fold(T - 1);
-        if (ok && n0 + r < p.N) {
-            const float inv = 1.0f / l;
-            float* dst = p.O + (static_cast<long long>(b) * p.N + n0 + r) * D;
+        // the normaliser of a row is the sum of its two partial ones
+        ctl->row_sum[half][r] = l;
+        pair_sync();
+        if (ok && !ctl->abort && n0 + r < p.N) {
+            const float inv = 1.0f / (l + ctl->row_sum[half ^ 1][r]);
+            float* dst = p.O + (static_cast<long long>(b) * p.N + n0 + r) * D + half * HD;
 #pragma unroll
-            for (int c = 0; c < D; c += 4)
+            for (int c = 0; c < HD; c += 4)
                 *reinterpret_cast<float4*>(dst + c) = make_float4(o[c] * inv, o[c + 1] * inv, o[c + 2] * inv, o[c + 3] * inv);
         }
         ptx::tc_fence_before();
