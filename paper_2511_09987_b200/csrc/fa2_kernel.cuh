@@ -8,7 +8,7 @@
 // tiles J_t (128 keys each):
 //   warp 0      TMA producer: Q once, then K_t and V_t into two buffers each (K_t is released as soon as S_t is done)
 //   warp 1      one thread issues tcgen05 MMAs:  S_t = Q K_t^T  (fp32, in tensor memory, two buffers) and
-//               U_t = P_t V_t (fp32, tensor memory), P_t = e^{S_t - mh} in bf16 read from shared memory
+//               U_t = P_t V_t (fp32, tensor memory, two buffers), P_t = e^{S_t - mh} in bf16 read from shared memory
 //   warps 2-9   two threads per query row (= one TMEM lane; warps 2-5 take keys 0-63 of the tile and the first half of
 //               the d columns, warps 6-9 the rest): running maximum (the two partial maxima meet through shared memory),
 //               P_t, partial normaliser, and the running output o <- e^{m-mh} o + U_t in registers
@@ -83,7 +83,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
            const Fa2Params p) {
     using Sm = Fa2Smem<D>;
     static_assert(D == 64 || D == 128, "head dimension 64 or 128");
-    constexpr uint32_t TMEM_COLS = 512;                 // S0 | S1 | U  (128 + 128 + D columns)
+    constexpr uint32_t TMEM_COLS = 512;                 // S0 | S1 | U0 | U1  (128 + 128 + D + D columns)
     constexpr uint32_t COL_S0 = 0, COL_U = 256;
     constexpr uint32_t IDESC_S = umma_instr_desc(1, 1, false, FA2_BM, FA2_BN);
     constexpr uint32_t IDESC_U = umma_instr_desc(1, 1, true, FA2_BM, D);
@@ -186,7 +186,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 for (int k = 0; k < FA2_BN / 16; ++k) {
                     const uint64_t adesc = umma_smem_desc(aP + (k >> 2) * Sm::SLAB + (k & 3) * 32, 16, 1024);
                     const uint64_t bdesc = umma_smem_desc(aV + k * (16 * 128), Sm::SLAB, 1024);
-                    ptx::umma<KIND_BF16, 1>(tmem_base + COL_U, adesc, bdesc, IDESC_U, k != 0 ? 1u : 0u);
+                    ptx::umma<KIND_BF16, 1>(tmem_base + COL_U + (u & 1) * D, adesc, bdesc, IDESC_U, k != 0 ? 1u : 0u);
                 }
                 ptx::umma_commit(&ctl->pv_done);
                 ptx::umma_commit(&ctl->v_empty[u & 1]);
@@ -227,19 +227,17 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         bool ok = true;
         // the two warps that share a lane quarter meet at a named barrier of their own
         auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory"); };
-        // o <- carry o + U_u  (U_u in tensor memory once pv_done has completed phase u & 1)
-        auto fold = [&](int u) -> bool {
-            if (!fa2_wait(&ctl->pv_done, u & 1, ctl, p.status, 6)) return false;
+        // o <- carry o + U_u  (U_u complete in its tensor-memory buffer: pv_done has completed phase u & 1)
+        auto fold = [&](int u) {
             ptx::tc_fence_after();
 #pragma unroll
             for (int c0 = 0; c0 < HD; c0 += 32) {
                 uint32_t v[32];
-                ptx::tmem_ld_32x32(lane_addr + COL_U + half * HD + c0, v);
+                ptx::tmem_ld_32x32(lane_addr + COL_U + (u & 1) * D + half * HD + c0, v);
                 ptx::tmem_ld_wait();
 #pragma unroll
                 for (int g = 0; g < 32; ++g) o[c0 + g] = fmaf(o[c0 + g], carry_prev, __uint_as_float(v[g]));
             }
-            return true;
         };
         // Both threads of a row pass the named barrier exactly once per key tile and once after the loop, whatever
         // happens: a thread whose wait ran out keeps walking the loop (doing nothing else) so that its partner is never
@@ -250,17 +248,36 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ptx::tc_fence_after();
             const uint32_t s_addr = lane_addr + COL_S0 + st * FA2_BN + half * HN;
             const int valid = min(FA2_BN, p.M - t * FA2_BN) - half * HN;  // keys of this thread's half that exist
-            // running maximum (of the raw dot products; the positive scale commutes with max)
+            // this thread's 64 scores: with the short running output (d = 64) they stay in registers from the maximum
+            // to the exponentials; with the long one (d = 128) they are read from tensor memory twice, 32 at a time
+            constexpr bool KEEP = (D == 64);
+            uint32_t sc[KEEP ? HN : 32];
             float mx = -INFINITY;
             if (ok) {
-#pragma unroll 1
-                for (int c0 = 0; c0 < HN; c0 += 32) {
-                    uint32_t v[32];
-                    ptx::tmem_ld_32x32(s_addr + c0, v);
+                if constexpr (KEEP) {
+                    ptx::tmem_ld_32x32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+                    ptx::tmem_ld_32x32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[KEEP ? 32 : 0]));
                     ptx::tmem_ld_wait();
+                    if (valid < HN) {  // only the last tile can be ragged
 #pragma unroll
-                    for (int g = 0; g < 32; ++g)
-                        if (c0 + g < valid) mx = fmaxf(mx, __uint_as_float(v[g]));
+                        for (int g = 0; g < HN; ++g)
+                            if (g >= valid) sc[KEEP ? g : 0] = 0xff800000u;  // a key that does not exist: -inf, weight 0
+                    }
+#pragma unroll
+                    for (int g = 0; g < HN; ++g) mx = fmaxf(mx, __uint_as_float(sc[KEEP ? g : 0]));
+                } else {
+#pragma unroll 1
+                    for (int c0 = 0; c0 < HN; c0 += 32) {
+                        ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+                        ptx::tmem_ld_wait();
+                        if (valid < HN) {
+#pragma unroll
+                            for (int g = 0; g < 32; ++g)
+                                if (c0 + g >= valid) sc[g] = 0xff800000u;
+                        }
+#pragma unroll
+                        for (int g = 0; g < 32; ++g) mx = fmaxf(mx, __uint_as_float(sc[g]));
+                    }
                 }
             }
             ctl->row_max[st][half][r] = mx;
@@ -270,35 +287,39 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             mx = fmaxf(mx, ctl->row_max[st][half ^ 1][r]);
             const float m_new = fmaxf(m, mx * p.scale_log2);
             const float carry = fa2_exp2(m - m_new);  // 2^(-inf) = 0 on the first tile
-            // previous tile's product must be complete before P is overwritten; fold it into the running output
-            if (t > 0 && !fold(t - 1)) { ok = false; continue; }
+            // the previous tile's product must have read P before P is overwritten
+            if (t > 0 && !fa2_wait(&ctl->pv_done, (t - 1) & 1, ctl, p.status, 6)) { ok = false; continue; }
             // P_t = 2^(S scale - m_new) as bf16 into shared memory (K-major, 128-byte swizzle), row sum in fp32
             float lsum = 0.f;
-#pragma unroll 1
+            uint8_t* slab = sP + half * Sm::SLAB + r * 128;  // this half's 64 keys are one 128-byte row of slab `half`
+#pragma unroll
             for (int c0 = 0; c0 < HN; c0 += 32) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(s_addr + c0, v);
-                ptx::tmem_ld_wait();
-                uint32_t packed[16];
+                if constexpr (!KEEP) {
+                    ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+                    ptx::tmem_ld_wait();
+                    if (valid < HN) {
 #pragma unroll
-                for (int g = 0; g < 32; g += 2) {
-                    float p0 = (c0 + g < valid) ? fa2_exp2(fmaf(__uint_as_float(v[g]), p.scale_log2, -m_new)) : 0.f;
-                    float p1 = (c0 + g + 1 < valid) ? fa2_exp2(fmaf(__uint_as_float(v[g + 1]), p.scale_log2, -m_new)) : 0.f;
-                    lsum += p0 + p1;
-                    __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                    packed[g >> 1] = *reinterpret_cast<uint32_t*>(&h);
+                        for (int g = 0; g < 32; ++g)
+                            if (c0 + g >= valid) sc[g] = 0xff800000u;
+                    }
                 }
-                uint8_t* slab = sP + half * Sm::SLAB + r * 128;  // this half's 64 keys are one 128-byte row of slab `half`
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const int chunk = (c0 >> 3) + g;  // 16-byte chunk of the 128-byte row
-                    *reinterpret_cast<uint4*>(slab + ((chunk ^ (r & 7)) << 4)) =
-                        make_uint4(packed[4 * g], packed[4 * g + 1], packed[4 * g + 2], packed[4 * g + 3]);
+                for (int g8 = 0; g8 < 4; ++g8) {  // 16-byte chunk of the row: eight exponentials
+                    uint32_t packed[4];
+#pragma unroll
+                    for (int e = 0; e < 8; e += 2) {
+                        const int at = (KEEP ? c0 : 0) + 8 * g8 + e;
+                        const float p0 = fa2_exp2(fmaf(__uint_as_float(sc[at]), p.scale_log2, -m_new));
+                        const float p1 = fa2_exp2(fmaf(__uint_as_float(sc[at + 1]), p.scale_log2, -m_new));
+                        lsum += p0 + p1;
+                        __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                        packed[e >> 1] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(slab + ((((c0 >> 3) + g8) ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                 }
             }
             l = fmaf(l, carry, lsum);
             m = m_new;
-            carry_prev = carry;
             ptx::tc_fence_before();
             ptx::fence_proxy_async_smem();  // the MMA reads P through the async proxy
             __syncwarp();
@@ -306,8 +327,12 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 ptx::mbar_arrive(&ctl->p_ready);
                 ptx::mbar_arrive(&ctl->s_empty[st]);
             }
+            // with P_t handed over, fold the previous tile's product (in the other U buffer) into the running output
+            if (t > 0) fold(t - 1);
+            carry_prev = carry;
         }
-        if (ok) ok = fold(T - 1);
+        if (ok) ok = fa2_wait(&ctl->pv_done, (T - 1) & 1, ctl, p.status, 10);
+        if (ok) fold(T - 1);
         // the normaliser of a row is the sum of its two partial ones
         ctl->row_sum[half][r] = l;
         pair_sync();
