@@ -4,7 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
 
 Workloads c1..c5 are the matrix-multiply recurrence (the default, c2, is the headline); t1 and t2 are the block
-lower-triangular solve built on it.
+lower-triangular solve built on it; a1 and a2 are the FlashAttention-2 recurrence.
 
 One step = one evaluation of the whole recurrence (weight load, B injection, the
 multiply-accumulate chain along k, export of C) for one workload.  Prints ONE JSON
@@ -505,6 +505,161 @@ def run_trsm_reference(args, w):
         "e2e": {"value": value, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
 
 
+def describe_attention(w):
+    return "%s: FlashAttention-2 recurrence bf16 batch=%d N=%d M=%d d=%d seed=%d qk_std=%g" % (w.name, w.batch, w.N, w.M, w.d, w.seed, w.qk_std)
+
+
+def cpu_attention_rate(w, Q, K, V, target_seconds=12.0, threads=None):
+    """Time the attention oracle (fp64 recurrence over key tiles of 128, as it stands) on a prefix of the query rows of
+    problem 0, repeated over problem 0 when one whole problem is too short a sample."""
+    from oracle import fa2 as ofa2
+    threads = threads or os.cpu_count() or 1
+    rows = min(w.N, threads)
+    while True:
+        reps_ = max(1, rows // w.N)
+        t0 = time.perf_counter()
+        for _ in range(reps_):
+            ofa2.attention(Q[0][:min(rows, w.N)], K[0], V[0], 128, threads=threads)
+        dt = time.perf_counter() - t0
+        if dt >= 0.5 * target_seconds or rows >= 4096 * w.N:
+            break
+        rows = int(rows * min(8.0, max(2.0, 0.9 * target_seconds / max(dt, 1e-3))))
+        if rows > w.N:
+            rows = (rows // w.N) * w.N
+    done = reps_ * min(rows, w.N)
+    rate = 4.0 * done * w.M * w.d / dt / 1e12
+    what = "query rows 0..%d" % (rows - 1) if rows <= w.N else "%d passes over all %d query rows" % (reps_, w.N)
+    return rate, threads, "%s of problem 0 of %s (M=%d d=%d), fp64 recurrence, %d threads, %.1f s" % (what, w.name, w.M, w.d, threads, dt)
+
+
+def run_attention_reference(args, w):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    Q, K, V = inputs.make_attention_operands(inputs.AttentionWorkload(w.name, 1, w.N, w.M, w.d, seed=w.seed, qk_std=w.qk_std))
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, sample, threads = [], "", os.cpu_count() or 1
+    for s in range(args.warmup + args.steps):
+        v, threads, sample = cpu_attention_rate(w, Q, K, V, target_seconds=per_step)
+        if s >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    print(json.dumps({
+        "impl": "reference", "metric": "flash_attention_throughput", "value": value, "unit": "TFLOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": w.flops / (value * 1e12) * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": describe_attention(w), "note": "ms_per_step extrapolated from the sampled rate"},
+        "cpu_baseline": {"value": value, "unit": "TFLOPS", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
+
+
+def run_attention(args, w):
+    """FlashAttention-2 recurrence (workloads a1, a2): one step = one launch over every (problem, query tile)."""
+    import torch
+    from paper_2511_09987_b200 import binding
+    from paper_2511_09987_b200.replicas import Replicas
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    reps = Replicas("nccl", torch.device("cuda", local))
+    world, rank = reps.world, reps.rank
+    peaks, peak_kind = load_peaks()
+    Q, K, V = inputs.make_attention_operands(w)
+    hQ, hK, hV = (torch.from_numpy(x).view(torch.bfloat16).pin_memory() for x in (Q, K, V))
+    hO = torch.empty((w.batch, w.N, w.d), dtype=torch.float32).pin_memory()
+    set_bytes = w.algorithmic_bytes
+    nsets = int(min(8, max(2, -(-3 * L2_BYTES // set_bytes))))
+    sets = [(hQ.cuda(), hK.cuda(), hV.cuda(), torch.empty((w.batch, w.N, w.d), dtype=torch.float32, device="cuda")) for _ in range(nsets)]
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        dQ, dK, dV, dO = sets[i % nsets]
+        binding.flash_attention(dQ, dK, dV, dO)
+
+    def barrier():
+        reps.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = binding.cyc_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    launches = binding.cyc_launch_count() - launches0
+    if binding.last_device_status() != binding.CYC_OK:
+        raise SystemExit("a device-side wait timed out during the benchmark: " + binding.cyc_last_cuda_error().decode())
+    clocks = sampler.stop()
+    total_ms = reps.max_over_ranks(e0.elapsed_time(e1))
+    ms_per_step = total_ms / args.steps
+    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+
+    # end to end: pinned host Q, K, V up, one launch, O down, every step
+    e2e_steps = 0 if args.kernel_only else max(3, min(args.steps, 10))
+    dQ, dK, dV, dO = sets[0]
+
+    def e2e_step():
+        dQ.copy_(hQ, non_blocking=True)
+        dK.copy_(hK, non_blocking=True)
+        dV.copy_(hV, non_blocking=True)
+        binding.flash_attention(dQ, dK, dV, dO)
+        hO.copy_(dO, non_blocking=True)
+
+    for _ in range(0 if args.kernel_only else 2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(1, e2e_steps)
+    e2e_value = None if args.kernel_only else world * w.flops / (reps.max_over_ranks(e2e_ms) * 1e-3) / 1e12
+    if rank != 0:
+        reps.close()
+        return
+    step_s = ms_per_step * 1e-3
+    which = "burst" if total_ms < 1000.0 else "sustained"
+    peak = float(peaks["bf16_tflops"] if which == "burst" else peaks["bf16_tflops_sustained"])
+    family = "fa2_d%d" % w.d
+    roofline = {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s", "frac": value / world / peak,
+                "traffic": load_traffic(w, family),
+                "peak_source": "%s bf16 cuBLAS %s; 4 N M d flop per problem (both products, exponentials not counted)" % (peak_kind, which),
+                "kernel": "fa2_kernel<%d>" % w.d, "kernel_us": step_s * 1e6}
+    if args.kernel_only:
+        cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
+    else:
+        cpu_v, cores, sample = cpu_attention_rate(w, Q, K, V)
+    if nsets * set_bytes > 2 * L2_BYTES:
+        l2_note = "inputs rotate over %d device copies (%.0f MB in total, larger than the 126 MB L2)" % (nsets, nsets * set_bytes / 1e6)
+    else:
+        l2_note = "working set of %d rotating copies is %.1f MB, below L2: no DRAM figure is claimed" % (nsets, nsets * set_bytes / 1e6)
+    line = {
+        "metric": "flash_attention_throughput", "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": describe_attention(w), "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": l2_note, "launch": "one library call per step"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "TFLOPS", "h2d_bytes_per_step": int((hQ.numel() + hK.numel() + hV.numel()) * 2),
+                "d2h_bytes_per_step": int(hO.numel() * 4), "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_v, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": sample},
+    }
+    print(json.dumps(line))
+    reps.close()
+
+
 # CUDA sources each kernel family is built from (host-side launch code is not part of a kernel's identity)
 KERNEL_SOURCES = {
     "simt": ["simt_kernel.cuh"],
@@ -513,6 +668,8 @@ KERNEL_SOURCES = {
     "tcgen05_pair_tall": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "umma_pair_tall_kernel.cuh"],
     "tcgen05_pair_splitk": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "splitk_reduce_kernel.cuh"],
     "tcgen05_3xtf32": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "umma_pair_tf32x3_kernel.cuh"],
+    "fa2_d64": ["ptx.cuh", "umma_kernel.cuh", "fa2_kernel.cuh"],
+    "fa2_d128": ["ptx.cuh", "umma_kernel.cuh", "fa2_kernel.cuh"],
 }
 
 
@@ -550,9 +707,9 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS))
+    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS) + sorted(inputs.ATTENTION_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--shape", default=None, help="M,N,K[,batch] (c1..c5) or n,m[,tile] (t1, t2): a smaller case of the workload's recipe (for profiling)")
+    ap.add_argument("--shape", default=None, help="M,N,K[,batch] (c1..c5), n,m[,tile] (t1, t2) or batch,N,M,d (a1, a2): a smaller case of the workload's recipe (for profiling)")
     ap.add_argument("--strict", action="store_true", help="set the fixed-k-order flag (fp32: the per-element FMA chain kernel)")
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="replay the timed steps from a CUDA graph (auto: only for launch-bound workloads)")
@@ -567,6 +724,15 @@ def main():
         if args.steps is None:
             args.steps = 3 if args.impl == "reference" else {"t1": 500, "t2": 50}[w.name.split("@")[0]]
         (run_trsm_reference if args.impl == "reference" else run_trsm)(args, w)
+        return
+    if args.workload in inputs.ATTENTION_WORKLOADS:
+        w = inputs.ATTENTION_WORKLOADS[args.workload]
+        if args.shape:
+            dims = [int(x) for x in args.shape.split(",")]
+            w = inputs.AttentionWorkload(w.name + "@" + args.shape, dims[0], dims[1], dims[2], dims[3], seed=w.seed, qk_std=w.qk_std)
+        if args.steps is None:
+            args.steps = 3 if args.impl == "reference" else {"a1": 500, "a2": 50}[w.name.split("@")[0]]
+        (run_attention_reference if args.impl == "reference" else run_attention)(args, w)
         return
     w = inputs.WORKLOADS[args.workload]
     if args.shape:
