@@ -4,7 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
 
 Workloads c1..c5 are the matrix-multiply recurrence (the default, c2, is the headline); t1 and t2 are the block
-lower-triangular solve built on it; a1 and a2 are the FlashAttention-2 recurrence.
+lower-triangular solve built on it; a1 and a2 are the FlashAttention-2 recurrence; p1..p3 the prefix-sum recurrence.
 
 One step = one evaluation of the whole recurrence (weight load, B injection, the
 multiply-accumulate chain along k, export of C) for one workload.  Prints ONE JSON
@@ -660,6 +660,157 @@ def run_attention(args, w):
     reps.close()
 
 
+def describe_scan(w):
+    return "%s: prefix-sum recurrence %s rows=%d n=%d seed=%d" % (w.name, w.dtype, w.rows, w.n, w.seed)
+
+
+def cpu_scan_rate(w, A, target_seconds=12.0):
+    """Time the prefix-sum oracle (the literal walk, as it stands; one thread: the recurrence is a single dependency
+    chain per row and the oracle does not split it) on a prefix of the elements, repeated when the workload is small."""
+    from oracle import scan as oscan
+    arith = "i32" if w.dtype == "i32" else "f64"
+    flat = A.reshape(-1)
+    count = min(flat.size, 1 << 20)
+    while True:
+        reps_ = max(1, count // flat.size)
+        t0 = time.perf_counter()
+        for _ in range(reps_):
+            oscan.prefix_sum(flat[:min(count, flat.size)], arithmetic=arith)
+        dt = time.perf_counter() - t0
+        if dt >= 0.5 * target_seconds or count >= 64 * flat.size:
+            break
+        count = int(count * min(8.0, max(2.0, 0.9 * target_seconds / max(dt, 1e-3))))
+        if count > flat.size:
+            count = (count // flat.size) * flat.size
+    done = reps_ * min(count, flat.size)
+    what = "elements 0..%d as one sequence" % (count - 1) if count <= flat.size else "%d passes over all %d elements" % (reps_, flat.size)
+    return done / dt / 1e9, 1, "%s of %s, literal walk (%s), 1 thread, %.1f s" % (what, w.name, arith, dt)
+
+
+def run_scan_reference(args, w):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    A = inputs.make_scan_operand(w)
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, sample = [], ""
+    for s in range(args.warmup + args.steps):
+        v, _, sample = cpu_scan_rate(w, A, target_seconds=per_step)
+        if s >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    print(json.dumps({
+        "impl": "reference", "metric": "prefix_sum_throughput", "value": value, "unit": "Gelem/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": w.elements / (value * 1e9) * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": describe_scan(w), "note": "ms_per_step extrapolated from the sampled rate"},
+        "cpu_baseline": {"value": value, "unit": "Gelem/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "Gelem/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
+
+
+def run_scan(args, w):
+    """Prefix-sum recurrence (workloads p1, p2, p3): one step = one launch over every tile of every row."""
+    import torch
+    from paper_2511_09987_b200 import binding
+    from paper_2511_09987_b200.replicas import Replicas
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    reps = Replicas("nccl", torch.device("cuda", local))
+    world, rank = reps.world, reps.rank
+    peaks, peak_kind = load_peaks()
+    A = inputs.make_scan_operand(w)
+    hA = torch.from_numpy(A).pin_memory()
+    hP = torch.empty_like(hA).pin_memory()
+    set_bytes = w.algorithmic_bytes
+    nsets = int(min(8, max(2, -(-3 * L2_BYTES // set_bytes))))
+    sets = [(hA.cuda(), torch.empty(A.shape, dtype=hA.dtype, device="cuda")) for _ in range(nsets)]
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        dA, dP = sets[i % nsets]
+        binding.prefix_sum(dA, dP)
+
+    def barrier():
+        reps.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = binding.cyc_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    launches = binding.cyc_launch_count() - launches0
+    if binding.last_device_status() != binding.CYC_OK:
+        raise SystemExit("a device-side wait timed out during the benchmark: " + binding.cyc_last_cuda_error().decode())
+    clocks = sampler.stop()
+    ms_per_step = reps.max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    value = world * w.elements / (ms_per_step * 1e-3) / 1e9
+
+    e2e_steps = 0 if args.kernel_only else max(3, min(args.steps, 10))
+    dA, dP = sets[0]
+
+    def e2e_step():
+        dA.copy_(hA, non_blocking=True)
+        binding.prefix_sum(dA, dP)
+        hP.copy_(dP, non_blocking=True)
+
+    for _ in range(0 if args.kernel_only else 2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(1, e2e_steps)
+    e2e_value = None if args.kernel_only else world * w.elements / (reps.max_over_ranks(e2e_ms) * 1e-3) / 1e9
+    if rank != 0:
+        reps.close()
+        return
+    step_s = ms_per_step * 1e-3
+    achieved = w.algorithmic_bytes / step_s / 1e9
+    peak = float(peaks["hbm_gbs"])
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": load_traffic(w, "scan"),
+                "peak_source": "%s STREAM-style copy; 8 bytes per element (read once, written once); the step also holds a "
+                               "memset of the tile descriptors (8 bytes per 4096 elements)" % peak_kind,
+                "kernel": "scan_kernel<%s>" % ("float" if w.dtype == "f32" else "int"), "kernel_us": step_s * 1e6}
+    if args.kernel_only:
+        cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
+    else:
+        cpu_v, cores, sample = cpu_scan_rate(w, A)
+    if nsets * set_bytes > 2 * L2_BYTES:
+        l2_note = "inputs rotate over %d device copies (%.0f MB in total, larger than the 126 MB L2)" % (nsets, nsets * set_bytes / 1e6)
+    else:
+        l2_note = "working set of %d rotating copies is %.1f MB, below L2: no DRAM figure is claimed" % (nsets, nsets * set_bytes / 1e6)
+    line = {
+        "metric": "prefix_sum_throughput", "value": value, "unit": "Gelem/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": describe_scan(w), "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": l2_note, "launch": "one library call per step"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "Gelem/s", "h2d_bytes_per_step": int(hA.numel() * 4),
+                "d2h_bytes_per_step": int(hP.numel() * 4), "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_v, "unit": "Gelem/s", "cores": cores, "kind": "oracle", "sample": sample},
+    }
+    print(json.dumps(line))
+    reps.close()
+
+
 # CUDA sources each kernel family is built from (host-side launch code is not part of a kernel's identity)
 KERNEL_SOURCES = {
     "simt": ["simt_kernel.cuh"],
@@ -668,6 +819,7 @@ KERNEL_SOURCES = {
     "tcgen05_pair_tall": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "umma_pair_tall_kernel.cuh"],
     "tcgen05_pair_splitk": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "splitk_reduce_kernel.cuh"],
     "tcgen05_3xtf32": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "umma_pair_tf32x3_kernel.cuh"],
+    "scan": ["scan_kernel.cuh"],
     "fa2_d64": ["ptx.cuh", "umma_kernel.cuh", "fa2_kernel.cuh"],
     "fa2_d128": ["ptx.cuh", "umma_kernel.cuh", "fa2_kernel.cuh"],
 }
@@ -707,9 +859,9 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS) + sorted(inputs.ATTENTION_WORKLOADS))
+    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS) + sorted(inputs.ATTENTION_WORKLOADS) + sorted(inputs.SCAN_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--shape", default=None, help="M,N,K[,batch] (c1..c5), n,m[,tile] (t1, t2) or batch,N,M,d (a1, a2): a smaller case of the workload's recipe (for profiling)")
+    ap.add_argument("--shape", default=None, help="M,N,K[,batch] (c1..c5), n,m[,tile] (t1, t2) batch,N,M,d (a1, a2) or rows,n (p1..p3): a smaller case of the workload's recipe (for profiling)")
     ap.add_argument("--strict", action="store_true", help="set the fixed-k-order flag (fp32: the per-element FMA chain kernel)")
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="replay the timed steps from a CUDA graph (auto: only for launch-bound workloads)")
@@ -724,6 +876,15 @@ def main():
         if args.steps is None:
             args.steps = 3 if args.impl == "reference" else {"t1": 500, "t2": 50}[w.name.split("@")[0]]
         (run_trsm_reference if args.impl == "reference" else run_trsm)(args, w)
+        return
+    if args.workload in inputs.SCAN_WORKLOADS:
+        w = inputs.SCAN_WORKLOADS[args.workload]
+        if args.shape:
+            dims = [int(x) for x in args.shape.split(",")]
+            w = inputs.ScanWorkload(w.name + "@" + args.shape, dims[0], dims[1], w.dtype, seed=w.seed)
+        if args.steps is None:
+            args.steps = 3 if args.impl == "reference" else {"p1": 2000, "p2": 200, "p3": 200}[w.name.split("@")[0]]
+        (run_scan_reference if args.impl == "reference" else run_scan)(args, w)
         return
     if args.workload in inputs.ATTENTION_WORKLOADS:
         w = inputs.ATTENTION_WORKLOADS[args.workload]

@@ -54,7 +54,8 @@ extern "C" {
 typedef enum {
     CYC_F32 = 0,
     CYC_BF16_F32 = 1,
-    CYC_I8_I32 = 2
+    CYC_I8_I32 = 2,
+    CYC_I32 = 3 /* int32 in, int32 out, wrap-around: cyc_prefix_sum only */
 } cyc_dtype_t;
 
 enum {
@@ -195,6 +196,31 @@ int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, const void* L,
  */
 int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t d, int dtype, const void* Q, const void* K, const void* V,
                         void* O, void* stream, unsigned flags);
+
+/*
+ * Prefix-sum recurrence (Figure "Representative recurrences"):  P_i = P_{i-1} + A_i, read with
+ * P_{-1} = 0, i.e. P_i = A_0 + ... + A_i, for `rows` independent sequences of n elements.
+ *
+ *   A      DEVICE, element i of sequence r at A[r * strideA + i]
+ *   P      DEVICE, same indexing with strideP; fully overwritten for i < n.  P may be the very
+ *          same buffer as A with the same stride (in place); any other overlap is
+ *          CYC_ERR_INVALID_ARG.
+ *   strideA, strideP   in elements, >= n; 0 means n (sequences back to back)
+ *   dtype  CYC_F32: sums of neighbouring elements are formed in fp32 inside tiles of 4096
+ *          elements, the value carried from tile to tile is fp64, and every P_i is rounded to
+ *          fp32 once: |P_i - exact| <= 1e-6 * sum_{k<=i} |A_k|, independent of n.  The order in
+ *          which tile sums are combined follows their arrival, so the last bit of a result may
+ *          differ between runs.
+ *          CYC_I32: two's-complement 32-bit integers, wrap-around on overflow; exact and
+ *          run-to-run identical.  Other types are refused with CYC_ERR_UNSUPPORTED.
+ *   flags  0
+ * rows, n >= 1; rows * ceil(n / 4096) < 2^31.  One pass over the data (each element read once,
+ * written once) in a single kernel; the tile descriptors (8 bytes per 4096 elements) come from
+ * the library's stream-ordered pool for the duration of the call.  Asynchronous on `stream`;
+ * the caller owns A and P; errors as for cyc_recurrence_matmul.
+ */
+int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A, int64_t strideA, void* P, int64_t strideP, void* stream,
+                   unsigned flags);
 
 /*
  * Synchronise `stream` and report whether a kernel enqueued by this library on

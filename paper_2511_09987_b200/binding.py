@@ -15,7 +15,7 @@ import os
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libcyc.so")
 
-CYC_F32, CYC_BF16_F32, CYC_I8_I32 = 0, 1, 2
+CYC_F32, CYC_BF16_F32, CYC_I8_I32, CYC_I32 = 0, 1, 2, 3
 CYC_FLAG_FIXED_K_ORDER, CYC_FLAG_B_COL_MAJOR = 1, 2
 CYC_OK, CYC_ERR_INVALID_ARG, CYC_ERR_UNSUPPORTED, CYC_ERR_CUDA, CYC_ERR_TIMEOUT = 0, 1, 2, 3, 4
 DTYPE_CODES = {"f32": CYC_F32, "bf16": CYC_BF16_F32, "i8": CYC_I8_I32}
@@ -29,6 +29,7 @@ SYMBOLS = {
     "cyc_recurrence_matmul_splitk_static": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_block_trsm": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_flash_attention": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _ptr, _u32]),
+    "cyc_prefix_sum": (_int, [_i64, _i64, _int, _ptr, _i64, _ptr, _i64, _ptr, _u32]),
     "cyc_selftest_bounded_wait": (_int, [_ptr, _i64]),
     "cyc_last_device_status": (_int, [_ptr, ctypes.POINTER(ctypes.c_int)]),
     "cyc_kernel_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
@@ -64,6 +65,7 @@ cyc_recurrence_matmul_host = _lib.cyc_recurrence_matmul_host
 cyc_recurrence_matmul_splitk_static = _lib.cyc_recurrence_matmul_splitk_static
 cyc_block_trsm = _lib.cyc_block_trsm
 cyc_flash_attention = _lib.cyc_flash_attention
+cyc_prefix_sum = _lib.cyc_prefix_sum
 cyc_selftest_bounded_wait = _lib.cyc_selftest_bounded_wait
 cyc_last_device_status = _lib.cyc_last_device_status
 CYC_STATIC_WORKSPACE_BYTES = 8 << 20
@@ -207,6 +209,28 @@ def flash_attention(Q, K, V, O=None):
     check(cyc_flash_attention(batch, N, M, d, _torch_dtype_code(Q), Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(),
                               _stream(), 0))
     return O[0] if squeeze else O
+
+
+def prefix_sum(A, P=None):
+    """Inclusive prefix sums ``P_i = P_{i-1} + A_i`` along the last dimension of a CUDA tensor ``A`` of rank 1 or 2
+    (float32 or int32; rows of a rank-2 tensor are independent sequences and may be strided).  ``P`` may be ``A``."""
+    import torch
+    if not A.is_cuda or A.dim() not in (1, 2) or A.stride(-1) != 1:
+        raise ValueError("A must be a CUDA tensor of rank 1 or 2 with a contiguous last dimension")
+    codes = {torch.float32: CYC_F32, torch.int32: CYC_I32}
+    if A.dtype not in codes:
+        raise ValueError("float32 or int32 only")
+    if P is None:
+        P = torch.empty(A.shape, dtype=A.dtype, device=A.device)
+    if P.shape != A.shape or P.dtype != A.dtype or not P.is_cuda or P.stride(-1) != 1:
+        raise ValueError("P must match A")
+    rows, n = (1, A.shape[0]) if A.dim() == 1 else A.shape
+    if rows * n == 0:
+        return P
+    sA = A.stride(0) if A.dim() == 2 and rows > 1 else n
+    sP = P.stride(0) if P.dim() == 2 and rows > 1 else n
+    check(cyc_prefix_sum(rows, n, codes[A.dtype], A.data_ptr(), sA, P.data_ptr(), sP, _stream(), 0))
+    return P
 
 
 def last_device_status() -> int:

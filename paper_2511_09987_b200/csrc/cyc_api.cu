@@ -21,6 +21,7 @@
 #include "umma_pair_tf32x3_kernel.cuh"
 #include "trsm_diag_kernel.cuh"
 #include "fa2_kernel.cuh"
+#include "scan_kernel.cuh"
 
 namespace cyc {
 
@@ -862,6 +863,59 @@ extern "C" int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return d == 64 ? launch_fa2<64>(batch, N, M, Q, K, V, static_cast<float*>(O), st)
                    : launch_fa2<128>(batch, N, M, Q, K, V, static_cast<float*>(O), st);
+}
+
+template <typename T>
+static int launch_scan(long long rows, long long n, const void* A, long long sA, void* P, long long sP, cudaStream_t st) {
+    ScanParams<T> p;
+    p.A = static_cast<const T*>(A);
+    p.P = static_cast<T*>(P);
+    p.n = n; p.strideA = sA; p.strideP = sP;
+    p.tiles_per_row = (n + SCAN_TILE - 1) / SCAN_TILE;
+    const long long tiles = rows * p.tiles_per_row;
+    p.vec_ok = (reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(P) % 16 == 0 && (rows == 1 || (sA % 4 == 0 && sP % 4 == 0)))
+                   ? 1 : 0;
+    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    cudaMemPool_t pool;
+    int rc = workspace_pool(&pool);
+    if (rc) return rc;
+    void* ws = nullptr;
+    const size_t bytes = sizeof(ScanHeader) + static_cast<size_t>(tiles) * sizeof(unsigned long long);
+    CYC_CUDA(cudaMallocFromPoolAsync(&ws, bytes, pool, st));
+    p.header = static_cast<ScanHeader*>(ws);
+    p.desc = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(ws) + sizeof(ScanHeader));
+    cudaError_t e = cudaMemsetAsync(ws, 0, bytes, st);  // counter, abort flag and every descriptor start at zero
+    if (e == cudaSuccess) {
+        scan_kernel<T><<<static_cast<unsigned>(tiles), SCAN_THREADS, 0, st>>>(p);
+        e = cudaGetLastError();
+        if (e == cudaSuccess) g_launches.fetch_add(1);
+    }
+    const cudaError_t e2 = cudaFreeAsync(ws, st);
+    if (e != cudaSuccess) return cuda_fail(e, "scan_kernel");
+    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaFreeAsync");
+    return CYC_OK;
+}
+
+extern "C" int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A, int64_t strideA, void* P, int64_t strideP,
+                              void* stream, unsigned flags) {
+    if (rows <= 0 || n <= 0 || !A || !P || flags != 0 || strideA < 0 || strideP < 0) return CYC_ERR_INVALID_ARG;
+    if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32 && dtype != CYC_I32) return CYC_ERR_INVALID_ARG;
+    const long long sA = strideA ? strideA : n, sP = strideP ? strideP : n;
+    if (sA < n || sP < n) return CYC_ERR_INVALID_ARG;
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(A), p0 = reinterpret_cast<uintptr_t>(P);
+    if ((a0 | p0) % 4) return CYC_ERR_INVALID_ARG;
+    if (rows > (1ll << 40) || n > (1ll << 40)) return CYC_ERR_UNSUPPORTED;
+    const uintptr_t abytes = (static_cast<uintptr_t>(rows - 1) * sA + n) * 4, pbytes = (static_cast<uintptr_t>(rows - 1) * sP + n) * 4;
+    const bool in_place = a0 == p0 && sA == sP;
+    if (!in_place && a0 < p0 + pbytes && p0 < a0 + abytes) return CYC_ERR_INVALID_ARG;
+    if (dtype != CYC_F32 && dtype != CYC_I32) {
+        snprintf(g_err, sizeof g_err, "prefix sum: fp32 or int32 only");
+        return CYC_ERR_UNSUPPORTED;
+    }
+    const long long tiles_per_row = (n + SCAN_TILE - 1) / SCAN_TILE;
+    if (tiles_per_row > 0x7fffffffll / rows) return CYC_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return dtype == CYC_F32 ? launch_scan<float>(rows, n, A, sA, P, sP, st) : launch_scan<int>(rows, n, A, sA, P, sP, st);
 }
 
 extern "C" int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles) {

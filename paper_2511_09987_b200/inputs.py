@@ -280,3 +280,47 @@ def make_attention_operands(w: AttentionWorkload):
     K = f32_to_bf16_bits(normal_f32(w.seed, TENSOR_K, w.batch * w.M * w.d, w.qk_std)).reshape(w.batch, w.M, w.d)
     V = f32_to_bf16_bits(uniform_f32(w.seed, TENSOR_V, w.batch * w.M * w.d, -1.0, 1.0)).reshape(w.batch, w.M, w.d)
     return Q, K, V
+
+
+# ---------------------------------------------------------------------- prefix-sum recurrence
+TENSOR_SCAN = 8
+
+
+@dataclass(frozen=True)
+class ScanWorkload:
+    """``rows`` independent sequences of ``n`` elements: float32 uniform in ``[-1, 1)`` (running sums that wander around
+    zero while ``sum |A|`` grows linearly: the case in which the carried value needs more than fp32), or int32 over the
+    whole 32-bit range (running sums that wrap around)."""
+    name: str
+    rows: int
+    n: int
+    dtype: str  # "f32" or "i32"
+    seed: int
+
+    @property
+    def elements(self) -> int:
+        return self.rows * self.n
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        """Each element read once and written once."""
+        return 8 * self.rows * self.n
+
+
+SCAN_WORKLOADS = {
+    "p1": ScanWorkload("p1", 3, 10000, "f32", seed=30),
+    "p2": ScanWorkload("p2", 1, 1 << 28, "f32", seed=31),
+    "p3": ScanWorkload("p3", 4096, 65536, "i32", seed=32),
+}
+
+
+def make_scan_operand(w: ScanWorkload) -> np.ndarray:
+    """Host array ``A`` of shape ``[rows][n]``."""
+    n = w.rows * w.n
+    if w.dtype == "f32":
+        return uniform_f32(w.seed, TENSOR_SCAN, n, -1.0, 1.0).reshape(w.rows, w.n)
+    if w.dtype == "i32":
+        def fn(s, c):
+            return (_bits(w.seed, TENSOR_SCAN, s, c) >> np.uint64(32)).astype(np.uint32).view(np.int32)
+        return _fill(n, fn, np.int32).reshape(w.rows, w.n)
+    raise ValueError("scan workloads are f32 or i32")

@@ -102,6 +102,26 @@ def test_flash_attention_arguments_rejected_on_host(binding):
     assert f(1, 8, 8, 64, 1, Q + 2, K, V, O, None, 0) == b.CYC_ERR_UNSUPPORTED      # not 16-byte aligned
 
 
+def test_prefix_sum_arguments_rejected_on_host(binding):
+    b = binding
+    A, P = 1 << 20, 1 << 30   # never dereferenced: validation comes first
+    f = b.cyc_prefix_sum
+    assert f(0, 8, 0, A, 0, P, 0, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(1, 0, 0, A, 0, P, 0, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(1, 8, 9, A, 0, P, 0, None, 0) == b.CYC_ERR_INVALID_ARG                # unknown dtype
+    assert f(1, 8, 0, A, 0, P, 0, None, 1) == b.CYC_ERR_INVALID_ARG                # no flag applies
+    assert f(1, 8, 0, None, 0, P, 0, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(1, 8, 0, A, 0, None, 0, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(2, 8, 0, A, 7, P, 0, None, 0) == b.CYC_ERR_INVALID_ARG                # stride shorter than a sequence
+    assert f(1, 8, 0, A + 2, 0, P, 0, None, 0) == b.CYC_ERR_INVALID_ARG            # not 4-byte aligned
+    assert f(1, 8, 0, A, 0, A + 16, 0, None, 0) == b.CYC_ERR_INVALID_ARG           # P over A, other than in place
+    assert f(2, 8, 0, A, 8, A, 16, None, 0) == b.CYC_ERR_INVALID_ARG               # same base, different strides
+    assert f(1, 8, 1, A, 0, P, 0, None, 0) == b.CYC_ERR_UNSUPPORTED                # bf16
+    assert f(1, 8, 2, A, 0, P, 0, None, 0) == b.CYC_ERR_UNSUPPORTED                # int8
+    assert f(1, (1 << 40) + 1, 3, A, 0, P, 0, None, 0) == b.CYC_ERR_UNSUPPORTED    # sequence too long
+    assert f(1 << 20, 1 << 24, 3, A, 0, 1 << 50, 0, None, 0) == b.CYC_ERR_UNSUPPORTED  # 2^32 tiles
+
+
 def test_kernel_selection(binding):
     k = binding.kernel_for
     assert k(1, 64, 64, 64, "f32", fixed_k_order=True) == "simt"
