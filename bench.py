@@ -784,7 +784,7 @@ def run_scan(args, w):
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": load_traffic(w, "scan"),
                 "peak_source": "%s STREAM-style copy; 8 bytes per element (read once, written once); the step also holds a "
-                               "memset of the tile descriptors (8 bytes per 4096 elements)" % peak_kind,
+                               "memset of the tile descriptors (8 bytes per 16384 elements)" % peak_kind,
                 "kernel": "scan_kernel<%s>" % ("float" if w.dtype == "f32" else "int"), "kernel_us": step_s * 1e6}
     if args.kernel_only:
         cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"

@@ -1,5 +1,6 @@
 // C ABI of the library: argument validation, kernel selection, tensor-map
 // construction and launches.  See include/cyc.h for the contract.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdint>
@@ -873,9 +874,11 @@ static int launch_scan(long long rows, long long n, const void* A, long long sA,
     p.n = n; p.strideA = sA; p.strideP = sP;
     p.tiles_per_row = (n + SCAN_TILE - 1) / SCAN_TILE;
     const long long tiles = rows * p.tiles_per_row;
+    p.total_tiles = tiles;
     p.vec_ok = (reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(P) % 16 == 0 && (rows == 1 || (sA % 4 == 0 && sP % 4 == 0)))
                    ? 1 : 0;
     CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    CYC_CUDA(cudaFuncSetAttribute(scan_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_BYTES));
     cudaMemPool_t pool;
     int rc = workspace_pool(&pool);
     if (rc) return rc;
@@ -886,7 +889,7 @@ static int launch_scan(long long rows, long long n, const void* A, long long sA,
     p.desc = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(ws) + sizeof(ScanHeader));
     cudaError_t e = cudaMemsetAsync(ws, 0, bytes, st);  // counter, abort flag and every descriptor start at zero
     if (e == cudaSuccess) {
-        scan_kernel<T><<<static_cast<unsigned>(tiles), SCAN_THREADS, 0, st>>>(p);
+        scan_kernel<T><<<static_cast<unsigned>(tiles), SCAN_THREADS, SCAN_SMEM_BYTES, st>>>(p);
         e = cudaGetLastError();
         if (e == cudaSuccess) g_launches.fetch_add(1);
     }

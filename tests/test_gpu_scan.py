@@ -2,11 +2,11 @@
 
 int32: bit-exact (wrap-around arithmetic is associative, so any grouping gives the same bits).
 float32: ``|P_i - P_oracle_i| <= 1e-6 * S_i`` with ``S_i = sum_{k<=i} |A_k|`` and the oracle's walk in fp64.  Derivation:
-the GPU forms sums inside a tile of 4096 elements in fp32 along a path of at most 15 additions (3 inside a group of four,
-5 across a warp, 5 across the warp totals, 2 to combine them), each with relative error 2^-24 on a partial sum bounded
-by the ``|A|`` mass it covers; the tile sums handed from tile to tile pass through at most 13 of those additions and are
-then carried in fp64; the final rounding of ``P_i`` to fp32 adds ``2^-24 |P_i|``.  Together at most
-``16 * 2^-24 * S_i = 9.6e-7 * S_i``, whatever the length of the sequence.
+the GPU forms fp32 sums only inside the 128 consecutive elements a warp owns: 3 additions inside a group of four, 5 across
+the lanes, 1 to combine them, each with relative error 2^-24 on a partial sum bounded by the ``|A|`` mass it covers; sums
+of 128 elements, tile sums and the value carried from tile to tile are fp64 (descriptors keep 50 significand bits); the
+final ``head + (tail + y)`` adds one rounding relative to the warp's own mass and one relative to ``|P_i|``.  Together at
+most ``11 * 2^-24 * S_i = 6.6e-7 * S_i``, whatever the length of the sequence.
 """
 import numpy as np
 import pytest
@@ -49,10 +49,12 @@ def check(P, A):
     return float((err / np.maximum(S, 1e-300)).max())
 
 
-CASES = [SW("one", 1, 1, "f32", 60), SW("one_i", 1, 1, "i32", 61), SW("three", 1, 3, "f32", 62), SW("tile_minus_1", 1, 4095, "i32", 63),
-         SW("tile", 1, 4096, "f32", 64), SW("tile_plus_1", 1, 4097, "f32", 65), SW("ragged", 1, 10001, "i32", 66),
+CASES = [SW("one", 1, 1, "f32", 60), SW("one_i", 1, 1, "i32", 61), SW("three", 1, 3, "f32", 62), SW("quarter_minus_1", 1, 4095, "i32", 63),
+         SW("quarter", 1, 4096, "f32", 64), SW("quarter_plus_1", 1, 4097, "f32", 65), SW("ragged", 1, 10001, "i32", 66),
+         SW("tile_minus_1", 1, 16383, "f32", 74), SW("tile", 2, 16384, "i32", 75), SW("tile_plus_1", 1, 16385, "f32", 76),
+         SW("tile_plus_quarter", 3, 16384 + 4096, "f32", 77),
          SW("p1", 3, 10000, "f32", 30), SW("odd_rows", 7, 4099, "i32", 67), SW("short_rows", 500, 37, "f32", 68),
-         SW("many_tiles", 1, 40 * 4096 + 13, "f32", 69), SW("many_tiles_i", 2, 70 * 4096 + 1, "i32", 70),
+         SW("many_tiles", 1, 40 * 16384 + 13, "f32", 69), SW("many_tiles_i", 2, 70 * 16384 + 4097, "i32", 70),
          SW("long_lookback", 1, 3000 * 4096 + 5, "f32", 71)]
 
 
@@ -76,7 +78,7 @@ def test_in_place_unaligned_and_pitched(dtype):
 
 
 def test_closed_forms_and_exact_cases():
-    n = 3 * 4096 + 77
+    n = 3 * 16384 + 77
     ones = np.ones((2, n), dtype=np.float32)
     assert (gpu_scan(ones) == np.arange(1, n + 1, dtype=np.float32)).all()          # exact: every partial sum is an integer < 2^24
     assert (gpu_scan(ones.astype(np.int32)) == np.arange(1, n + 1)).all()
