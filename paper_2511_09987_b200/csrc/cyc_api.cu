@@ -889,7 +889,9 @@ static int launch_scan(long long rows, long long n, const void* A, long long sA,
     p.desc = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(ws) + sizeof(ScanHeader));
     cudaError_t e = cudaMemsetAsync(ws, 0, bytes, st);  // counter, abort flag and every descriptor start at zero
     if (e == cudaSuccess) {
-        scan_kernel<T><<<static_cast<unsigned>(tiles), SCAN_THREADS, SCAN_SMEM_BYTES, st>>>(p);
+        // short rows need only their own quarters of the staging buffer: more CTAs fit an SM
+        const int quarters = static_cast<int>(std::min<long long>(SCAN_SUBS, (n + SCAN_SUB - 1) / SCAN_SUB));
+        scan_kernel<T><<<static_cast<unsigned>(tiles), SCAN_THREADS, quarters * SCAN_SUB * sizeof(T) + 128, st>>>(p);
         e = cudaGetLastError();
         if (e == cudaSuccess) g_launches.fetch_add(1);
     }

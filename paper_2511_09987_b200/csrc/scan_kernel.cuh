@@ -7,8 +7,9 @@
 // then the lanes of a warp) and the 128 warp-level sums of a tile are combined in element order by one warp; from tile
 // to tile it is carried through one 64-bit descriptor per tile in global memory: a tile first publishes the sum of its
 // own elements ("partial"), then looks back over its predecessors -- adding partial sums until it meets a tile that
-// already knows its running value ("inclusive") -- and publishes its own running value.  The running value advances by
-// at most 32 tiles per descriptor round trip, which is why tiles are this large.  Tiles take their index from a counter
+// already knows its running value ("inclusive") -- and publishes its own running value.  Along one long row the running
+// value advances by at most one look-back window per descriptor round trip (about a microsecond under load), which is
+// why tiles are this large.  Tiles take their index from a counter
 // in launch order, so every predecessor of a tile is resident and makes progress; every wait is bounded.
 //
 // fp32: sums inside a warp's 128 elements are fp32; warp-level sums, tile sums and the value carried between tiles are
@@ -26,6 +27,7 @@ constexpr int SCAN_THREADS = 256, SCAN_CHUNKS = 4, SCAN_SUB = SCAN_THREADS * SCA
 constexpr int SCAN_SUBS = 4, SCAN_TILE = SCAN_SUBS * SCAN_SUB;                                     // 16384 elements per tile
 constexpr int SCAN_WARPS = SCAN_THREADS / 32;
 constexpr int SCAN_SMEM_BYTES = SCAN_TILE * 4 + 128;
+constexpr int SCAN_WINDOW = 32;  // predecessors examined per round of the look-back (128 measured slower: 3.6 against 4.0 TB/s)
 constexpr long long SCAN_WAIT_CYCLES = 1ll << 31;
 constexpr unsigned long long SCAN_PARTIAL = 1, SCAN_INCLUSIVE = 2;
 
@@ -224,14 +226,21 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const ScanParams<T> 
             long long pos = tile - 1;           // nearest predecessor not yet added
             const long long t0 = clock64();
             while (true) {
-                const long long idx = pos - lane;
-                const bool in_row = idx >= first;
-                // a lane past the start of the row behaves like a finished tile with value zero: the walk ends there
-                unsigned long long word = ScanCarry<T>::pack(Carry(0), SCAN_INCLUSIVE);
+                // one round looks at the SCAN_WINDOW nearest predecessors not yet added, SCAN_WINDOW / 32 per lane (group e of a
+                // lane is predecessor e * 32 + lane of the round); a slot past the start of the row behaves like a
+                // finished tile with value zero, so the walk ends there
+                unsigned long long word[SCAN_WINDOW / 32];
                 unsigned int spins = 0;
                 while (true) {
-                    if (in_row) word = scan_ld_desc(&p.desc[idx]);
-                    if (__all_sync(0xffffffffu, (word & 3ull) != 0)) break;
+                    bool ready = true;
+#pragma unroll
+                    for (int e = 0; e < SCAN_WINDOW / 32; ++e) {
+                        const long long idx = pos - (e * 32 + lane);
+                        word[e] = idx >= first ? scan_ld_desc(&p.desc[idx]) : ScanCarry<T>::pack(Carry(0), SCAN_INCLUSIVE);
+                    }
+#pragma unroll
+                    for (int e = 0; e < SCAN_WINDOW / 32; ++e) ready = ready && (word[e] & 3ull) != 0;
+                    if (__all_sync(0xffffffffu, ready)) break;
                     if ((++spins & 63u) == 0) {
                         int give_up = 0;
                         if (lane == 0) {
@@ -246,14 +255,20 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const ScanParams<T> 
                     }
                 }
                 if (!wok) break;
-                const unsigned int done = __ballot_sync(0xffffffffu, (word & 3ull) == SCAN_INCLUSIVE);
-                const int stop = done ? __ffs(done) - 1 : 32;  // nearest tile that knows its running value
-                Carry v = lane <= stop ? ScanCarry<T>::value(word) : Carry(0);
+                bool found = false;
 #pragma unroll
-                for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-                carry += v;
-                if (done) break;
-                pos -= 32;
+                for (int e = 0; e < SCAN_WINDOW / 32; ++e) {
+                    if (found) continue;
+                    const unsigned int done = __ballot_sync(0xffffffffu, (word[e] & 3ull) == SCAN_INCLUSIVE);
+                    const int stop = done ? __ffs(done) - 1 : 32;  // nearest tile that knows its running value
+                    Carry v = lane <= stop ? ScanCarry<T>::value(word[e]) : Carry(0);
+#pragma unroll
+                    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+                    carry += v;
+                    found = done != 0;
+                }
+                if (found) break;
+                pos -= SCAN_WINDOW;
             }
             if (wok && lane == 0) scan_st_desc(&p.desc[tile], ScanCarry<T>::pack(carry + own, SCAN_INCLUSIVE));
         }
