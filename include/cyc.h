@@ -223,6 +223,34 @@ int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A, int64_t st
                    unsigned flags);
 
 /*
+ * Tiled Cholesky recurrence (Section "Simulated Cholesky and Flash Attention"; scalar form in
+ * Figure "Representative recurrences"): the lower-triangular L with A = L L^T, panel by panel,
+ *     L_jj = CHOL(A_jj - sum_{k<j} SYRK(L_jk)),   L_ij = TRSM(A_ij - sum_{k<j} GEMM(L_ik, L_jk), L_jj),  i > j.
+ *
+ *   n      order of A;  n >= 1
+ *   tile   edge of the square tiles, 1 .. 256; 0 selects 256.  The last tile may be ragged.  The
+ *          tile size changes only the grouping of the additions, not the mathematical result.
+ *   dtype  CYC_F32 (fp32 in, fp32 arithmetic, fp32 out); other types: CYC_ERR_UNSUPPORTED
+ *   A      DEVICE, [n][n] row-major, symmetric positive definite; only entries on and below the
+ *          diagonal are read (the rest may hold anything, NaN included)
+ *   L      DEVICE, [n][n] row-major.  Entries on and below the diagonal receive the factor.  L may
+ *          be the very same buffer as A (in place: entries above the diagonal are then left as
+ *          they are); otherwise the two must not overlap and entries above the diagonal are set
+ *          to zero.
+ *   flags  0, or CYC_FLAG_FIXED_K_ORDER: the SYRK / GEMM sums then run as per-element fp32
+ *          fused-multiply-add chains in increasing k (bit-reproducible, slower); without it they
+ *          may run on the tensor cores (fp32 split into TF32 parts).
+ * A matrix that is not positive definite yields NaN from the square root of a non-positive
+ * pivot, as the recurrence does; it is not an error.  The SYRK / GEMM sums are evaluated by the
+ * same kernels as cyc_recurrence_matmul (both operands sub-blocks of L with row pitch n) into a
+ * workspace of (n - T) * T * 4 bytes from the library's stream-ordered pool; diagonal tiles are
+ * factored in fp32 with IEEE square roots and divisions, the tiles below them solved by forward
+ * substitution in fp32 with rows scaled by the correctly rounded reciprocal of the diagonal entry.
+ * Asynchronous on `stream`; the caller owns A and L; errors as for cyc_recurrence_matmul.
+ */
+int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, void* L, void* stream, unsigned flags);
+
+/*
  * Synchronise `stream` and report whether a kernel enqueued by this library on
  * the current device since the previous call of this function gave up on a
  * bounded wait.  *out (HOST pointer, may be NULL) receives CYC_OK or

@@ -30,6 +30,7 @@ SYMBOLS = {
     "cyc_block_trsm": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_flash_attention": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_prefix_sum": (_int, [_i64, _i64, _int, _ptr, _i64, _ptr, _i64, _ptr, _u32]),
+    "cyc_cholesky": (_int, [_i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
     "cyc_selftest_bounded_wait": (_int, [_ptr, _i64]),
     "cyc_last_device_status": (_int, [_ptr, ctypes.POINTER(ctypes.c_int)]),
     "cyc_kernel_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
@@ -66,6 +67,7 @@ cyc_recurrence_matmul_splitk_static = _lib.cyc_recurrence_matmul_splitk_static
 cyc_block_trsm = _lib.cyc_block_trsm
 cyc_flash_attention = _lib.cyc_flash_attention
 cyc_prefix_sum = _lib.cyc_prefix_sum
+cyc_cholesky = _lib.cyc_cholesky
 cyc_selftest_bounded_wait = _lib.cyc_selftest_bounded_wait
 cyc_last_device_status = _lib.cyc_last_device_status
 CYC_STATIC_WORKSPACE_BYTES = 8 << 20
@@ -231,6 +233,20 @@ def prefix_sum(A, P=None):
     sP = P.stride(0) if P.dim() == 2 and rows > 1 else n
     check(cyc_prefix_sum(rows, n, codes[A.dtype], A.data_ptr(), sA, P.data_ptr(), sP, _stream(), 0))
     return P
+
+
+def cholesky(A, L=None, *, tile: int = 0, fixed_k_order: bool = False):
+    """Lower Cholesky factor of the symmetric positive definite float32 CUDA matrix ``A[n,n]`` (only its lower triangle is
+    read) by the tiled recurrence; ``L`` may be ``A`` (in place)."""
+    import torch
+    if not (A.is_cuda and A.is_contiguous() and A.dim() == 2 and A.shape[0] == A.shape[1] and A.dtype == torch.float32):
+        raise ValueError("A must be a contiguous square float32 CUDA tensor")
+    if L is None:
+        L = torch.empty_like(A)
+    if L.shape != A.shape or L.dtype != A.dtype or not L.is_cuda or not L.is_contiguous():
+        raise ValueError("L must match A")
+    check(cyc_cholesky(A.shape[0], tile, CYC_F32, A.data_ptr(), L.data_ptr(), _stream(), _flags(False, fixed_k_order)))
+    return L
 
 
 def last_device_status() -> int:

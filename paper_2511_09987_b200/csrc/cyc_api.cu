@@ -23,6 +23,7 @@
 #include "trsm_diag_kernel.cuh"
 #include "fa2_kernel.cuh"
 #include "scan_kernel.cuh"
+#include "chol_diag_kernel.cuh"
 
 namespace cyc {
 
@@ -84,8 +85,10 @@ struct Problem {
     long long sA, sB, sC;
     unsigned flags;
     long long lda = 0;  // row pitch of A in elements; 0 = dense (K).  Only internal callers set it (sub-blocks of L).
+    long long ldb = 0;  // pitch of B in elements (between rows k, or between columns j when stored [N][K]); 0 = dense
 };
 static long long lda_of(const Problem& q) { return q.lda ? q.lda : q.K; }
+static long long ldb_of(const Problem& q) { return q.ldb ? q.ldb : ((q.flags & CYC_FLAG_B_COL_MAJOR) ? q.K : q.N); }
 
 // host-side validation; no CUDA call
 static int validate(const Problem& q) {
@@ -116,8 +119,8 @@ static bool tma_ok(const Problem& q) {
     const bool colmajor = (q.flags & CYC_FLAG_B_COL_MAJOR) != 0;
     if (reinterpret_cast<uintptr_t>(q.A) % 16 || reinterpret_cast<uintptr_t>(q.B) % 16) return false;
     if ((lda_of(q) * eb) % 16) return false;            // A pitch
-    if (colmajor && (q.K * eb) % 16) return false;      // B pitch when stored [N][K]
-    if (!colmajor && (q.N * eb) % 16) return false;     // B pitch when stored [K][N]
+    (void)colmajor;
+    if ((ldb_of(q) * eb) % 16) return false;            // B pitch ([N][K] or [K][N] storage)
     if (q.batch > 1 && ((q.sA * eb) % 16 || (q.sB * eb) % 16)) return false;
     return true;
 }
@@ -171,8 +174,8 @@ static int launch_simt(const Problem& q, cudaStream_t st) {
     p.sA = q.sA; p.sB = q.sB; p.sC = q.sC;
     p.lda = lda_of(q);
     const bool colmajor = (q.flags & CYC_FLAG_B_COL_MAJOR) != 0;
-    p.b_sk = colmajor ? 1 : q.N;
-    p.b_sj = colmajor ? q.K : 1;
+    p.b_sk = colmajor ? 1 : ldb_of(q);
+    p.b_sj = colmajor ? ldb_of(q) : 1;
     p.tiles_m = static_cast<int>((q.M + SIMT_BM - 1) / SIMT_BM);
     p.tiles_n = static_cast<int>((q.N + SIMT_BN - 1) / SIMT_BN);
     const long long blocks = q.batch * p.tiles_m * p.tiles_n;
@@ -188,7 +191,7 @@ static int launch_simt(const Problem& q, cudaStream_t st) {
     }
     bool vec = false;
     if constexpr (sizeof(TIn) == 4) {
-        vec = !colmajor && q.K % 4 == 0 && lda_of(q) % 4 == 0 && q.N % 4 == 0 && q.sA % 4 == 0 && q.sB % 4 == 0 && q.sC % 4 == 0 &&
+        vec = !colmajor && q.ldb == 0 && q.K % 4 == 0 && lda_of(q) % 4 == 0 && q.N % 4 == 0 && q.sA % 4 == 0 && q.sB % 4 == 0 && q.sC % 4 == 0 &&
               reinterpret_cast<uintptr_t>(q.A) % 16 == 0 && reinterpret_cast<uintptr_t>(q.B) % 16 == 0 &&
               reinterpret_cast<uintptr_t>(q.C) % 16 == 0;
     }
@@ -289,8 +292,8 @@ static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
     CUtensorMap tmA, tmB;
     int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, BK, UMMA_BM);
     if (rc) return rc;
-    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
-    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, BN);
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, ldb_of(q), q.sB, CH, BK);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, ldb_of(q), q.sB, BK, BN);
     if (rc) return rc;
 
     UmmaParams p;
@@ -322,8 +325,8 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws 
     CUtensorMap tmA, tmB, tmC;
     int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, BK, PAIR_HALF);
     if (rc) return rc;
-    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
-    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, PAIR_HALF);
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, ldb_of(q), q.sB, CH, BK);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, ldb_of(q), q.sB, BK, PAIR_HALF);
     if (rc) return rc;
     PairParams p;
     void* out = ws ? ws : q.C;
@@ -424,8 +427,8 @@ static int launch_pair_tall_cfg(const Problem& q, cudaStream_t st, int sms) {
     CUtensorMap tmA, tmB, tmC;
     int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, BK, PAIR_HALF);
     if (rc) return rc;
-    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, CH, BK);
-    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, BK, PAIR_HALF);
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, ldb_of(q), q.sB, CH, BK);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, ldb_of(q), q.sB, BK, PAIR_HALF);
     if (rc) return rc;
     PairParams p;
     p.tma_store = (reinterpret_cast<uintptr_t>(q.C) % 16 == 0 && q.N % 4 == 0 && (q.batch == 1 || q.sC % 4 == 0)) ? 1 : 0;
@@ -458,8 +461,8 @@ static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
     int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, 32, PAIR_HALF);
     if (rc) return rc;
     // fp32 B stored [K][N] feeds the MMA column-contiguous: 32-byte-chunk swizzle (see umma_smem_desc)
-    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, q.N, q.sB, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
-    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, q.K, q.sB, 32, PAIR_HALF);
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, ldb_of(q), q.sB, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, ldb_of(q), q.sB, 32, PAIR_HALF);
     if (rc) return rc;
     PairParams p;
     p.tma_store = (reinterpret_cast<uintptr_t>(q.C) % 16 == 0 && q.N % 4 == 0 && (q.batch == 1 || q.sC % 4 == 0)) ? 1 : 0;
@@ -559,8 +562,11 @@ struct TrsmPlan {
 
 static int trsm_diag(const TrsmPlan& t, long long b, unsigned mask) {
     TrsmDiagParams p;
-    p.L = t.L; p.B = t.B; p.X = t.X; p.W = t.W;
+    p.L = t.L;
+    p.B = t.B + b * t.T * t.m; p.X = t.X + b * t.T * t.m; p.W = t.W ? t.W + b * t.T * t.m : nullptr;  // first row of the tile
     p.plane = t.plane;
+    p.b_r = p.x_r = p.w_r = t.m;
+    p.b_c = p.x_c = p.w_c = 1;
     p.n = static_cast<int>(t.n); p.m = static_cast<int>(t.m);
     p.r0 = static_cast<int>(b * t.T);
     p.rows = static_cast<int>(t.n - b * t.T < t.T ? t.n - b * t.T : t.T);
@@ -921,6 +927,81 @@ extern "C" int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A,
     if (tiles_per_row > 0x7fffffffll / rows) return CYC_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == CYC_F32 ? launch_scan<float>(rows, n, A, sA, P, sP, st) : launch_scan<int>(rows, n, A, sA, P, sP, st);
+}
+
+// ------------------------------------------------------------------ tiled Cholesky
+// Panel j (columns c0 .. c1 of L), left-looking: one recurrence-matmul launch forms W = L[c0:n, 0:c0] L[c0:c1, 0:c0]^T
+// (the SYRK sum of the diagonal tile in its first rows, the GEMM sums of the tiles below it in the rest); the diagonal
+// tile is factored by chol_diag_kernel; the tiles below are the rows of X L_jj^T = A[c1:n, c0:c1] - W, solved by
+// trsm_diag_kernel with the right-hand sides addressed as rows.
+extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, void* L, void* stream, unsigned flags) {
+    if (n <= 0 || tile < 0 || tile > CHOL_T_MAX || !A || !L) return CYC_ERR_INVALID_ARG;
+    if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
+    if (flags & ~CYC_FLAG_FIXED_K_ORDER) return CYC_ERR_INVALID_ARG;
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(A), l0 = reinterpret_cast<uintptr_t>(L);
+    if ((a0 | l0) % 4) return CYC_ERR_INVALID_ARG;
+    if (n > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
+    if (dtype != CYC_F32) return CYC_ERR_UNSUPPORTED;  // the factorisation is defined for fp32 only
+    const uintptr_t bytes = static_cast<uintptr_t>(n) * n * 4;
+    if (a0 != l0 && a0 < l0 + bytes && l0 < a0 + bytes) return CYC_ERR_INVALID_ARG;  // overlap other than in place
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const float* Af = static_cast<const float*>(A);
+    float* Lf = static_cast<float*>(L);
+    const long long T = tile ? tile : CHOL_T_MAX;
+    const bool in_place = a0 == l0;
+    CYC_CUDA(cudaFuncSetAttribute(chol_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM_BYTES));
+    CYC_CUDA(cudaFuncSetAttribute(trsm_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TRSM_SMEM_BYTES));
+    float* W = nullptr;
+    if (n > T) {
+        cudaMemPool_t pool;
+        int rc = workspace_pool(&pool);
+        if (rc) return rc;
+        void* ws = nullptr;
+        CYC_CUDA(cudaMallocFromPoolAsync(&ws, static_cast<size_t>(n - T) * T * sizeof(float), pool, st));
+        W = static_cast<float*>(ws);
+    }
+    int rc = CYC_OK;
+    for (long long c0 = 0; c0 < n && rc == CYC_OK; c0 += T) {
+        const long long c1 = std::min<long long>(n, c0 + T), w = c1 - c0, below = n - c1;
+        if (c0 > 0) {
+            Problem q{1, n - c0, w, c0, CYC_F32, Lf + c0 * n, Lf + c0 * n, W, (n - c0) * n, w * n, (n - c0) * w,
+                      (flags & CYC_FLAG_FIXED_K_ORDER) | CYC_FLAG_B_COL_MAJOR, n, n};
+            rc = route(q, st);
+            if (rc) break;
+        }
+        CholDiagParams d;
+        d.A = Af + c0 * n + c0; d.W = c0 > 0 ? W : nullptr; d.L = Lf + c0 * n + c0;
+        d.lda = n; d.ldw = w; d.ldl = n;
+        d.rows = static_cast<int>(w);
+        d.zero_upper = in_place ? 0 : 1;
+        chol_diag_kernel<<<1, CHOL_THREADS, CHOL_SMEM_BYTES, st>>>(d);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) { rc = cuda_fail(e, "chol_diag_kernel"); break; }
+        g_launches.fetch_add(1);
+        if (below > 0) {
+            TrsmDiagParams p;
+            p.L = Lf;
+            p.B = Af + c1 * n + c0; p.X = Lf + c1 * n + c0; p.W = c0 > 0 ? W + w * w : nullptr;
+            p.plane = 0;
+            p.b_r = 1; p.b_c = n; p.x_r = 1; p.x_c = n; p.w_r = 1; p.w_c = w;
+            p.n = static_cast<int>(n); p.m = static_cast<int>(below);
+            p.r0 = static_cast<int>(c0); p.rows = static_cast<int>(w);
+            p.mask = c0 > 0 ? 1u : 0u;
+            trsm_diag_kernel<<<static_cast<unsigned>((below + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, st>>>(p);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) { rc = cuda_fail(e, "trsm_diag_kernel"); break; }
+            g_launches.fetch_add(1);
+            if (!in_place) {  // zeros above the diagonal: the block row to the right of the diagonal tile
+                e = cudaMemset2DAsync(Lf + c0 * n + c1, static_cast<size_t>(n) * 4, 0, static_cast<size_t>(below) * 4, static_cast<size_t>(w), st);
+                if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMemset2DAsync"); break; }
+            }
+        }
+    }
+    if (W) {
+        cudaError_t e = cudaFreeAsync(W, st);
+        if (e != cudaSuccess && rc == CYC_OK) rc = cuda_fail(e, "cudaFreeAsync");
+    }
+    return rc;
 }
 
 extern "C" int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles) {

@@ -26,12 +26,14 @@ namespace cyc {
 
 struct TrsmDiagParams {
     const float* L;   // [n][n] row-major
-    const float* B;   // [n][m]
-    float* X;         // [n][m]; may be B
-    const float* W;   // planes [levels][n][m] of partial sums; not read when mask == 0
-    long long plane;  // n * m
-    int n, m;
-    int r0, rows;     // the tile: rows [r0, r0 + rows), rows <= TRSM_T_MAX
+    const float* B;   // right-hand side: entry (tile row r, column c) at B[r * b_r + c * b_c]
+    float* X;         // solution, entry (r, c) at X[r * x_r + c * x_c]; may be B
+    const float* W;   // planes of partial sums, entry (r, c) of plane l at W[l * plane + r * w_r + c * w_c]; not read when mask == 0
+    long long plane;
+    long long b_r, b_c, x_r, x_c, w_r, w_c;  // element strides: (m, 1) for row-major [rows][m]; (1, pitch) when the
+                                             // right-hand sides are the rows of a row-major matrix (X L^T = B)
+    int n, m;         // order of L; number of right-hand-side columns
+    int r0, rows;     // the tile of L: rows and columns [r0, r0 + rows), rows <= TRSM_T_MAX
     unsigned mask;    // bit l set: plane l holds a partial sum for these rows
 };
 
@@ -153,8 +155,8 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
         for (int i = 0; i < 8; ++i) {
             const int r = rb + TRSM_WARPS * i + warp;
             ok[i] = r < p.rows && col_ok;
-            at[i] = static_cast<long long>(p.r0 + r) * p.m + c;
-            v[i] = ok[i] ? __ldg(p.B + at[i]) : 0.f;
+            at[i] = r * p.w_r + c * p.w_c;
+            v[i] = ok[i] ? __ldg(p.B + r * p.b_r + c * p.b_c) : 0.f;
             xa[i] = 0.f;
         }
         unsigned mk = p.mask;
@@ -230,7 +232,7 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
 #pragma unroll
             for (int r = 0; r < TRSM_SB; ++r) {
                 Xs[s0 + r][lane] = sv[r];
-                if (s0 + r < p.rows && col_ok) p.X[static_cast<long long>(p.r0 + s0 + r) * p.m + c] = sv[r];
+                if (s0 + r < p.rows && col_ok) p.X[(s0 + r) * p.x_r + c * p.x_c] = sv[r];
             }
         } else if ((warp & 3) != 0 && s >= 1 && s + 1 < nsb) {
             // ---- trailing(s): rows below sub-block s, sixteen per warp at a time, with x of sub-block s-1.  Twelve

@@ -324,3 +324,48 @@ def make_scan_operand(w: ScanWorkload) -> np.ndarray:
             return (_bits(w.seed, TENSOR_SCAN, s, c) >> np.uint64(32)).astype(np.uint32).view(np.int32)
         return _fill(n, fn, np.int32).reshape(w.rows, w.n)
     raise ValueError("scan workloads are f32 or i32")
+
+
+# ---------------------------------------------------------------------- Cholesky recurrence
+TENSOR_CHOL = 9
+TENSOR_CHOL_DIAG = 10
+
+
+@dataclass(frozen=True)
+class CholWorkload:
+    """Symmetric positive definite ``A`` of order ``n``: diagonal ``1 + v``, ``v`` uniform in ``[0, 1)``; below the diagonal
+    ``coupling = "dominant"``: ``0.5 u_ij / n`` (every row strictly diagonally dominant, so positive definite by
+    Gershgorin) or ``"wigner"``: ``0.5 u_ij / sqrt(n)`` (order-one coupling: the off-diagonal part has spectral radius
+    about 0.58, eigenvalues of ``A`` stay above 0.4, condition number about 6), ``u`` uniform in ``[-1, 1)``.  Entries
+    above the diagonal are NaN: only the lower triangle is an input."""
+    name: str
+    n: int
+    tile: int
+    seed: int
+    coupling: str = "wigner"
+
+    @property
+    def flops(self) -> int:
+        """``n^3 / 3`` multiply-adds counted as two operations each, lower-order terms dropped."""
+        return self.n ** 3 // 3
+
+    @property
+    def algorithmic_bytes(self) -> int:
+        """Lower triangle of A read once, lower triangle of L written once."""
+        return self.n * (self.n + 1) // 2 * 8
+
+
+CHOL_WORKLOADS = {
+    "h1": CholWorkload("h1", 600, 64, seed=50),
+    "h2": CholWorkload("h2", 8192, 256, seed=51),
+}
+
+
+def make_chol_operand(w: CholWorkload) -> np.ndarray:
+    """Host array ``A`` ``[n][n]`` float32 with NaN above the diagonal."""
+    n = w.n
+    scale = 0.5 / n if w.coupling == "dominant" else 0.5 / np.sqrt(n)
+    A = (uniform_f32(w.seed, TENSOR_CHOL, n * n, -1.0, 1.0) * np.float32(scale)).reshape(n, n)
+    A[np.arange(n), np.arange(n)] = 1.0 + uniform_f32(w.seed, TENSOR_CHOL_DIAG, n, 0.0, 1.0)
+    A[np.triu_indices(n, 1)] = np.nan
+    return A

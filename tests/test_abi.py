@@ -119,7 +119,24 @@ def test_prefix_sum_arguments_rejected_on_host(binding):
     assert f(1, 8, 1, A, 0, P, 0, None, 0) == b.CYC_ERR_UNSUPPORTED                # bf16
     assert f(1, 8, 2, A, 0, P, 0, None, 0) == b.CYC_ERR_UNSUPPORTED                # int8
     assert f(1, (1 << 40) + 1, 3, A, 0, P, 0, None, 0) == b.CYC_ERR_UNSUPPORTED    # sequence too long
-    assert f(1 << 20, 1 << 24, 3, A, 0, 1 << 50, 0, None, 0) == b.CYC_ERR_UNSUPPORTED  # 2^32 tiles
+    assert f(1 << 22, 1 << 24, 3, A, 0, 1 << 50, 0, None, 0) == b.CYC_ERR_UNSUPPORTED  # 2^32 tiles
+
+
+def test_cholesky_arguments_rejected_on_host(binding):
+    b = binding
+    A, L = 1 << 20, 1 << 40   # never dereferenced: validation comes first
+    f = b.cyc_cholesky
+    assert f(0, 0, 0, A, L, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(8, -1, 0, A, L, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(8, 257, 0, A, L, None, 0) == b.CYC_ERR_INVALID_ARG                  # tile edge above 256
+    assert f(8, 0, 9, A, L, None, 0) == b.CYC_ERR_INVALID_ARG                    # unknown dtype
+    assert f(8, 0, 0, A, L, None, 2) == b.CYC_ERR_INVALID_ARG                    # only the fixed-k-order flag applies
+    assert f(8, 0, 0, None, L, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(8, 0, 0, A, None, None, 0) == b.CYC_ERR_INVALID_ARG
+    assert f(8, 0, 0, A + 2, L, None, 0) == b.CYC_ERR_INVALID_ARG                # not 4-byte aligned
+    assert f(8, 0, 0, A, A + 64, None, 0) == b.CYC_ERR_INVALID_ARG               # overlap other than in place
+    assert f(8, 0, 1, A, L, None, 0) == b.CYC_ERR_UNSUPPORTED                    # bf16
+    assert f(1 << 31, 0, 0, A, 1 << 62, None, 0) == b.CYC_ERR_UNSUPPORTED
 
 
 def test_kernel_selection(binding):
