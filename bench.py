@@ -4,7 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
 
 Workloads c1..c5 are the matrix-multiply recurrence (the default, c2, is the headline); t1 and t2 are the block
-lower-triangular solve built on it; a1 and a2 are the FlashAttention-2 recurrence; p1..p3 the prefix-sum recurrence.
+lower-triangular solve built on it; a1 and a2 are the FlashAttention-2 recurrence; p1..p3 the prefix-sum recurrence; h1 and h2 the tiled Cholesky recurrence.
 
 One step = one evaluation of the whole recurrence (weight load, B injection, the
 multiply-accumulate chain along k, export of C) for one workload.  Prints ONE JSON
@@ -811,6 +811,146 @@ def run_scan(args, w):
     reps.close()
 
 
+def describe_chol(w):
+    return "%s: tiled Cholesky f32 n=%d tile=%d seed=%d coupling=%s" % (w.name, w.n, w.tile, w.seed, w.coupling)
+
+
+def cpu_chol_rate(w, A, target_seconds=12.0, threads=None):
+    """Time the Cholesky oracle (tiled form, as it stands) on a leading principal block of A."""
+    from oracle import chol as ochol
+    threads = threads or os.cpu_count() or 1
+    m = min(w.n, 512)
+    while True:
+        t0 = time.perf_counter()
+        ochol.cholesky(np.ascontiguousarray(A[:m, :m]), w.tile, threads=threads)
+        dt = time.perf_counter() - t0
+        if dt >= 0.5 * target_seconds or m >= w.n:
+            break
+        m = int(min(w.n, m * min(2.0, max(1.26, (0.9 * target_seconds / max(dt, 1e-3)) ** (1.0 / 3.0)))))
+    rate = (m ** 3 / 3.0) / dt / 1e12
+    return rate, threads, "leading %d x %d block of %s, tiled form (tile %d), fp64, %d threads, %.1f s" % (m, m, w.name, w.tile, threads, dt)
+
+
+def run_chol_reference(args, w):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    A = inputs.make_chol_operand(w)
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, sample, threads = [], "", os.cpu_count() or 1
+    for s in range(args.warmup + args.steps):
+        v, threads, sample = cpu_chol_rate(w, A, target_seconds=per_step)
+        if s >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    print(json.dumps({
+        "impl": "reference", "metric": "cholesky_throughput", "value": value, "unit": "TFLOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": w.flops / (value * 1e12) * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": describe_chol(w), "note": "ms_per_step extrapolated from the sampled rate"},
+        "cpu_baseline": {"value": value, "unit": "TFLOPS", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
+
+
+def run_chol(args, w):
+    """Tiled Cholesky (workloads h1, h2): one step = one whole factorisation (every SYRK / GEMM launch, every diagonal
+    tile, every panel solve)."""
+    import torch
+    from paper_2511_09987_b200 import binding
+    from paper_2511_09987_b200.replicas import Replicas
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    reps = Replicas("nccl", torch.device("cuda", local))
+    world, rank = reps.world, reps.rank
+    peaks, peak_kind = load_peaks()
+    A = inputs.make_chol_operand(w)
+    hA = torch.from_numpy(A).pin_memory()
+    hL = torch.empty_like(hA).pin_memory()
+    dA = hA.cuda()
+    dL = torch.empty_like(dA)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        reps.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        binding.cholesky(dA, dL, tile=w.tile)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = binding.cyc_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        binding.cholesky(dA, dL, tile=w.tile)
+    e1.record(stream)
+    barrier()
+    launches = binding.cyc_launch_count() - launches0
+    if binding.last_device_status() != binding.CYC_OK:
+        raise SystemExit("a device-side wait timed out during the benchmark: " + binding.cyc_last_cuda_error().decode())
+    clocks = sampler.stop()
+    total_ms = reps.max_over_ranks(e0.elapsed_time(e1))
+    ms_per_step = total_ms / args.steps
+    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+
+    e2e_steps = 0 if args.kernel_only else max(3, min(args.steps, 10))
+
+    def e2e_step():
+        dA.copy_(hA, non_blocking=True)
+        binding.cholesky(dA, dL, tile=w.tile)
+        hL.copy_(dL, non_blocking=True)
+
+    for _ in range(0 if args.kernel_only else 2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(1, e2e_steps)
+    e2e_value = None if args.kernel_only else world * w.flops / (reps.max_over_ranks(e2e_ms) * 1e-3) / 1e12
+    if rank != 0:
+        reps.close()
+        return
+    step_s = ms_per_step * 1e-3
+    which = "burst" if total_ms < 1000.0 else "sustained"
+    base = float(peaks["bf16_tflops"] if which == "burst" else peaks["bf16_tflops_sustained"])
+    peak = base * NOMINAL_RATIO["tf32"]
+    roofline = {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s", "frac": value / world / peak,
+                "traffic": None,
+                "peak_source": "%s bf16 cuBLAS %s x nominal tf32/bf16 ratio %.1f; the whole step is rated (n^3/3 flop, the three "
+                               "TF32 products of each fp32 product counted once): %d launches per factorisation"
+                               % (peak_kind, which, NOMINAL_RATIO["tf32"], launches // max(1, args.steps)),
+                "kernel": "tcgen05_3xtf32 (SYRK/GEMM sums) + chol_diag (diagonal tiles) + trsm_diag (tiles below)", "kernel_us": step_s * 1e6}
+    if args.kernel_only:
+        cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
+    else:
+        cpu_v, cores, sample = cpu_chol_rate(w, A)
+    line = {
+        "metric": "cholesky_throughput", "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": describe_chol(w), "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "A and L (%.0f MB) exceed the 126 MB L2" % (2 * w.n * w.n * 4 / 1e6) if 2 * w.n * w.n * 4 > 2 * L2_BYTES
+                   else "working set below L2: latency-bound, no DRAM figure claimed",
+                   "launch": "one library call per step"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "TFLOPS", "h2d_bytes_per_step": int(hA.numel() * 4), "d2h_bytes_per_step": int(hL.numel() * 4),
+                "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_v, "unit": "TFLOPS", "cores": cores, "kind": "oracle", "sample": sample},
+    }
+    print(json.dumps(line))
+    reps.close()
+
+
 # CUDA sources each kernel family is built from (host-side launch code is not part of a kernel's identity)
 KERNEL_SOURCES = {
     "simt": ["simt_kernel.cuh"],
@@ -859,9 +999,10 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS) + sorted(inputs.ATTENTION_WORKLOADS) + sorted(inputs.SCAN_WORKLOADS))
+    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS) + sorted(inputs.ATTENTION_WORKLOADS) + sorted(inputs.SCAN_WORKLOADS)
+                    + sorted(inputs.CHOL_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--shape", default=None, help="M,N,K[,batch] (c1..c5), n,m[,tile] (t1, t2) batch,N,M,d (a1, a2) or rows,n (p1..p3): a smaller case of the workload's recipe (for profiling)")
+    ap.add_argument("--shape", default=None, help="M,N,K[,batch] (c1..c5), n,m[,tile] (t1, t2) batch,N,M,d (a1, a2), rows,n (p1..p3) or n[,tile] (h1, h2): a smaller case of the workload's recipe (for profiling)")
     ap.add_argument("--strict", action="store_true", help="set the fixed-k-order flag (fp32: the per-element FMA chain kernel)")
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="replay the timed steps from a CUDA graph (auto: only for launch-bound workloads)")
@@ -876,6 +1017,15 @@ def main():
         if args.steps is None:
             args.steps = 3 if args.impl == "reference" else {"t1": 500, "t2": 50}[w.name.split("@")[0]]
         (run_trsm_reference if args.impl == "reference" else run_trsm)(args, w)
+        return
+    if args.workload in inputs.CHOL_WORKLOADS:
+        w = inputs.CHOL_WORKLOADS[args.workload]
+        if args.shape:
+            dims = [int(x) for x in args.shape.split(",")]
+            w = inputs.CholWorkload(w.name + "@" + args.shape, dims[0], dims[1] if len(dims) > 1 else w.tile, seed=w.seed, coupling=w.coupling)
+        if args.steps is None:
+            args.steps = 3 if args.impl == "reference" else {"h1": 200, "h2": 30}[w.name.split("@")[0]]
+        (run_chol_reference if args.impl == "reference" else run_chol)(args, w)
         return
     if args.workload in inputs.SCAN_WORKLOADS:
         w = inputs.SCAN_WORKLOADS[args.workload]

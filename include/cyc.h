@@ -243,9 +243,9 @@ int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A, int64_t st
  * A matrix that is not positive definite yields NaN from the square root of a non-positive
  * pivot, as the recurrence does; it is not an error.  The SYRK / GEMM sums are evaluated by the
  * same kernels as cyc_recurrence_matmul (both operands sub-blocks of L with row pitch n) into a
- * workspace of (n - T) * T * 4 bytes from the library's stream-ordered pool; diagonal tiles are
- * factored in fp32 with IEEE square roots and divisions, the tiles below them solved by forward
- * substitution in fp32 with rows scaled by the correctly rounded reciprocal of the diagonal entry.
+ * workspace of (n - T) * T * 4 bytes from the library's stream-ordered pool; everything
+ * else is fp32 with IEEE square roots; divisions by a pivot are multiplications by its correctly
+ * rounded reciprocal.
  * Asynchronous on `stream`; the caller owns A and L; errors as for cyc_recurrence_matmul.
  */
 int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, void* L, void* stream, unsigned flags);
