@@ -951,26 +951,44 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
     const bool in_place = a0 == l0;
     CYC_CUDA(cudaFuncSetAttribute(chol_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM_BYTES));
     CYC_CUDA(cudaFuncSetAttribute(trsm_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TRSM_SMEM_BYTES));
+    // The k range of a panel's sums is cut into up to CHOL_MAX_SLICES equal slices (one batched launch: a panel has
+    // few 256-row tiles, and the slices give every CTA pair work) plus one launch for the remainder; the consumers
+    // add the slices' partial sums in increasing k.
+    constexpr int CHOL_MAX_SLICES = 8;
     float* W = nullptr;
+    const long long plane = (n - T) * T;
     if (n > T) {
         cudaMemPool_t pool;
         int rc = workspace_pool(&pool);
         if (rc) return rc;
         void* ws = nullptr;
-        CYC_CUDA(cudaMallocFromPoolAsync(&ws, static_cast<size_t>(n - T) * T * sizeof(float), pool, st));
+        CYC_CUDA(cudaMallocFromPoolAsync(&ws, static_cast<size_t>(CHOL_MAX_SLICES + 1) * plane * sizeof(float), pool, st));
         W = static_cast<float*>(ws);
     }
     int rc = CYC_OK;
     for (long long c0 = 0; c0 < n && rc == CYC_OK; c0 += T) {
         const long long c1 = std::min<long long>(n, c0 + T), w = c1 - c0, below = n - c1;
+        int planes = 0;
         if (c0 > 0) {
-            Problem q{1, n - c0, w, c0, CYC_F32, Lf + c0 * n, Lf + c0 * n, W, (n - c0) * n, w * n, (n - c0) * w,
-                      (flags & CYC_FLAG_FIXED_K_ORDER) | CYC_FLAG_B_COL_MAJOR, n, n};
+            const long long kblocks = c0 / T, tiles_m = (n - c0 + 255) / 256;
+            long long S = std::min<long long>({static_cast<long long>(CHOL_MAX_SLICES), kblocks, std::max<long long>(1, kCtaPairs / tiles_m)});
+            const long long kc = (kblocks / S) * T, rem = c0 - S * kc;
+            const unsigned gflags = (flags & CYC_FLAG_FIXED_K_ORDER) | CYC_FLAG_B_COL_MAJOR;
+            Problem q{S, n - c0, w, kc, CYC_F32, Lf + c0 * n, Lf + c0 * n, W, kc, kc, plane, gflags, n, n};
             rc = route(q, st);
             if (rc) break;
+            planes = static_cast<int>(S);
+            if (rem > 0) {
+                Problem r{1, n - c0, w, rem, CYC_F32, Lf + c0 * n + S * kc, Lf + c0 * n + S * kc, W + S * plane, (n - c0) * n, w * n, plane,
+                          gflags, n, n};
+                rc = route(r, st);
+                if (rc) break;
+                ++planes;
+            }
         }
         CholDiagParams d;
-        d.A = Af + c0 * n + c0; d.W = c0 > 0 ? W : nullptr; d.L = Lf + c0 * n + c0;
+        d.A = Af + c0 * n + c0; d.W = W; d.L = Lf + c0 * n + c0;
+        d.plane = plane; d.planes = planes;
         d.lda = n; d.ldw = w; d.ldl = n;
         d.rows = static_cast<int>(w);
         d.zero_upper = in_place ? 0 : 1;
@@ -981,12 +999,12 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
         if (below > 0) {
             TrsmDiagParams p;
             p.L = Lf;
-            p.B = Af + c1 * n + c0; p.X = Lf + c1 * n + c0; p.W = c0 > 0 ? W + w * w : nullptr;
-            p.plane = 0;
+            p.B = Af + c1 * n + c0; p.X = Lf + c1 * n + c0; p.W = planes ? W + w * w : nullptr;
+            p.plane = plane;
             p.b_r = 1; p.b_c = n; p.x_r = 1; p.x_c = n; p.w_r = 1; p.w_c = w;
             p.n = static_cast<int>(n); p.m = static_cast<int>(below);
             p.r0 = static_cast<int>(c0); p.rows = static_cast<int>(w);
-            p.mask = c0 > 0 ? 1u : 0u;
+            p.mask = planes ? ((1u << planes) - 1u) : 0u;
             trsm_diag_kernel<<<static_cast<unsigned>((below + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, st>>>(p);
             e = cudaGetLastError();
             if (e != cudaSuccess) { rc = cuda_fail(e, "trsm_diag_kernel"); break; }
