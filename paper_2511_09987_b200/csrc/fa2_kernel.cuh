@@ -8,11 +8,14 @@
 // tiles J_t (128 keys each):
 //   warp 0      TMA producer: Q once, then K_t and V_t into two buffers each (K_t is released as soon as S_t is done)
 //   warp 1      one thread issues tcgen05 MMAs:  S_t = Q K_t^T  (fp32, in tensor memory, two buffers) and
-//               U_t = P_t V_t (fp32, tensor memory, two buffers), P_t = e^{S_t - mh} in bf16 read from shared memory
+//               U_t = P_t V_t (fp32, tensor memory, two buffers), P_t = e^{S_t - mh} in bf16 read from TENSOR memory:
+//               the row threads write P_t over the first 64 columns of the buffer S_t came in ("in place"), so P is
+//               double-buffered with S and never passes through shared memory
 //   warps 2-9   two threads per query row (= one TMEM lane; warps 2-5 take keys 0-63 of the tile and the first half of
 //               the d columns, warps 6-9 the rest): running maximum (the two partial maxima meet through shared memory),
 //               P_t, partial normaliser, and the running output o <- e^{m-mh} o + U_t in registers
-// S_{t+1} is issued before U_t, so the tensor core works on the next scores while the row threads exponentiate.
+// S_{t+1} is issued before U_t, so the tensor core works on the next scores while the row threads exponentiate, and
+// the exponentials of tile t do not wait for the product of tile t-1.
 // Exponentials are 2^x on the scores scaled by alpha*log2(e).  bf16 inputs, fp32 output.  Every wait is bounded.
 #pragma once
 #include <cstdint>
@@ -38,8 +41,8 @@ struct Fa2Params {
 struct Fa2Ctl {
     uint64_t q_full;
     uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
-    uint64_t s_full[2], s_empty[2];
-    uint64_t p_ready, pv_done;
+    uint64_t s_full[2], sp_free[2];   // scores ready / buffer free again (its P has been consumed)
+    uint64_t p_ready[2], pv_done[2];  // P written over the scores / U complete
     uint32_t tmem_base;
     volatile int abort;
     float row_max[2][2][FA2_BM];  // [tile parity][half][row]: partial maxima of the two threads of a row
@@ -53,8 +56,7 @@ struct Fa2Smem {
     static constexpr int K_BYTES = (D / 64) * SLAB;   // K-major B operand of S
     static constexpr int V_BYTES = (D / 64) * SLAB;   // MN-major B operand of U: D/64 chunks of 128 keys x 128 bytes of d
     static constexpr int STAGE_BYTES = K_BYTES + V_BYTES;
-    static constexpr int P_BYTES = 2 * SLAB;          // K-major A operand of U: two slabs of 64 keys
-    static constexpr int TOTAL = Q_BYTES + 2 * STAGE_BYTES + P_BYTES + 4096 + 1024;  // + control block + alignment slack
+    static constexpr int TOTAL = Q_BYTES + 2 * STAGE_BYTES + 4096 + 1024;  // + control block + alignment slack
 };
 
 __device__ __forceinline__ bool fa2_wait(uint64_t* bar, uint32_t parity, Fa2Ctl* ctl, int* status, int where) {
@@ -77,6 +79,31 @@ __device__ __forceinline__ float fa2_exp2(float x) {
     return y;
 }
 
+// D[tmem] (+)= A[tmem] * B[smem], bf16 operands, one CTA
+__device__ __forceinline__ void fa2_umma_tmem_a(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns from registers: thread t of the warp writes lane (base_lane + t)
+__device__ __forceinline__ void fa2_tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+        "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
+        "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void fa2_tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 template <int D>
 __global__ void __launch_bounds__(FA2_THREADS, 1)
 fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -92,8 +119,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* sQ = smem;
     uint8_t* sKV = sQ + Sm::Q_BYTES;
-    uint8_t* sP = sKV + 2 * Sm::STAGE_BYTES;
-    Fa2Ctl* ctl = reinterpret_cast<Fa2Ctl*>(sP + Sm::P_BYTES);
+    Fa2Ctl* ctl = reinterpret_cast<Fa2Ctl*>(sKV + 2 * Sm::STAGE_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x / p.tiles_q, qt = blockIdx.x - b * p.tiles_q;
@@ -108,10 +134,10 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ptx::mbar_init(&ctl->v_full[s], 1);
             ptx::mbar_init(&ctl->v_empty[s], 1);
             ptx::mbar_init(&ctl->s_full[s], 1);
-            ptx::mbar_init(&ctl->s_empty[s], 8);
+            ptx::mbar_init(&ctl->sp_free[s], 1);
+            ptx::mbar_init(&ctl->p_ready[s], 8);
+            ptx::mbar_init(&ctl->pv_done[s], 1);
         }
-        ptx::mbar_init(&ctl->p_ready, 8);
-        ptx::mbar_init(&ctl->pv_done, 1);
         ctl->abort = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmQ);
@@ -173,30 +199,32 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t aQ = ptx::smem_u32(sQ), aP = ptx::smem_u32(sP);
+            const uint32_t aQ = ptx::smem_u32(sQ);
             bool ok = fa2_wait(&ctl->q_full, 0, ctl, p.status, 2);
-            // U_u = P_u V_u : A = P (K-major, two slabs of 64 keys), B = V (MN-major: 128-byte rows of d, 8-key groups
-            // 1024 B apart, next 64 columns of d one slab on)
+            // U_u = P_u V_u : A = P in tensor memory (row = lane, two keys per 32-bit column, 16 keys = 8 columns per
+            // MMA), B = V (MN-major: 128-byte rows of d, 8-key groups 1024 B apart, next 64 columns of d one slab on)
             auto issue_u = [&](int u) -> bool {
-                if (!fa2_wait(&ctl->v_full[u & 1], (u >> 1) & 1, ctl, p.status, 9)) return false;
-                if (!fa2_wait(&ctl->p_ready, u & 1, ctl, p.status, 3)) return false;
+                const int su = u & 1;
+                const uint32_t pu = (u >> 1) & 1;
+                if (!fa2_wait(&ctl->v_full[su], pu, ctl, p.status, 9)) return false;
+                if (!fa2_wait(&ctl->p_ready[su], pu, ctl, p.status, 3)) return false;
                 ptx::tc_fence_after();
-                const uint32_t aV = ptx::smem_u32(sKV + (u & 1) * Sm::STAGE_BYTES + Sm::K_BYTES);
+                const uint32_t aV = ptx::smem_u32(sKV + su * Sm::STAGE_BYTES + Sm::K_BYTES);
 #pragma unroll
                 for (int k = 0; k < FA2_BN / 16; ++k) {
-                    const uint64_t adesc = umma_smem_desc(aP + (k >> 2) * Sm::SLAB + (k & 3) * 32, 16, 1024);
                     const uint64_t bdesc = umma_smem_desc(aV + k * (16 * 128), Sm::SLAB, 1024);
-                    ptx::umma<KIND_BF16, 1>(tmem_base + COL_U + (u & 1) * D, adesc, bdesc, IDESC_U, k != 0 ? 1u : 0u);
+                    fa2_umma_tmem_a(tmem_base + COL_U + su * D, tmem_base + COL_S0 + su * FA2_BN + k * 8, bdesc, IDESC_U, k != 0 ? 1u : 0u);
                 }
-                ptx::umma_commit(&ctl->pv_done);
-                ptx::umma_commit(&ctl->v_empty[u & 1]);
+                ptx::umma_commit(&ctl->pv_done[su]);
+                ptx::umma_commit(&ctl->v_empty[su]);
+                ptx::umma_commit(&ctl->sp_free[su]);
                 return true;
             };
             for (int t = 0; t < T && ok; ++t) {
                 const int st = t & 1;
                 const uint32_t ph = (t >> 1) & 1;
                 if (!fa2_wait(&ctl->k_full[st], ph, ctl, p.status, 4)) { ok = false; break; }
-                if (!fa2_wait(&ctl->s_empty[st], ph ^ 1, ctl, p.status, 5)) { ok = false; break; }
+                if (!fa2_wait(&ctl->sp_free[st], ph ^ 1, ctl, p.status, 5)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t aK = ptx::smem_u32(sKV + st * Sm::STAGE_BYTES);
 #pragma unroll
@@ -216,7 +244,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         // ------------------------------------------------------------ row threads: two per query row
         constexpr int HD = D / 2;               // d columns of the running output per thread
         constexpr int HN = FA2_BN / 2;          // keys of a tile per thread
-        const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int q = warp & 3;                 // TMEM lane quarter this warp may access
         const int half = (warp - 2) >> 2;       // 0: keys 0-63, d columns 0..HD ; 1: the rest
         const int r = q * 32 + lane;            // row of the query tile
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
@@ -227,7 +255,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         bool ok = true;
         // the two warps that share a lane quarter meet at a named barrier of their own
         auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory"); };
-        // o <- carry o + U_u  (U_u complete in its tensor-memory buffer: pv_done has completed phase u & 1)
+        // o <- carry o + U_u  (U_u complete in its tensor-memory buffer: pv_done[u & 1] has completed its phase)
         auto fold = [&](int u) {
             ptx::tc_fence_after();
 #pragma unroll
@@ -251,87 +279,94 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // this thread's 64 scores: with the short running output (d = 64) they stay in registers from the maximum
             // to the exponentials; with the long one (d = 128) they are read from tensor memory twice, 32 at a time
             constexpr bool KEEP = (D == 64);
-            uint32_t sc[KEEP ? HN : 32];
+            uint32_t sc[HN];  // scores (KEEP) / the packed exponentials in its first half
+            uint32_t tmp[KEEP ? 1 : 32];
             float mx = -INFINITY;
             if (ok) {
                 if constexpr (KEEP) {
                     ptx::tmem_ld_32x32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
-                    ptx::tmem_ld_32x32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[KEEP ? 32 : 0]));
+                    ptx::tmem_ld_32x32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[32]));
                     ptx::tmem_ld_wait();
                     if (valid < HN) {  // only the last tile can be ragged
 #pragma unroll
                         for (int g = 0; g < HN; ++g)
-                            if (g >= valid) sc[KEEP ? g : 0] = 0xff800000u;  // a key that does not exist: -inf, weight 0
+                            if (g >= valid) sc[g] = 0xff800000u;  // a key that does not exist: -inf, weight 0
                     }
 #pragma unroll
-                    for (int g = 0; g < HN; ++g) mx = fmaxf(mx, __uint_as_float(sc[KEEP ? g : 0]));
+                    for (int g = 0; g < HN; ++g) mx = fmaxf(mx, __uint_as_float(sc[g]));
                 } else {
 #pragma unroll 1
                     for (int c0 = 0; c0 < HN; c0 += 32) {
-                        ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+                        ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&tmp[0]));
                         ptx::tmem_ld_wait();
                         if (valid < HN) {
 #pragma unroll
                             for (int g = 0; g < 32; ++g)
-                                if (c0 + g >= valid) sc[g] = 0xff800000u;
+                                if (c0 + g >= valid) tmp[g] = 0xff800000u;
                         }
 #pragma unroll
-                        for (int g = 0; g < 32; ++g) mx = fmaxf(mx, __uint_as_float(sc[g]));
+                        for (int g = 0; g < 32; ++g) mx = fmaxf(mx, __uint_as_float(tmp[g]));
                     }
                 }
             }
             ctl->row_max[st][half][r] = mx;
             pair_sync();
             if (ctl->abort) ok = false;
-            if (!ok) continue;
+            if (!ok) {
+                if constexpr (!KEEP) pair_sync();  // the partner's second barrier of this tile
+                continue;
+            }
             mx = fmaxf(mx, ctl->row_max[st][half ^ 1][r]);
             const float m_new = fmaxf(m, mx * p.scale_log2);
             const float carry = fa2_exp2(m - m_new);  // 2^(-inf) = 0 on the first tile
-            // the previous tile's product must have read P before P is overwritten
-            if (t > 0 && !fa2_wait(&ctl->pv_done, (t - 1) & 1, ctl, p.status, 6)) { ok = false; continue; }
-            // P_t = 2^(S scale - m_new) as bf16 into shared memory (K-major, 128-byte swizzle), row sum in fp32
+            // P_t = 2^(S scale - m_new) as bf16, two keys per 32-bit word (the lower key in the lower half), row sum in fp32
             float lsum = 0.f;
-            uint8_t* slab = sP + half * Sm::SLAB + r * 128;  // this half's 64 keys are one 128-byte row of slab `half`
+            if constexpr (KEEP) {
 #pragma unroll
-            for (int c0 = 0; c0 < HN; c0 += 32) {
-                if constexpr (!KEEP) {
-                    ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+                for (int g = 0; g < HN; g += 2) {
+                    const float p0 = fa2_exp2(fmaf(__uint_as_float(sc[g]), p.scale_log2, -m_new));
+                    const float p1 = fa2_exp2(fmaf(__uint_as_float(sc[g + 1]), p.scale_log2, -m_new));
+                    lsum += p0 + p1;
+                    __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                    sc[g >> 1] = *reinterpret_cast<uint32_t*>(&h);  // word g/2 <= g: nothing still needed is overwritten
+                }
+            } else {
+#pragma unroll
+                for (int c0 = 0; c0 < HN; c0 += 32) {
+                    ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&tmp[0]));
                     ptx::tmem_ld_wait();
                     if (valid < HN) {
 #pragma unroll
                         for (int g = 0; g < 32; ++g)
-                            if (c0 + g >= valid) sc[g] = 0xff800000u;
+                            if (c0 + g >= valid) tmp[g] = 0xff800000u;
                     }
-                }
 #pragma unroll
-                for (int g8 = 0; g8 < 4; ++g8) {  // 16-byte chunk of the row: eight exponentials
-                    uint32_t packed[4];
-#pragma unroll
-                    for (int e = 0; e < 8; e += 2) {
-                        const int at = (KEEP ? c0 : 0) + 8 * g8 + e;
-                        const float p0 = fa2_exp2(fmaf(__uint_as_float(sc[at]), p.scale_log2, -m_new));
-                        const float p1 = fa2_exp2(fmaf(__uint_as_float(sc[at + 1]), p.scale_log2, -m_new));
+                    for (int g = 0; g < 32; g += 2) {
+                        const float p0 = fa2_exp2(fmaf(__uint_as_float(tmp[g]), p.scale_log2, -m_new));
+                        const float p1 = fa2_exp2(fmaf(__uint_as_float(tmp[g + 1]), p.scale_log2, -m_new));
                         lsum += p0 + p1;
                         __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                        packed[e >> 1] = *reinterpret_cast<uint32_t*>(&h);
+                        sc[(c0 + g) >> 1] = *reinterpret_cast<uint32_t*>(&h);
                     }
-                    *reinterpret_cast<uint4*>(slab + ((((c0 >> 3) + g8) ^ (r & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                 }
+                pair_sync();  // both threads of the row have read their scores a second time: the columns may be overwritten
             }
             l = fmaf(l, carry, lsum);
             m = m_new;
+            // over the first 64 columns of the buffer the scores came in: keys 64 half .. + 63 are columns 32 half .. + 31
+            fa2_tmem_st_32x32(lane_addr + COL_S0 + st * FA2_BN + half * (HN / 2), *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
+            fa2_tmem_st_wait();
             ptx::tc_fence_before();
-            ptx::fence_proxy_async_smem();  // the MMA reads P through the async proxy
             __syncwarp();
-            if (lane == 0) {
-                ptx::mbar_arrive(&ctl->p_ready);
-                ptx::mbar_arrive(&ctl->s_empty[st]);
-            }
+            if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[st]);
             // with P_t handed over, fold the previous tile's product (in the other U buffer) into the running output
-            if (t > 0) fold(t - 1);
+            if (t > 0) {
+                if (!fa2_wait(&ctl->pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1, ctl, p.status, 6)) { ok = false; continue; }
+                fold(t - 1);
+            }
             carry_prev = carry;
         }
-        if (ok) ok = fa2_wait(&ctl->pv_done, (T - 1) & 1, ctl, p.status, 10);
+        if (ok) ok = fa2_wait(&ctl->pv_done[(T - 1) & 1], ((T - 1) >> 1) & 1, ctl, p.status, 10);
         if (ok) fold(T - 1);
         // the normaliser of a row is the sum of its two partial ones
         ctl->row_sum[half][r] = l;
