@@ -37,3 +37,41 @@ def test_many_launches_stay_clean_and_identical(case):
     assert binding.last_device_status() == binding.CYC_OK, binding.cyc_last_cuda_error()
     for o in outs:
         assert torch.equal(o, first)
+
+
+def test_many_scan_launches_stay_clean_and_identical():
+    """The look-back of the prefix-sum kernel is the one place where CTAs of a launch wait for one another: thousands of
+    launches on long and short chains must leave the status word clean; int32 results are identical every time."""
+    import torch
+    from paper_2511_09987_b200 import binding
+    for rows, n, launches in ((1, 1 << 22, 1500), (64, 70001, 1500), (4096, 4096, 500)):
+        A = torch.from_numpy(inputs.make_scan_operand(inputs.ScanWorkload("s", rows, n, "i32", 91))).cuda()
+        outs = [binding.prefix_sum(A) for _ in range(3)]
+        first = outs[0].clone()
+        for i in range(launches):
+            binding.prefix_sum(A, outs[i % 3])
+        assert binding.last_device_status() == binding.CYC_OK, binding.cyc_last_cuda_error()
+        for o in outs:
+            assert torch.equal(o, first)
+
+
+def test_many_attention_and_cholesky_launches_stay_clean_and_identical():
+    import torch
+    from paper_2511_09987_b200 import binding
+    Q, K, V = (torch.from_numpy(x).view(torch.bfloat16).cuda()
+               for x in inputs.make_attention_operands(inputs.AttentionWorkload("s", 8, 1000, 1500, 128, seed=92)))
+    outs = [binding.flash_attention(Q, K, V) for _ in range(3)]
+    first = outs[0].clone()
+    for i in range(1500):
+        binding.flash_attention(Q, K, V, outs[i % 3])
+    assert binding.last_device_status() == binding.CYC_OK, binding.cyc_last_cuda_error()
+    for o in outs:
+        assert torch.equal(o, first)
+    A = torch.from_numpy(inputs.make_chol_operand(inputs.CholWorkload("s", 1100, 256, 93))).cuda()
+    outs = [binding.cholesky(A) for _ in range(3)]
+    first = outs[0].clone()
+    for i in range(100):
+        binding.cholesky(A, outs[i % 3])
+    assert binding.last_device_status() == binding.CYC_OK, binding.cyc_last_cuda_error()
+    for o in outs:
+        assert torch.equal(o, first)
