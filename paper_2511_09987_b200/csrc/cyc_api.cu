@@ -962,33 +962,49 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
         int rc = workspace_pool(&pool);
         if (rc) return rc;
         void* ws = nullptr;
-        CYC_CUDA(cudaMallocFromPoolAsync(&ws, static_cast<size_t>(CHOL_MAX_SLICES + 1) * plane * sizeof(float), pool, st));
+        CYC_CUDA(cudaMallocFromPoolAsync(&ws, static_cast<size_t>(CHOL_MAX_SLICES + 1) * (plane + 4) * sizeof(float), pool, st));
         W = static_cast<float*>(ws);
     }
     int rc = CYC_OK;
     for (long long c0 = 0; c0 < n && rc == CYC_OK; c0 += T) {
         const long long c1 = std::min<long long>(n, c0 + T), w = c1 - c0, below = n - c1;
         int planes = 0;
+        // this panel's planes lie back to back, each (n - c0) x w floats rounded up to a multiple of four
+        const long long pstride = ((n - c0) * w + 3) / 4 * 4;
         if (c0 > 0) {
             const long long kblocks = c0 / T, tiles_m = (n - c0 + 255) / 256;
             long long S = std::min<long long>({static_cast<long long>(CHOL_MAX_SLICES), kblocks, std::max<long long>(1, kCtaPairs / tiles_m)});
             const long long kc = (kblocks / S) * T, rem = c0 - S * kc;
             const unsigned gflags = (flags & CYC_FLAG_FIXED_K_ORDER) | CYC_FLAG_B_COL_MAJOR;
-            Problem q{S, n - c0, w, kc, CYC_F32, Lf + c0 * n, Lf + c0 * n, W, kc, kc, plane, gflags, n, n};
+            Problem q{S, n - c0, w, kc, CYC_F32, Lf + c0 * n, Lf + c0 * n, W, kc, kc, pstride, gflags, n, n};
             rc = route(q, st);
             if (rc) break;
             planes = static_cast<int>(S);
             if (rem > 0) {
-                Problem r{1, n - c0, w, rem, CYC_F32, Lf + c0 * n + S * kc, Lf + c0 * n + S * kc, W + S * plane, (n - c0) * n, w * n, plane,
+                Problem r{1, n - c0, w, rem, CYC_F32, Lf + c0 * n + S * kc, Lf + c0 * n + S * kc, W + S * pstride, (n - c0) * n, w * n, pstride,
                           gflags, n, n};
                 rc = route(r, st);
                 if (rc) break;
                 ++planes;
             }
+            if (planes > 1) {
+                // the slices' partial sums added in increasing k into the first plane, by all SMs at once, so that the
+                // two consumers (one CTA for the diagonal tile, few CTAs per solve) read a single plane
+                DeviceInfo di;
+                rc = device_info(&di);
+                if (rc) break;
+                const long long work = pstride / 4;
+                long long blocks = std::min<long long>((work + 127) / 128, 16ll * di.sms);
+                splitk_reduce_kernel<float><<<static_cast<unsigned>(blocks), 128, 0, st>>>(W, W, pstride, pstride, planes, 1, 1);
+                cudaError_t e = cudaGetLastError();
+                if (e != cudaSuccess) { rc = cuda_fail(e, "splitk_reduce_kernel"); break; }
+                g_launches.fetch_add(1);
+                planes = 1;
+            }
         }
         CholDiagParams d;
         d.A = Af + c0 * n + c0; d.W = W; d.L = Lf + c0 * n + c0;
-        d.plane = plane; d.planes = planes;
+        d.plane = pstride; d.planes = planes;
         d.lda = n; d.ldw = w; d.ldl = n;
         d.rows = static_cast<int>(w);
         d.zero_upper = in_place ? 0 : 1;
@@ -1000,7 +1016,7 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
             TrsmDiagParams p;
             p.L = Lf;
             p.B = Af + c1 * n + c0; p.X = Lf + c1 * n + c0; p.W = planes ? W + w * w : nullptr;
-            p.plane = plane;
+            p.plane = pstride;
             p.b_r = 1; p.b_c = n; p.x_r = 1; p.x_c = n; p.w_r = 1; p.w_c = w;
             p.n = static_cast<int>(n); p.m = static_cast<int>(below);
             p.r0 = static_cast<int>(c0); p.rows = static_cast<int>(w);
