@@ -55,7 +55,10 @@ CASES = [SW("one", 1, 1, "f32", 60), SW("one_i", 1, 1, "i32", 61), SW("three", 1
          SW("tile_plus_quarter", 3, 16384 + 4096, "f32", 77),
          SW("p1", 3, 10000, "f32", 30), SW("odd_rows", 7, 4099, "i32", 67), SW("short_rows", 500, 37, "f32", 68),
          SW("many_tiles", 1, 40 * 16384 + 13, "f32", 69), SW("many_tiles_i", 2, 70 * 16384 + 4097, "i32", 70),
-         SW("long_lookback", 1, 3000 * 4096 + 5, "f32", 71)]
+         SW("long_lookback", 1, 3000 * 4096 + 5, "f32", 71),
+         # long rows: hundreds of tiles per row, several rows
+         SW("long_row_exact", 1, 1 << 22, "i32", 78), SW("long_rows_ragged", 3, (1 << 22) + 12345, "f32", 79),
+         SW("long_row_two_sections", 1, 6_000_000 + 3, "i32", 94), SW("long_row_three_sections", 2, 11_000_000 + 1, "f32", 95)]
 
 
 @pytest.mark.parametrize("w", CASES, ids=[c.name for c in CASES])
@@ -75,6 +78,12 @@ def test_in_place_unaligned_and_pitched(dtype):
     flat = torch.from_numpy(A.reshape(-1)).cuda()
     P = binding.prefix_sum(flat[1:])                     # base pointer off the 16-byte grid
     check(P.cpu().numpy()[None, :], A.reshape(1, -1)[:, 1:])
+
+
+def test_long_rows_in_place_and_pitched():
+    A = inputs.make_scan_operand(SW("x", 2, (1 << 22) + 77, "f32", 96))
+    check(gpu_scan(A, in_place=True), A)
+    check(gpu_scan(A, pitch=(1 << 22) + 79), A)          # rows not 16-byte aligned: the scalar path
 
 
 def test_closed_forms_and_exact_cases():
