@@ -207,15 +207,15 @@ int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t d, int dtyp
  *          CYC_ERR_INVALID_ARG.
  *   strideA, strideP   in elements, >= n; 0 means n (sequences back to back)
  *   dtype  CYC_F32: sums of neighbouring elements are formed in fp32 inside runs of 128
- *          elements, everything carried further (across a tile of 16384 elements and from
+ *          elements, everything carried further (across a tile of 16384 or 8192 elements and from
  *          tile to tile) is fp64: |P_i - exact| <= 1e-6 * sum_{k<=i} |A_k|, independent of n.  The order in
  *          which tile sums are combined follows their arrival, so the last bit of a result may
  *          differ between runs.
  *          CYC_I32: two's-complement 32-bit integers, wrap-around on overflow; exact and
  *          run-to-run identical.  Other types are refused with CYC_ERR_UNSUPPORTED.
  *   flags  0
- * rows, n >= 1; rows * ceil(n / 16384) < 2^31.  One pass over the data (each element read once,
- * written once) in a single kernel; the tile descriptors (8 bytes per 16384 elements) come from
+ * rows, n >= 1; rows * ceil(n / 8192) < 2^31.  One pass over the data (each element read once,
+ * written once) in a single kernel; the tile descriptors (8 bytes per tile of 16384 elements, 8192 for rows of at most 262144 elements) come from
  * the library's stream-ordered pool for the duration of the call.  Asynchronous on `stream`;
  * the caller owns A and P; errors as for cyc_recurrence_matmul.
  */

@@ -872,19 +872,25 @@ extern "C" int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t 
                    : launch_fa2<128>(batch, N, M, Q, K, V, static_cast<float*>(O), st);
 }
 
-template <typename T>
+// tile of SUBS * 4096 elements: 16384 for long rows (the running value of one chain advances by at most 32 tiles per
+// descriptor round trip), 8192 when a row has at most 32 such tiles (its look-back never leaves one window; half the
+// shared memory per CTA, twice the CTAs per SM)
+static int scan_subs(long long n) { return (n + SCAN_SUBS_SHORT * SCAN_SUB - 1) / (SCAN_SUBS_SHORT * SCAN_SUB) <= SCAN_WINDOW ? SCAN_SUBS_SHORT : SCAN_SUBS; }
+
+template <typename T, int SUBS>
 static int launch_scan(long long rows, long long n, const void* A, long long sA, void* P, long long sP, cudaStream_t st) {
+    constexpr long long TILE = static_cast<long long>(SUBS) * SCAN_SUB;
     ScanParams<T> p;
     p.A = static_cast<const T*>(A);
     p.P = static_cast<T*>(P);
     p.n = n; p.strideA = sA; p.strideP = sP;
-    p.tiles_per_row = (n + SCAN_TILE - 1) / SCAN_TILE;
+    p.tiles_per_row = (n + TILE - 1) / TILE;
     const long long tiles = rows * p.tiles_per_row;
     p.total_tiles = tiles;
     p.vec_ok = (reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(P) % 16 == 0 && (rows == 1 || (sA % 4 == 0 && sP % 4 == 0)))
                    ? 1 : 0;
     CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
-    CYC_CUDA(cudaFuncSetAttribute(scan_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_BYTES));
+    CYC_CUDA(cudaFuncSetAttribute(scan_kernel<T, SUBS>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(TILE * sizeof(T)) + 128));
     cudaMemPool_t pool;
     int rc = workspace_pool(&pool);
     if (rc) return rc;
@@ -896,8 +902,8 @@ static int launch_scan(long long rows, long long n, const void* A, long long sA,
     cudaError_t e = cudaMemsetAsync(ws, 0, bytes, st);  // counter, abort flag and every descriptor start at zero
     if (e == cudaSuccess) {
         // short rows need only their own quarters of the staging buffer: more CTAs fit an SM
-        const int quarters = static_cast<int>(std::min<long long>(SCAN_SUBS, (n + SCAN_SUB - 1) / SCAN_SUB));
-        scan_kernel<T><<<static_cast<unsigned>(tiles), SCAN_THREADS, quarters * SCAN_SUB * sizeof(T) + 128, st>>>(p);
+        const int quarters = static_cast<int>(std::min<long long>(SUBS, (n + SCAN_SUB - 1) / SCAN_SUB));
+        scan_kernel<T, SUBS><<<static_cast<unsigned>(tiles), SCAN_THREADS, quarters * SCAN_SUB * sizeof(T) + 128, st>>>(p);
         e = cudaGetLastError();
         if (e == cudaSuccess) g_launches.fetch_add(1);
     }
@@ -923,10 +929,13 @@ extern "C" int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A,
         snprintf(g_err, sizeof g_err, "prefix sum: fp32 or int32 only");
         return CYC_ERR_UNSUPPORTED;
     }
-    const long long tiles_per_row = (n + SCAN_TILE - 1) / SCAN_TILE;
+    const int subs = scan_subs(n);
+    const long long tiles_per_row = (n + subs * SCAN_SUB - 1) / (subs * SCAN_SUB);
     if (tiles_per_row > 0x7fffffffll / rows) return CYC_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return dtype == CYC_F32 ? launch_scan<float>(rows, n, A, sA, P, sP, st) : launch_scan<int>(rows, n, A, sA, P, sP, st);
+    if (subs == SCAN_SUBS_SHORT)
+        return dtype == CYC_F32 ? launch_scan<float, SCAN_SUBS_SHORT>(rows, n, A, sA, P, sP, st) : launch_scan<int, SCAN_SUBS_SHORT>(rows, n, A, sA, P, sP, st);
+    return dtype == CYC_F32 ? launch_scan<float, SCAN_SUBS>(rows, n, A, sA, P, sP, st) : launch_scan<int, SCAN_SUBS>(rows, n, A, sA, P, sP, st);
 }
 
 // ------------------------------------------------------------------ tiled Cholesky

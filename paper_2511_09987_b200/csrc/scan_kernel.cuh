@@ -24,7 +24,8 @@
 namespace cyc {
 
 constexpr int SCAN_THREADS = 256, SCAN_CHUNKS = 4, SCAN_SUB = SCAN_THREADS * SCAN_CHUNKS * 4;  // 4096 elements per quarter
-constexpr int SCAN_SUBS = 4, SCAN_TILE = SCAN_SUBS * SCAN_SUB;                                     // 16384 elements per tile
+constexpr int SCAN_SUBS = 4, SCAN_TILE = SCAN_SUBS * SCAN_SUB;                                     // 16384 elements per tile (long rows)
+constexpr int SCAN_SUBS_SHORT = 2;  // 8192-element tiles for rows of at most SCAN_WINDOW such tiles: twice the CTAs per SM
 constexpr int SCAN_WARPS = SCAN_THREADS / 32;
 constexpr int SCAN_SMEM_BYTES = SCAN_TILE * 4 + 128;
 constexpr int SCAN_WINDOW = 32;  // predecessors examined per round of the look-back (128 measured slower: 3.6 against 4.0 TB/s)
@@ -99,14 +100,14 @@ __device__ __forceinline__ void scan_bulk_load(void* smem_dst, const void* gmem_
                  : "memory");
 }
 
-template <typename T>
+template <typename T, int SUBS>
 __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const ScanParams<T> p) {
     using Carry = typename ScanCarry<T>::type;
     using V4 = typename std::conditional<std::is_same<T, float>::value, float4, int4>::type;
-    constexpr int ENTRIES = SCAN_SUBS * SCAN_CHUNKS * SCAN_WARPS;  // warp-level sums of a tile, in element order
+    constexpr int ENTRIES = SUBS * SCAN_CHUNKS * SCAN_WARPS;  // warp-level sums of a tile, in element order
     extern __shared__ uint8_t scan_smem_raw[];
     T* buf = reinterpret_cast<T*>((reinterpret_cast<uintptr_t>(scan_smem_raw) + 127) & ~static_cast<uintptr_t>(127));
-    __shared__ uint64_t s_bar[SCAN_SUBS];
+    __shared__ uint64_t s_bar[SUBS];
     __shared__ unsigned int s_tile;
     __shared__ T s_total[ENTRIES];
     __shared__ Carry s_offset[ENTRIES];
@@ -116,7 +117,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const ScanParams<T> 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
 #pragma unroll
-        for (int s = 0; s < SCAN_SUBS; ++s) ptx::mbar_init(&s_bar[s], 1);
+        for (int s = 0; s < SUBS; ++s) ptx::mbar_init(&s_bar[s], 1);
         ptx::fence_mbar_init();
         s_abort = 0;
         const unsigned int t = atomicAdd(&p.header->next_tile, 1u);
@@ -124,10 +125,10 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const ScanParams<T> 
         // quarters that lie completely inside the row come by bulk copy; a ragged or unaligned quarter is read by the threads
         if (p.vec_ok) {
             const long long row = t / p.tiles_per_row, tr = t - row * p.tiles_per_row;
-            const long long base = tr * SCAN_TILE;
+            const long long base = tr * (SUBS * SCAN_SUB);
             const T* a = p.A + row * p.strideA + base;
 #pragma unroll
-            for (int s = 0; s < SCAN_SUBS; ++s)
+            for (int s = 0; s < SUBS; ++s)
                 if (base + (s + 1) * SCAN_SUB <= p.n) {
                     ptx::mbar_arrive_expect_tx(&s_bar[s], SCAN_SUB * sizeof(T));
                     scan_bulk_load(buf + s * SCAN_SUB, a + s * SCAN_SUB, SCAN_SUB * sizeof(T), &s_bar[s]);
@@ -137,8 +138,8 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const ScanParams<T> 
     __syncthreads();
     const long long tile = s_tile;
     const long long row = tile / p.tiles_per_row, tr = tile - row * p.tiles_per_row;
-    const long long base = tr * SCAN_TILE;
-    const int len = static_cast<int>(min(static_cast<long long>(SCAN_TILE), p.n - base));
+    const long long base = tr * (SUBS * SCAN_SUB);
+    const int len = static_cast<int>(min(static_cast<long long>((SUBS * SCAN_SUB)), p.n - base));
     const int subs = (len + SCAN_SUB - 1) / SCAN_SUB;
     const T* a = p.A + row * p.strideA + base;
     T* out = p.P + row * p.strideP + base;
@@ -281,7 +282,7 @@ __global__ void __launch_bounds__(SCAN_THREADS) scan_kernel(const ScanParams<T> 
     if (s_abort) {
         // leave no copy in flight: wait (bounded) for the quarters that were requested
         if (tid == 0 && p.vec_ok)
-            for (int s = 0; s < SCAN_SUBS; ++s)
+            for (int s = 0; s < SUBS; ++s)
                 if (base + (s + 1) * SCAN_SUB <= p.n) {
                     const long long t0 = clock64();
                     while (!ptx::mbar_try_wait(&s_bar[s], 0) && clock64() - t0 < SCAN_WAIT_CYCLES) {}
