@@ -277,7 +277,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const uint32_t s_addr = lane_addr + COL_S0 + st * FA2_BN + half * HN;
             const int valid = min(FA2_BN, p.M - t * FA2_BN) - half * HN;  // keys of this thread's half that exist
             // this thread's 64 scores: with the short running output (d = 64) they stay in registers from the maximum
-            // to the exponentials; with the long one (d = 128) they are read from tensor memory twice, 32 at a time
+            // to the exponentials; with the long one (d = 128) they pass through 32 registers, the first 32 read twice
             constexpr bool KEEP = (D == 64);
             uint32_t sc[HN];  // scores (KEEP) / the packed exponentials in its first half
             uint32_t tmp[KEEP ? 1 : 32];
@@ -331,14 +331,18 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     sc[g >> 1] = *reinterpret_cast<uint32_t*>(&h);  // word g/2 <= g: nothing still needed is overwritten
                 }
             } else {
+                // the scores of keys 32-63 are still in `tmp` from the pass for the maximum: they go first, and only
+                // keys 0-31 are read from tensor memory a second time
 #pragma unroll
-                for (int c0 = 0; c0 < HN; c0 += 32) {
-                    ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&tmp[0]));
-                    ptx::tmem_ld_wait();
-                    if (valid < HN) {
+                for (int c0 = HN - 32; c0 >= 0; c0 -= 32) {
+                    if (c0 != HN - 32) {
+                        ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&tmp[0]));
+                        ptx::tmem_ld_wait();
+                        if (valid < HN) {
 #pragma unroll
-                        for (int g = 0; g < 32; ++g)
-                            if (c0 + g >= valid) tmp[g] = 0xff800000u;
+                            for (int g = 0; g < 32; ++g)
+                                if (c0 + g >= valid) tmp[g] = 0xff800000u;
+                        }
                     }
 #pragma unroll
                     for (int g = 0; g < 32; g += 2) {
