@@ -312,10 +312,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ctl->row_max[st][half][r] = mx;
             pair_sync();
             if (ctl->abort) ok = false;
-            if (!ok) {
-                if constexpr (!KEEP) pair_sync();  // the partner's second barrier of this tile
-                continue;
-            }
+            if (!ok) continue;
             mx = fmaxf(mx, ctl->row_max[st][half ^ 1][r]);
             const float m_new = fmaxf(m, mx * p.scale_log2);
             const float carry = fa2_exp2(m - m_new);  // 2^(-inf) = 0 on the first tile
@@ -353,7 +350,9 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         sc[(c0 + g) >> 1] = *reinterpret_cast<uint32_t*>(&h);
                     }
                 }
-                pair_sync();  // both threads of the row have read their scores a second time: the columns may be overwritten
+                // No second barrier: P goes to columns 0-63 of the buffer.  Columns 32-63 held this row's scores of
+                // keys 32-63, which their owner (half 0) took from registers above; the scores read a second time sit
+                // in columns 0-31 (half 0, overwritten only by its own store below) and 64-95 (half 1, never overwritten).
             }
             l = fmaf(l, carry, lsum);
             m = m_new;
