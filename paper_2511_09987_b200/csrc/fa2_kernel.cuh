@@ -295,7 +295,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                     for (int g = 0; g < HN; ++g) mx = fmaxf(mx, __uint_as_float(sc[g]));
                 } else {
-#pragma unroll 1
+#pragma unroll
                     for (int c0 = 0; c0 < HN; c0 += 32) {
                         ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&tmp[0]));
                         ptx::tmem_ld_wait();
