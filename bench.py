@@ -3,8 +3,10 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
 
-Workloads c1..c5 are the matrix-multiply recurrence (the default, c2, is the headline); t1 and t2 are the block
-lower-triangular solve built on it; a1 and a2 are the FlashAttention-2 recurrence; p1..p3 the prefix-sum recurrence; h1 and h2 the tiled Cholesky recurrence.
+Workloads c1..c5 are the matrix-multiply recurrence.  With no --workload the largest configuration that fits one GPU
+(c3) is the headline and the line carries a `configs` object with the same record for c1, c2, c4 and c5 (each timed over
+at least a quarter of a second of back-to-back steps) and `sustained` sub-records (at least one second) for c2 and c3.
+t1 and t2 are the block lower-triangular solve built on the recurrence; a1 and a2 are the FlashAttention-2 recurrence; p1..p3 the prefix-sum recurrence; h1 and h2 the tiled Cholesky recurrence.
 
 One step = one evaluation of the whole recurrence (weight load, B injection, the
 multiply-accumulate chain along k, export of C) for one workload.  Prints ONE JSON
@@ -32,6 +34,9 @@ from paper_2511_09987_b200 import inputs  # noqa: E402
 
 # nominal dense tensor ratios relative to bf16 (2.25 PFLOP/s): int8 4.5 POPS, tf32 1.1 PFLOP/s
 NOMINAL_RATIO = {"bf16": 1.0, "i8": 2.0, "tf32": 0.5}
+# datasheet dense peaks (TFLOP/s or TOPS), reported beside the measured ones as `frac_nominal`
+NOMINAL_PEAK = {"bf16": 2250.0, "i8": 4500.0, "tf32": 1100.0}
+NOMINAL_HBM_GBS = 7700.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 L2_BYTES = 126 * 1024 * 1024
 # FP32 FMA roof: 148 SMs x 128 lanes x 2 flop x max SM clock
@@ -51,20 +56,37 @@ def unit_of(w):
     return "TOPS" if w.dtype == "i8" else "TFLOPS"
 
 
-def bound_of(w, family):
-    """Which roof bounds the dominant kernel of this workload."""
+def tensor_kind(w):
+    return "tf32" if w.dtype == "f32" else w.dtype
+
+
+def bound_of(w, family, peaks):
+    """Which roof bounds the dominant kernel of this workload: the ridge is the measured tensor rate of the dtype
+    (bf16 cuBLAS burst x the nominal ratio of the dtype) over the measured copy bandwidth."""
     if family == "simt":
         return "alu"
     ai = 2.0 * w.macs / w.algorithmic_bytes
-    ridge = {"bf16": 1663e12 / 6.55e12, "i8": 3326e12 / 6.55e12, "f32": 830e12 / 6.55e12}[w.dtype]
+    ridge = float(peaks["bf16_tflops"]) * NOMINAL_RATIO[tensor_kind(w)] * 1e12 / (float(peaks["hbm_gbs"]) * 1e9)
     return "tensor" if ai > ridge else "hbm"
+
+
+def tensor_roofline(achieved, kind, peaks, peak_kind):
+    """Fractions of one tensor-bound figure: against the measured burst peak (`frac`, the denominator never depends on
+    how long the timed region was), the measured sustained peak and the datasheet dense peak of the dtype."""
+    burst = float(peaks["bf16_tflops"]) * NOMINAL_RATIO[kind]
+    sustained = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * NOMINAL_RATIO[kind]
+    return {"peak": burst, "frac": achieved / burst, "frac_measured": achieved / burst,
+            "frac_measured_sustained": achieved / sustained, "peak_sustained": sustained,
+            "frac_nominal": achieved / NOMINAL_PEAK[kind], "peak_nominal": NOMINAL_PEAK[kind],
+            "peak_source": "%s bf16 cuBLAS burst x nominal %s/bf16 ratio %.1f (of %s); frac_measured_sustained uses the "
+                           "seconds-long cuBLAS loop, frac_nominal the datasheet dense peak" % (peak_kind, kind, NOMINAL_RATIO[kind], peak_kind)}
 
 
 class ClockSampler:
     """Polls SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
-    def __init__(self, index: int):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+    def __init__(self, index: int, period: float = 0.004):
+        self.samples, self.reasons, self.max_mhz, self.period = [], set(), None, period
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -96,7 +118,7 @@ class ClockSampler:
                         self.reasons.add(n)
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(self.period)
 
     def start(self):
         if self.nv is not None:
@@ -192,23 +214,31 @@ def describe(w):
     return s
 
 
-def run_ours(args, w):
+def cuda_setup():
     import torch
-    from paper_2511_09987_b200 import binding
     from paper_2511_09987_b200.replicas import Replicas
-
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
     reps = Replicas("nccl", torch.device("cuda", local))
-    world, rank = reps.world, reps.rank
+    return torch, reps, local
+
+
+def measure_matmul(w, steps, args, torch, reps, local, *, min_seconds=0.0, sustained_seconds=0.0, cpu_seconds=12.0,
+                   with_cpu=True, with_e2e=True):
+    """One record for the matrix-multiply recurrence on workload `w`.
+
+    The timed region is `steps` back-to-back steps (one library call each); when `min_seconds` is given and `steps` is
+    None, the number of steps is chosen from a short calibration so that the region lasts at least that long.  Clocks
+    are sampled by NVML inside the region.  `sustained_seconds` adds a second, longer region of its own."""
+    from paper_2511_09987_b200 import binding
+    world = reps.world
     peaks, peak_kind = load_peaks()
 
-    # ---- operands: generated once on the host, uploaded; several device copies rotate so that
-    # ---- a set has left L2 before it is used again
+    # ---- operands: generated once on the host, uploaded; several device copies rotate so that a set has left L2
+    # ---- before it is used again
     A, B = inputs.make_operands(w)
-    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i8": torch.int8}[w.dtype]
     hA = torch.from_numpy(A)
     hB = torch.from_numpy(B)
     if w.dtype == "bf16":
@@ -220,6 +250,7 @@ def run_ours(args, w):
     nsets = int(min(8, max(2, -(-3 * L2_BYTES // set_bytes))))
     sets = [(hA.cuda(), hB.cuda(), torch.empty(cshape, dtype=out_dt, device="cuda")) for _ in range(nsets)]
     stream = torch.cuda.current_stream()
+    ops_step = 2.0 * w.macs
 
     def step(i):
         dA, dB, dC = sets[i % nsets]
@@ -235,15 +266,35 @@ def run_ours(args, w):
         reps.barrier()
         torch.cuda.synchronize()
 
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def region(n, replay=None):
+        """n steps between two events on the launching stream, a barrier and a synchronize on both sides."""
+        barrier()
+        e0.record(stream)
+        if replay is not None:
+            for _ in range(n // replay[1]):
+                replay[0].replay()
+        else:
+            for i in range(n):
+                step(i)
+        e1.record(stream)
+        barrier()
+        return e0.elapsed_time(e1)
+
     for i in range(max(3, args.warmup)):
         step(i)
     barrier()
+    if steps is None:  # calibrate: as many steps as fill `min_seconds`
+        est = region(20) / 20.0
+        steps = int(max(20, min(200000, -(-min_seconds * 1e3 // max(est, 1e-4)))))
     # launch-bound workloads (a few microseconds per kernel): replay the steps from a CUDA graph so that the
     # device, not the Python launch path, is what is timed.  The graph holds `chunk` launches; K steps = K/chunk replays.
-    graph, chunk = None, 1
-    if args.graph == "on" or (args.graph == "auto" and 2.0 * w.macs < 5e7):
-        chunk = max(1, min(100, args.steps))
-        while args.steps % chunk:
+    graph, chunk, plain_call_us = None, 1, None
+    if args.graph == "on" or (args.graph == "auto" and ops_step < 5e7):
+        plain_call_us = region(min(steps, 2000)) / min(steps, 2000) * 1e3   # the same steps as plain library calls
+        chunk = max(1, min(100, steps))
+        while steps % chunk:
             chunk -= 1
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
@@ -260,25 +311,14 @@ def run_ours(args, w):
     sampler = ClockSampler(local)
     sampler.start()
     launches0 = binding.cyc_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record(stream)
-    if graph is not None:
-        for _ in range(args.steps // chunk):
-            graph.replay()
-    else:
-        for i in range(args.steps):
-            step(i)
-    e1.record(stream)
-    barrier()
-    ms = e0.elapsed_time(e1)
-    launches = args.steps if graph is not None else binding.cyc_launch_count() - launches0
+    ms = region(steps, (graph, chunk) if graph is not None else None)
+    launches = steps if graph is not None else binding.cyc_launch_count() - launches0
     if binding.last_device_status() != binding.CYC_OK:
         raise SystemExit("a device-side wait timed out during the benchmark: " + binding.cyc_last_cuda_error().decode())
     # keep the GPU loaded a little longer if the timed region was too short to catch a clock sample
     extra_note = None
     if len(sampler.samples) < 3:
-        t_end = time.time() + 0.5
+        t_end = time.time() + 0.3
         i = 0
         while time.time() < t_end:
             step(i)
@@ -286,80 +326,125 @@ def run_ours(args, w):
             if i % 64 == 0:
                 torch.cuda.synchronize()
         torch.cuda.synchronize()
-        extra_note = "timed region shorter than the sampling period; clocks sampled under the same load right after it"
+        extra_note = "timed region shorter than three sampling periods; clocks sampled under the same load right after it"
     clocks = sampler.stop()
     if extra_note:
         clocks["note"] = extra_note
 
     ms = reps.max_over_ranks(ms)
-    ms_per_step = ms / args.steps
-    ops_step = 2.0 * w.macs
+    ms_per_step = ms / steps
     value = world * ops_step / (ms_per_step * 1e-3) / 1e12
 
-    # ---- end to end through the host entry point (pinned buffers, copies inside the timed region)
-    hC = torch.empty(cshape, dtype=out_dt).pin_memory()
-    e2e_steps = 0 if args.kernel_only else max(3, min(args.steps, 20))
-    for _ in range(0 if args.kernel_only else 2):
-        binding.recurrence_matmul_host(hA, hB, hC, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
-    barrier()
-    t0 = time.perf_counter()
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        binding.recurrence_matmul_host(hA, hB, hC, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
-    e1.record(stream)
-    barrier()
-    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / max(1, e2e_steps)
-    e2e_value = world * ops_step / (reps.max_over_ranks(e2e_ms) * 1e-3) / 1e12
+    # ---- a second, seconds-long region: what the kernel sustains under the power cap
+    sustained = None
+    if sustained_seconds > 0:
+        n = int(max(steps, -(-sustained_seconds * 1e3 // ms_per_step)))
+        s2 = ClockSampler(local)
+        s2.start()
+        ms2 = reps.max_over_ranks(region(n))
+        c2 = s2.stop()
+        v2 = ops_step / (ms2 / n * 1e-3) / 1e12
+        sustained = {"value": world * v2, "unit": unit_of(w), "steps": n, "seconds": ms2 * 1e-3, "ms_per_step": ms2 / n, "clocks": c2}
 
-    if rank != 0:
-        reps.close()
-        return
+    # ---- end to end through the host entry point (pinned buffers, copies inside the timed region)
+    e2e = None
+    if with_e2e:
+        hC = torch.empty(cshape, dtype=out_dt).pin_memory()
+        e2e_steps = max(3, min(steps, 20))
+        for _ in range(2):
+            binding.recurrence_matmul_host(hA, hB, hC, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
+        barrier()
+        t0 = time.perf_counter()
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            binding.recurrence_matmul_host(hA, hB, hC, b_col_major=w.b_col_major, fixed_k_order=w.fixed_k_order)
+        e1.record(stream)
+        barrier()
+        e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / e2e_steps
+        e2e = {"value": world * ops_step / (reps.max_over_ranks(e2e_ms) * 1e-3) / 1e12, "unit": unit_of(w),
+               "h2d_bytes_per_step": int(hA.numel() * hA.element_size() + hB.numel() * hB.element_size()),
+               "d2h_bytes_per_step": int(hC.numel() * hC.element_size()), "steps": e2e_steps, "ms_per_step": e2e_ms}
+        del hC
+    else:
+        e2e = {"value": None, "unit": unit_of(w), "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "steps": 0}
+    del sets, graph
+    torch.cuda.empty_cache()
 
     # ---- roofline of the dominant (only) kernel: one launch per step
     kernel_s = ms_per_step * 1e-3
-    bound = bound_of(w, family)
+    bound = bound_of(w, family, peaks)
     traffic = load_traffic(w, family)
     if bound == "hbm":
-        achieved, peak, runit = w.algorithmic_bytes / kernel_s / 1e9, float(peaks["hbm_gbs"]), "GB/s"
-        peak_note = "%s STREAM-style copy" % peak_kind
+        achieved, runit = w.algorithmic_bytes / kernel_s / 1e9, "GB/s"
+        peak = float(peaks["hbm_gbs"])
+        fr = {"peak": peak, "frac": achieved / peak, "frac_measured": achieved / peak, "frac_nominal": achieved / NOMINAL_HBM_GBS,
+              "peak_nominal": NOMINAL_HBM_GBS, "peak_source": "%s STREAM-style copy (of %s); frac_nominal against 7.7 TB/s" % (peak_kind, peak_kind)}
     elif bound == "tensor":
-        base = float(peaks["bf16_tflops"]) if args.steps * kernel_s < 1.0 else float(peaks["bf16_tflops_sustained"])
-        which = "burst" if args.steps * kernel_s < 1.0 else "sustained"
-        kind = "tf32" if w.dtype == "f32" else w.dtype
-        achieved, peak, runit = ops_step / kernel_s / 1e12, base * NOMINAL_RATIO[kind], ("TOPS" if w.dtype == "i8" else "TFLOP/s")
-        peak_note = "%s bf16 cuBLAS %s x nominal %s/bf16 ratio %.1f" % (peak_kind, which, kind, NOMINAL_RATIO[kind])
+        achieved, runit = ops_step / kernel_s / 1e12, ("TOPS" if w.dtype == "i8" else "TFLOP/s")
+        fr = tensor_roofline(achieved, tensor_kind(w), peaks, peak_kind)
+        if sustained is not None:
+            sustained["frac_measured_sustained"] = sustained["value"] / world / fr["peak_sustained"]
+            sustained["frac_nominal"] = sustained["value"] / world / fr["peak_nominal"]
     else:
-        achieved, peak, runit = ops_step / kernel_s / 1e12, FP32_ALU_TFLOPS, "TFLOP/s"
-        peak_note = "FP32 FMA roof: 148 SMs x 128 lanes x 2 x 1.965 GHz (derived, not measured)"
-    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak, "traffic": traffic,
-                "peak_source": peak_note, "kernel": family, "kernel_us": kernel_s * 1e6}
+        achieved, runit = ops_step / kernel_s / 1e12, "TFLOP/s"
+        fr = {"peak": FP32_ALU_TFLOPS, "frac": achieved / FP32_ALU_TFLOPS, "frac_nominal": achieved / FP32_ALU_TFLOPS,
+              "peak_source": "FP32 FMA roof: 148 SMs x 128 lanes x 2 x 1.965 GHz (derived, not measured)"}
+    roofline = {"bound": bound, "achieved": achieved, "unit": runit, "traffic": traffic, "kernel": family, "kernel_us": kernel_s * 1e6}
+    roofline.update(fr)
+    if clocks.get("sm_mhz"):
+        roofline["kernel_us_x_sm_mhz"] = kernel_s * 1e6 * clocks["sm_mhz"]   # clock-independent duration: microseconds x MHz = cycles
 
-    if args.kernel_only:
-        cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
-        e2e_value = None
+    if with_cpu and reps.rank == 0 and world == 1:
+        cpu_v, cores, sample, _ = cpu_oracle_rate(w, target_seconds=cpu_seconds)
     else:
-        cpu_v, cores, sample, _ = cpu_oracle_rate(w)
+        cpu_v, cores, sample = None, 0, "skipped"
     if nsets * set_bytes > 2 * L2_BYTES:
         l2_note = "inputs rotate over %d device copies (%.0f MB in total, larger than the 126 MB L2)" % (nsets, nsets * set_bytes / 1e6)
     else:
         l2_note = ("working set of %d rotating copies is %.1f MB, far below L2: this workload is launch/latency-bound, "
                    "no DRAM figure is claimed for it" % (nsets, nsets * set_bytes / 1e6))
-    line = {
-        "metric": "recurrence_matmul_throughput", "value": value, "unit": unit_of(w), "n_gpus": world, "steps": args.steps,
-        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+    rec = {
+        "value": value, "unit": unit_of(w), "steps": steps, "ms_per_step": ms_per_step, "seconds": ms * 1e-3, "dtype": w.dtype,
         "config": {"workload": describe(w), "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": l2_note, "kernel": family,
-                   "launch": ("CUDA graph of %d launches, replayed %d times" % (chunk, args.steps // chunk)) if graph is not None
+                   "launch": ("CUDA graph of %d launches, replayed %d times" % (chunk, steps // chunk)) if chunk > 1 or args.graph == "on"
                    else "one library call per step"},
-        "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": unit_of(w), "h2d_bytes_per_step": int(hA.numel() * hA.element_size() + hB.numel() * hB.element_size()),
-                "d2h_bytes_per_step": int(hC.numel() * hC.element_size()), "steps": e2e_steps},
-        "gpu_launches": int(launches),
-        "roofline": roofline,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
         "cpu_baseline": {"value": cpu_v, "unit": unit_of(w), "cores": cores, "kind": "oracle", "sample": sample},
     }
-    print(json.dumps(line))
+    if plain_call_us is not None:
+        rec["plain_call_us"] = plain_call_us   # the same step as an ordinary library call from Python, no graph
+    if sustained is not None:
+        rec["sustained"] = sustained
+    return rec
+
+
+def run_ours(args, w, with_configs):
+    """The headline workload timed over exactly --steps steps; with `with_configs` (the default run) the other
+    configurations of the matrix-multiply recurrence follow as sub-records, each over a region of at least 0.25 s."""
+    torch, reps, local = cuda_setup()
+    kernel_only = args.kernel_only
+    base = w.name.split("@")[0].split("+")[0]
+    sustained = 1.0 if (with_configs or args.sustained) and base in ("c2", "c3") else 0.0
+    head = measure_matmul(w, args.steps, args, torch, reps, local, sustained_seconds=sustained,
+                          with_cpu=not kernel_only, with_e2e=not kernel_only)
+    line = {"metric": "recurrence_matmul_throughput", "value": head["value"], "unit": head["unit"], "n_gpus": reps.world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic"}
+    for k in ("config", "clocks", "e2e", "gpu_launches", "roofline", "cpu_baseline", "sustained", "plain_call_us"):
+        if k in head:
+            line[k] = head[k]
+    if with_configs and reps.world == 1:
+        subs = {}
+        for name in ("c1", "c2", "c4", "c5"):
+            if name == base:
+                continue
+            cw = inputs.WORKLOADS[name]
+            subs[name] = measure_matmul(cw, None, args, torch, reps, local, min_seconds=0.25,
+                                        sustained_seconds=1.0 if name == "c2" else 0.0, cpu_seconds=5.0)
+        line["configs"] = subs
+    if reps.rank == 0:
+        print(json.dumps(line))
     reps.close()
 
 
@@ -432,15 +517,11 @@ def run_trsm(args, w):
         reps.close()
         return
     step_s = ms_per_step * 1e-3
-    base = float(peaks["bf16_tflops"]) if args.steps * step_s < 1.0 else float(peaks["bf16_tflops_sustained"])
-    which = "burst" if args.steps * step_s < 1.0 else "sustained"
-    peak = base * NOMINAL_RATIO["tf32"]
-    roofline = {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s", "frac": value / world / peak,
-                "traffic": None,
-                "peak_source": "%s bf16 cuBLAS %s x nominal tf32/bf16 ratio %.1f; the whole step is rated (n(n+1)m flop, the three "
-                               "TF32 products of each fp32 product counted once): %d launches per solve"
-                               % (peak_kind, which, NOMINAL_RATIO["tf32"], launches // max(1, args.steps)),
+    roofline = {"bound": "tensor", "achieved": value / world, "unit": "TFLOP/s", "traffic": None,
+                "note": "the whole step is rated (n(n+1)m flop, the three TF32 products of each fp32 product counted once): "
+                        "%d launches per solve" % (launches // max(1, args.steps)),
                 "kernel": "tcgen05_3xtf32 (tile products) + trsm_diag (diagonal tiles)", "kernel_us": step_s * 1e6}
+    roofline.update(tensor_roofline(value / world, "tf32", peaks, peak_kind))
     if args.kernel_only:
         cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
     else:
@@ -628,13 +709,11 @@ def run_attention(args, w):
         reps.close()
         return
     step_s = ms_per_step * 1e-3
-    which = "burst" if total_ms < 1000.0 else "sustained"
-    peak = float(peaks["bf16_tflops"] if which == "burst" else peaks["bf16_tflops_sustained"])
     family = "fa2_d%d" % w.d
-    roofline = {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s", "frac": value / world / peak,
-                "traffic": load_traffic(w, family),
-                "peak_source": "%s bf16 cuBLAS %s; 4 N M d flop per problem (both products, exponentials not counted)" % (peak_kind, which),
+    roofline = {"bound": "tensor", "achieved": value / world, "unit": "TFLOP/s", "traffic": load_traffic(w, family),
+                "note": "4 N M d flop per problem (both products, exponentials not counted)",
                 "kernel": "fa2_kernel<%d>" % w.d, "kernel_us": step_s * 1e6}
+    roofline.update(tensor_roofline(value / world, "bf16", peaks, peak_kind))
     if args.kernel_only:
         cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
     else:
@@ -919,15 +998,11 @@ def run_chol(args, w):
         reps.close()
         return
     step_s = ms_per_step * 1e-3
-    which = "burst" if total_ms < 1000.0 else "sustained"
-    base = float(peaks["bf16_tflops"] if which == "burst" else peaks["bf16_tflops_sustained"])
-    peak = base * NOMINAL_RATIO["tf32"]
-    roofline = {"bound": "tensor", "achieved": value / world, "peak": peak, "unit": "TFLOP/s", "frac": value / world / peak,
-                "traffic": None,
-                "peak_source": "%s bf16 cuBLAS %s x nominal tf32/bf16 ratio %.1f; the whole step is rated (n^3/3 flop, the three "
-                               "TF32 products of each fp32 product counted once): %d launches per factorisation"
-                               % (peak_kind, which, NOMINAL_RATIO["tf32"], launches // max(1, args.steps)),
+    roofline = {"bound": "tensor", "achieved": value / world, "unit": "TFLOP/s", "traffic": None,
+                "note": "the whole step is rated (n^3/3 flop, the three TF32 products of each fp32 product counted once): "
+                        "%d launches per factorisation" % (launches // max(1, args.steps)),
                 "kernel": "tcgen05_3xtf32 (SYRK/GEMM sums) + chol_diag (diagonal tiles) + trsm_diag (tiles below)", "kernel_us": step_s * 1e6}
+    roofline.update(tensor_roofline(value / world, "tf32", peaks, peak_kind))
     if args.kernel_only:
         cpu_v, cores, sample = None, 0, "skipped (--kernel-only)"
     else:
@@ -999,7 +1074,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c2", choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS) + sorted(inputs.ATTENTION_WORKLOADS) + sorted(inputs.SCAN_WORKLOADS)
+    ap.add_argument("--workload", default=None, choices=sorted(inputs.WORKLOADS) + sorted(inputs.TRSM_WORKLOADS) + sorted(inputs.ATTENTION_WORKLOADS) + sorted(inputs.SCAN_WORKLOADS)
                     + sorted(inputs.CHOL_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--shape", default=None, help="M,N,K[,batch] (c1..c5), n,m[,tile] (t1, t2) batch,N,M,d (a1, a2), rows,n (p1..p3) or n[,tile] (h1, h2): a smaller case of the workload's recipe (for profiling)")
@@ -1007,7 +1082,13 @@ def main():
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="replay the timed steps from a CUDA graph (auto: only for launch-bound workloads)")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU-baseline legs (for profiling)")
+    ap.add_argument("--sustained", action="store_true", help="add a region of at least one second (c2, c3) to a single-workload run")
     args = ap.parse_args()
+    # no --workload: the largest configuration that fits one GPU (c3) is the headline, and the other four
+    # configurations of the matrix-multiply recurrence follow as sub-records of the same line
+    with_configs = args.workload is None and args.impl == "ours" and not args.kernel_only and not args.shape
+    if args.workload is None:
+        args.workload = "c3"
     if args.workload in inputs.TRSM_WORKLOADS:
         w = inputs.TRSM_WORKLOADS[args.workload]
         if args.shape:  # n,m[,tile]: a smaller case of the same recipe (for profiling)
@@ -1057,8 +1138,8 @@ def main():
         run_reference(args, w)
         return
     if args.steps is None:
-        args.steps = {"c1": 2000, "c2": 2000, "c3": 200, "c4": 1000, "c5": 1000}[w.name.split("@")[0].split("+")[0]]
-    run_ours(args, w)
+        args.steps = {"c1": 20000, "c2": 4000, "c3": 400, "c4": 4000, "c5": 3000}[w.name.split("@")[0].split("+")[0]]
+    run_ours(args, w, with_configs)
 
 
 if __name__ == "__main__":

@@ -131,9 +131,14 @@ int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, int64_t K, i
  * message in cyc_last_cuda_error().  Results equal the split-K path of
  * cyc_recurrence_matmul when both pick the same S, and stay within the usual tolerance
  * otherwise (int8: exact).
- * The first call on each device looks up the array's device address (a driver query, no
- * allocation); make that first call outside any stream capture.  No call of this
- * function allocates or frees memory.  Nothing in the array needs clearing: every
+ * The first call on each device looks up the array's device address with
+ * cudaGetSymbolAddress; make that first call outside any stream capture.  The look-up
+ * itself requests no memory, but if nothing of the library has run on the device yet,
+ * the CUDA runtime loads the library's device code at that moment (lazy module loading),
+ * and that is when the device receives its copy of the array: after one warm-up call per
+ * device, no call of this function allocates or frees memory -- neither through
+ * cudaMalloc / cudaFree nor through the library's pool (cyc_pool_reserved_bytes reports
+ * the pool's size for those who want to check).  Nothing in the array needs clearing: every
  * element a call reads was written by the same call.  All calls share the one array, so
  * two calls whose kernels can overlap on the GPU (different streams, no dependency) race
  * on it: order them on one stream or with events.
@@ -141,6 +146,14 @@ int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, int64_t K, i
 #define CYC_STATIC_WORKSPACE_BYTES (8u << 20)
 int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B, void* C,
                                         void* stream, unsigned flags);
+
+/*
+ * Bytes the library's stream-ordered workspace pool currently holds from the driver on
+ * the current device (cudaMemPoolAttrReservedMemCurrent; 0 if no call has needed the
+ * pool yet).  Introspection only (the paper has no counterpart): lets a host verify
+ * that a sequence of calls did not grow the library's memory.
+ */
+int cyc_pool_reserved_bytes(int64_t* out);
 
 /*
  * Block lower-triangular solve  L X = B  (Section "Multiple Iteration Spaces":
@@ -276,6 +289,19 @@ int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles);
  * Host only, makes no CUDA call. */
 const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
                            const void* C, unsigned flags);
+
+/* Which space-time mapping of the base recurrence the dispatcher would use for these
+ * arguments (Section "Space-time Mappings of Dataflow Recurrences" prints a
+ * weight-stationary and an output-stationary program for the same recurrence):
+ *   "output_stationary"  every block of C stays in place (tensor memory or registers) for
+ *                        its whole k loop while A and B stream past it -- k runs in time,
+ *                        one owner per C_ij; what CYC_FLAG_FIXED_K_ORDER always selects;
+ *   "k_sliced"           the k range of a block is cut into slices held by different CTA
+ *                        pairs at the same time (k partly in space) and the slices' partial
+ *                        sums are added in increasing k by a second kernel.
+ * NULL if the arguments are invalid.  Host only, makes no CUDA call. */
+const char* cyc_schedule_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
+                             const void* C, unsigned flags);
 
 /* Number of kernels this library has launched in the calling process (monotonic). */
 int64_t cyc_launch_count(void);

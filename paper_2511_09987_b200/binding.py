@@ -27,6 +27,7 @@ SYMBOLS = {
     "cyc_recurrence_matmul_batched": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _i64, _ptr, _i64, _ptr, _i64, _ptr, _u32]),
     "cyc_recurrence_matmul_host": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_recurrence_matmul_splitk_static": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
+    "cyc_pool_reserved_bytes": (_int, [ctypes.POINTER(ctypes.c_int64)]),
     "cyc_block_trsm": (_int, [_i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_flash_attention": (_int, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _ptr, _ptr, _u32]),
     "cyc_prefix_sum": (_int, [_i64, _i64, _int, _ptr, _i64, _ptr, _i64, _ptr, _u32]),
@@ -34,6 +35,7 @@ SYMBOLS = {
     "cyc_selftest_bounded_wait": (_int, [_ptr, _i64]),
     "cyc_last_device_status": (_int, [_ptr, ctypes.POINTER(ctypes.c_int)]),
     "cyc_kernel_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
+    "cyc_schedule_for": (ctypes.c_char_p, [_i64, _i64, _i64, _i64, _int, _ptr, _ptr, _ptr, _u32]),
     "cyc_launch_count": (_i64, []),
     "cyc_last_cuda_error": (ctypes.c_char_p, []),
     "cyc_status_string": (ctypes.c_char_p, [_int]),
@@ -64,6 +66,7 @@ cyc_recurrence_matmul = _lib.cyc_recurrence_matmul
 cyc_recurrence_matmul_batched = _lib.cyc_recurrence_matmul_batched
 cyc_recurrence_matmul_host = _lib.cyc_recurrence_matmul_host
 cyc_recurrence_matmul_splitk_static = _lib.cyc_recurrence_matmul_splitk_static
+cyc_pool_reserved_bytes = _lib.cyc_pool_reserved_bytes
 cyc_block_trsm = _lib.cyc_block_trsm
 cyc_flash_attention = _lib.cyc_flash_attention
 cyc_prefix_sum = _lib.cyc_prefix_sum
@@ -72,6 +75,7 @@ cyc_selftest_bounded_wait = _lib.cyc_selftest_bounded_wait
 cyc_last_device_status = _lib.cyc_last_device_status
 CYC_STATIC_WORKSPACE_BYTES = 8 << 20
 cyc_kernel_for = _lib.cyc_kernel_for
+cyc_schedule_for = _lib.cyc_schedule_for
 cyc_launch_count = _lib.cyc_launch_count
 cyc_last_cuda_error = _lib.cyc_last_cuda_error
 cyc_status_string = _lib.cyc_status_string
@@ -92,9 +96,20 @@ def _torch_dtype_code(t) -> int:
     return {torch.float32: CYC_F32, torch.bfloat16: CYC_BF16_F32, torch.int8: CYC_I8_I32}[t.dtype]
 
 
-def _stream() -> int:
+def _stream(t=None) -> int:
+    """The current torch stream of the device the operands live on (which must be the current device: the library
+    launches on the current device)."""
     import torch
+    if t is not None and t.device.index != torch.cuda.current_device():
+        raise ValueError("operands live on %s but the current device is cuda:%d" % (t.device, torch.cuda.current_device()))
     return torch.cuda.current_stream().cuda_stream
+
+
+def _check_out(name, T, shape, dtype, like):
+    """A caller-supplied result tensor goes to the kernels as a raw address: refuse anything but a contiguous CUDA
+    tensor of the exact shape and dtype on the operands' device."""
+    if not (T.is_cuda and T.device == like.device and T.is_contiguous() and tuple(T.shape) == tuple(shape) and T.dtype == dtype):
+        raise ValueError("%s must be a contiguous %s CUDA tensor of shape %s on %s" % (name, dtype, tuple(shape), like.device))
 
 
 def recurrence_matmul(A, B, C=None, *, b_col_major: bool = False, fixed_k_order: bool = False):
@@ -109,9 +124,14 @@ def recurrence_matmul(A, B, C=None, *, b_col_major: bool = False, fixed_k_order:
     N = B.shape[0] if b_col_major else B.shape[1]
     if (B.shape[1] if b_col_major else B.shape[0]) != K:
         raise ValueError("inner dimensions differ")
+    out_dtype = torch.int32 if code == CYC_I8_I32 else torch.float32
+    if B.device != A.device:
+        raise ValueError("A and B must live on the same device")
     if C is None:
-        C = torch.empty((M, N), dtype=torch.int32 if code == CYC_I8_I32 else torch.float32, device=A.device)
-    check(cyc_recurrence_matmul(M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(),
+        C = torch.empty((M, N), dtype=out_dtype, device=A.device)
+    else:
+        _check_out("C", C, (M, N), out_dtype, A)
+    check(cyc_recurrence_matmul(M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(A),
                                 _flags(b_col_major, fixed_k_order)))
     return C
 
@@ -126,9 +146,14 @@ def recurrence_matmul_batched(A, B, C=None, *, b_col_major: bool = False, fixed_
     N = B.shape[1] if b_col_major else B.shape[2]
     if B.shape[0] != batch or (B.shape[2] if b_col_major else B.shape[1]) != K or B.dtype != A.dtype:
         raise ValueError("operand shapes or dtypes differ")
+    out_dtype = torch.int32 if code == CYC_I8_I32 else torch.float32
+    if B.device != A.device:
+        raise ValueError("A and B must live on the same device")
     if C is None:
-        C = torch.empty((batch, M, N), dtype=torch.int32 if code == CYC_I8_I32 else torch.float32, device=A.device)
-    check(cyc_recurrence_matmul_batched(batch, M, N, K, code, A.data_ptr(), 0, B.data_ptr(), 0, C.data_ptr(), 0, _stream(),
+        C = torch.empty((batch, M, N), dtype=out_dtype, device=A.device)
+    else:
+        _check_out("C", C, (batch, M, N), out_dtype, A)
+    check(cyc_recurrence_matmul_batched(batch, M, N, K, code, A.data_ptr(), 0, B.data_ptr(), 0, C.data_ptr(), 0, _stream(A),
                                         _flags(b_col_major, fixed_k_order)))
     return C
 
@@ -165,9 +190,14 @@ def recurrence_matmul_splitk_static(A, B, C=None, *, b_col_major: bool = False):
     N = B.shape[0] if b_col_major else B.shape[1]
     if (B.shape[1] if b_col_major else B.shape[0]) != K or B.dtype != A.dtype:
         raise ValueError("operand shapes or dtypes differ")
+    out_dtype = torch.int32 if code == CYC_I8_I32 else torch.float32
+    if B.device != A.device:
+        raise ValueError("A and B must live on the same device")
     if C is None:
-        C = torch.empty((M, N), dtype=torch.int32 if code == CYC_I8_I32 else torch.float32, device=A.device)
-    check(cyc_recurrence_matmul_splitk_static(M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(),
+        C = torch.empty((M, N), dtype=out_dtype, device=A.device)
+    else:
+        _check_out("C", C, (M, N), out_dtype, A)
+    check(cyc_recurrence_matmul_splitk_static(M, N, K, code, A.data_ptr(), B.data_ptr(), C.data_ptr(), _stream(A),
                                               _flags(b_col_major, False)))
     return C
 
@@ -184,9 +214,11 @@ def block_trsm(L, B, X=None, *, tile: int = 0, fixed_k_order: bool = False):
         raise ValueError("L must be [n,n] and B [n,m] of one dtype")
     if X is None:
         X = torch.empty_like(B)
-    elif not (X.is_cuda and X.is_contiguous() and X.shape == B.shape and X.dtype == B.dtype):
+    elif not (X.is_cuda and X.device == B.device and X.is_contiguous() and X.shape == B.shape and X.dtype == B.dtype):
         raise ValueError("X must be a contiguous CUDA tensor shaped like B")
-    check(cyc_block_trsm(n, m, tile, _torch_dtype_code(L), L.data_ptr(), B.data_ptr(), X.data_ptr(), _stream(),
+    if L.device != B.device:
+        raise ValueError("L and B must live on the same device")
+    check(cyc_block_trsm(n, m, tile, _torch_dtype_code(L), L.data_ptr(), B.data_ptr(), X.data_ptr(), _stream(L),
                          _flags(False, fixed_k_order)))
     return X
 
@@ -206,10 +238,16 @@ def flash_attention(Q, K, V, O=None):
     M = K.shape[1]
     if K.shape != (batch, M, d) or V.shape != (batch, M, d) or K.dtype != Q.dtype or V.dtype != Q.dtype:
         raise ValueError("operand shapes or dtypes differ")
+    if K.device != Q.device or V.device != Q.device:
+        raise ValueError("Q, K and V must live on the same device")
     if O is None:
         O = torch.empty((batch, N, d), dtype=torch.float32, device=Q.device)
+    else:
+        if O.dim() == 2 and squeeze:
+            O = O.unsqueeze(0)
+        _check_out("O", O, (batch, N, d), torch.float32, Q)
     check(cyc_flash_attention(batch, N, M, d, _torch_dtype_code(Q), Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(),
-                              _stream(), 0))
+                              _stream(Q), 0))
     return O[0] if squeeze else O
 
 
@@ -224,14 +262,14 @@ def prefix_sum(A, P=None):
         raise ValueError("float32 or int32 only")
     if P is None:
         P = torch.empty(A.shape, dtype=A.dtype, device=A.device)
-    if P.shape != A.shape or P.dtype != A.dtype or not P.is_cuda or P.stride(-1) != 1:
+    if P.shape != A.shape or P.dtype != A.dtype or not P.is_cuda or P.device != A.device or P.stride(-1) != 1:
         raise ValueError("P must match A")
     rows, n = (1, A.shape[0]) if A.dim() == 1 else A.shape
     if rows * n == 0:
         return P
     sA = A.stride(0) if A.dim() == 2 and rows > 1 else n
     sP = P.stride(0) if P.dim() == 2 and rows > 1 else n
-    check(cyc_prefix_sum(rows, n, codes[A.dtype], A.data_ptr(), sA, P.data_ptr(), sP, _stream(), 0))
+    check(cyc_prefix_sum(rows, n, codes[A.dtype], A.data_ptr(), sA, P.data_ptr(), sP, _stream(A), 0))
     return P
 
 
@@ -243,9 +281,9 @@ def cholesky(A, L=None, *, tile: int = 0, fixed_k_order: bool = False):
         raise ValueError("A must be a contiguous square float32 CUDA tensor")
     if L is None:
         L = torch.empty_like(A)
-    if L.shape != A.shape or L.dtype != A.dtype or not L.is_cuda or not L.is_contiguous():
+    if L.shape != A.shape or L.dtype != A.dtype or not L.is_cuda or L.device != A.device or not L.is_contiguous():
         raise ValueError("L must match A")
-    check(cyc_cholesky(A.shape[0], tile, CYC_F32, A.data_ptr(), L.data_ptr(), _stream(), _flags(False, fixed_k_order)))
+    check(cyc_cholesky(A.shape[0], tile, CYC_F32, A.data_ptr(), L.data_ptr(), _stream(A), _flags(False, fixed_k_order)))
     return L
 
 
@@ -257,4 +295,9 @@ def last_device_status() -> int:
 
 def kernel_for(batch, M, N, K, dtype, a_ptr=256, b_ptr=1 << 40, c_ptr=1 << 41, *, b_col_major=False, fixed_k_order=False):
     r = cyc_kernel_for(batch, M, N, K, DTYPE_CODES.get(dtype, dtype), a_ptr, b_ptr, c_ptr, _flags(b_col_major, fixed_k_order))
+    return r.decode() if r else None
+
+
+def schedule_for(batch, M, N, K, dtype, a_ptr=256, b_ptr=1 << 40, c_ptr=1 << 41, *, b_col_major=False, fixed_k_order=False):
+    r = cyc_schedule_for(batch, M, N, K, DTYPE_CODES.get(dtype, dtype), a_ptr, b_ptr, c_ptr, _flags(b_col_major, fixed_k_order))
     return r.decode() if r else None

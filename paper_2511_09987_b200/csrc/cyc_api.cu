@@ -7,6 +7,8 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <set>
+#include <utility>
 #include <type_traits>
 
 #include <cuda.h>
@@ -283,6 +285,32 @@ static int device_info(DeviceInfo* out) {
     return CYC_OK;
 }
 
+// Once per device: the address of the status word, and the opt-in to more than 48 KB of dynamic shared memory for a
+// kernel.  Both are remembered so that the per-call path makes neither runtime call again.
+static int status_word(int** out) {
+    static std::mutex mu;
+    static int* addr[64] = {};
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!addr[dev]) CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&addr[dev]), g_device_status));
+    *out = addr[dev];
+    return CYC_OK;
+}
+
+static int ensure_dynamic_smem(const void* kernel, int bytes) {
+    static std::mutex mu;
+    static std::set<std::pair<const void*, int>> done;
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(mu);
+    if (done.count({kernel, dev})) return CYC_OK;
+    CYC_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    done.insert({kernel, dev});
+    return CYC_OK;
+}
+
 // ------------------------------------------------------------------ tensor-core launch
 template <int KIND, bool B_MN, int BN, int STAGES>
 static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
@@ -303,10 +331,10 @@ static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
     p.tiles_m = static_cast<int>((q.M + UMMA_BM - 1) / UMMA_BM);
     p.tiles_n = static_cast<int>((q.N + BN - 1) / BN);
     p.num_tiles = q.batch * p.tiles_m * p.tiles_n;
-    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    if (int rc_ = status_word(&p.status)) return rc_;
 
     auto kern = umma_recurrence_kernel<KIND, B_MN, BN, STAGES>;
-    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Sm::TOTAL));
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), Sm::TOTAL)) return rc_;
     const long long grid = p.num_tiles < sms ? p.num_tiles : sms;
     kern<<<static_cast<unsigned>(grid), UMMA_THREADS, Sm::TOTAL, st>>>(tmA, tmB, p);
     CYC_CUDA(cudaGetLastError());
@@ -349,9 +377,9 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws 
         p.split_k = plan.S;
         p.kb_per_slice = plan.kb_per_slice;
     }
-    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    if (int rc_ = status_word(&p.status)) return rc_;
     auto kern = umma_pair_kernel<KIND, B_MN, STAGES>;
-    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), SMEM)) return rc_;
     const long long max_pairs = sms / 2;
     const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
     kern<<<static_cast<unsigned>(2 * pairs), UMMA_THREADS, SMEM, st>>>(tmA, tmB, tmC, p);
@@ -363,14 +391,14 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws 
 // ------------------------------------------------------------------ split-K
 // Workspace for the partial sums: stream-ordered allocations from a pool the library owns (one per device),
 // so that repeated calls reuse the same memory without a synchronising cudaMalloc.
-static int workspace_pool(cudaMemPool_t* out) {
+static int workspace_pool(cudaMemPool_t* out, bool create = true) {
     static std::mutex mu;
     static cudaMemPool_t pools[64] = {};
     int dev = 0;
     CYC_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
     std::lock_guard<std::mutex> lk(mu);
-    if (!pools[dev]) {
+    if (!pools[dev] && create) {
         cudaMemPoolProps props = {};
         props.allocType = cudaMemAllocationTypePinned;
         props.handleTypes = cudaMemHandleTypeNone;
@@ -444,9 +472,9 @@ static int launch_pair_tall_cfg(const Problem& q, cudaStream_t st, int sms) {
     p.tiles_m = static_cast<int>((q.M + 511) / 512);
     p.tiles_n = static_cast<int>((q.N + PAIR_BN - 1) / PAIR_BN);
     p.num_tiles = q.batch * p.tiles_m * p.tiles_n;
-    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    if (int rc_ = status_word(&p.status)) return rc_;
     auto kern = umma_pair_tall_kernel<KIND, B_MN>;
-    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TALL_SMEM_BYTES));
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), TALL_SMEM_BYTES)) return rc_;
     const long long max_pairs = sms / 2;
     const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
     kern<<<static_cast<unsigned>(2 * pairs), TALL_THREADS, TALL_SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
@@ -478,9 +506,9 @@ static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
     p.tiles_m = static_cast<int>((q.M + 255) / 256);
     p.tiles_n = static_cast<int>((q.N + PAIR_BN - 1) / PAIR_BN);
     p.num_tiles = q.batch * p.tiles_m * p.tiles_n;
-    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    if (int rc_ = status_word(&p.status)) return rc_;
     auto kern = umma_pair_tf32x3_kernel<B_MN>;
-    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, X3_SMEM_BYTES));
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), X3_SMEM_BYTES)) return rc_;
     const long long max_pairs = sms / 2;
     const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
     kern<<<static_cast<unsigned>(2 * pairs), X3_THREADS, X3_SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
@@ -606,9 +634,9 @@ static int launch_fa2(long long batch, long long N, long long M, const void* Q, 
     p.N = static_cast<int>(N); p.M = static_cast<int>(M);
     p.tiles_q = static_cast<int>((N + FA2_BM - 1) / FA2_BM);
     p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
-    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
+    if (int rc_ = status_word(&p.status)) return rc_;
     auto kern = fa2_kernel<D>;
-    CYC_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Fa2Smem<D>::TOTAL));
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), Fa2Smem<D>::TOTAL)) return rc_;
     kern<<<static_cast<unsigned>(batch * p.tiles_q), FA2_THREADS, Fa2Smem<D>::TOTAL, st>>>(tmQ, tmK, tmV, p);
     CYC_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
@@ -802,6 +830,20 @@ extern "C" int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t
     return dtype == CYC_BF16_F32 ? launch_splitk<KIND_BF16>(q, st, di.sms, ws, plan) : launch_splitk<KIND_I8>(q, st, di.sms, ws, plan);
 }
 
+extern "C" int cyc_pool_reserved_bytes(int64_t* out) {
+    if (!out) return CYC_ERR_INVALID_ARG;
+    *out = 0;
+    cudaMemPool_t pool = nullptr;
+    int rc = workspace_pool(&pool, /*create=*/false);
+    if (rc) return rc;
+    if (pool) {
+        unsigned long long bytes = 0;
+        CYC_CUDA(cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReservedMemCurrent, &bytes));
+        *out = static_cast<int64_t>(bytes);
+    }
+    return CYC_OK;
+}
+
 extern "C" int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, const void* L, const void* B, void* X,
                               void* stream, unsigned flags) {
     if (n <= 0 || m <= 0 || tile < 0 || tile > TRSM_T_MAX || !L || !B || !X) return CYC_ERR_INVALID_ARG;
@@ -822,7 +864,7 @@ extern "C" int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, con
     const long long nb = (n + t.T - 1) / t.T;
     int levels = 0;
     while ((1ll << levels) < nb) ++levels;
-    CYC_CUDA(cudaFuncSetAttribute(trsm_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TRSM_SMEM_BYTES));
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel), TRSM_SMEM_BYTES)) return rc_;
     if (levels) {
         cudaMemPool_t pool;
         int rc = workspace_pool(&pool);
@@ -889,8 +931,8 @@ static int launch_scan(long long rows, long long n, const void* A, long long sA,
     p.total_tiles = tiles;
     p.vec_ok = (reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(P) % 16 == 0 && (rows == 1 || (sA % 4 == 0 && sP % 4 == 0)))
                    ? 1 : 0;
-    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p.status), g_device_status));
-    CYC_CUDA(cudaFuncSetAttribute(scan_kernel<T, SUBS>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(TILE * sizeof(T)) + 128));
+    if (int rc_ = status_word(&p.status)) return rc_;
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(scan_kernel<T, SUBS>), static_cast<int>(TILE * sizeof(T)) + 128)) return rc_;
     cudaMemPool_t pool;
     int rc = workspace_pool(&pool);
     if (rc) return rc;
@@ -958,8 +1000,8 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
     float* Lf = static_cast<float*>(L);
     const long long T = tile ? tile : CHOL_T_MAX;
     const bool in_place = a0 == l0;
-    CYC_CUDA(cudaFuncSetAttribute(chol_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CHOL_SMEM_BYTES));
-    CYC_CUDA(cudaFuncSetAttribute(trsm_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TRSM_SMEM_BYTES));
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(chol_diag_kernel), CHOL_SMEM_BYTES)) return rc_;
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel), TRSM_SMEM_BYTES)) return rc_;
     // The k range of a panel's sums is cut into up to CHOL_MAX_SLICES equal slices (one batched launch: a panel has
     // few 256-row tiles, and the slices give every CTA pair work) plus one launch for the remainder; the consumers
     // add the slices' partial sums in increasing k.
@@ -1083,6 +1125,14 @@ extern "C" const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64
         case FAM_UMMA_3XTF32: return "tcgen05_3xtf32";
         default: return "simt";
     }
+}
+
+extern "C" const char* cyc_schedule_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
+                                        const void* C, unsigned flags) {
+    if (batch <= 0 || M <= 0 || N <= 0 || K <= 0) return nullptr;
+    Problem q{batch, M, N, K, dtype, A, B, const_cast<void*>(C), M * K, K * N, M * N, flags};
+    if (validate(q) != CYC_OK) return nullptr;
+    return choose(q) == FAM_UMMA_SPLITK ? "k_sliced" : "output_stationary";
 }
 
 extern "C" int64_t cyc_launch_count(void) { return g_launches.load(); }

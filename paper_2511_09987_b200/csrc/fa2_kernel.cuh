@@ -3,9 +3,9 @@
 //   S_{i,J_t} = alpha Q_i K_{J_t}^T,  mh = max(m, max S),  l <- e^{m-mh} l + sum_j e^{S_ij-mh},
 //   o <- e^{m-mh} o + sum_j e^{S_ij-mh} V_j,  m <- mh,   O_i = o / l,     alpha = 1/sqrt(d)
 //
-// "Each processing element holds a query tile and computes a series of matrix multiplications followed by elementwise
-// activations in place": here a CTA holds a 128-row query tile in shared memory for its whole life and walks the key
-// tiles J_t (128 keys each):
+// The paper assigns one query tile to one processing element, which alternates matrix products with elementwise
+// updates of its own state.  Here that element is a CTA: it keeps a 128-row query tile in shared memory for its whole
+// life and walks the key tiles J_t (128 keys each):
 //   warp 0      TMA producer: Q once, then K_t and V_t into two buffers each (K_t is released as soon as S_t is done)
 //   warp 1      one thread issues tcgen05 MMAs:  S_t = Q K_t^T  (fp32, in tensor memory, two buffers) and
 //               U_t = P_t V_t (fp32, tensor memory, two buffers), P_t = e^{S_t - mh} in bf16 read from TENSOR memory:

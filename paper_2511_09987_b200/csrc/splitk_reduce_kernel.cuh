@@ -7,10 +7,12 @@
 
 namespace cyc {
 
-// ws: [batch][S][plane] ; C: [batch] planes with stride sC ; plane = M*N elements
+// ws: [batch][S][plane] ; C: [batch] planes with stride sC ; plane = M*N elements.
+// C may be plane 0 of ws (the sum taken in place): every thread reads the S values of its own index before it writes
+// that index and touches no other, so the pointers carry no no-alias promise.
 template <typename T>
-__global__ void __launch_bounds__(128) splitk_reduce_kernel(const T* __restrict__ ws, T* __restrict__ C, long long plane,
-                                                            long long sC, int S, long long batch, int vec4) {
+__global__ void __launch_bounds__(128) splitk_reduce_kernel(const T* ws, T* C, long long plane, long long sC, int S,
+                                                            long long batch, int vec4) {
     const long long per_batch = vec4 ? plane / 4 : plane;
     const long long total = per_batch * batch;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;

@@ -158,3 +158,18 @@ def test_kernel_selection(binding):
     assert k(1, 64, 64, 64, "bf16", a_ptr=258) == "simt"     # base not 16-byte aligned
     assert k(1, 64, 64, 64, "bf16", a_ptr=257) is None       # not even element aligned
     assert k(1, 0, 64, 64, "bf16") is None
+
+
+def test_static_workspace_entry_point_refuses_on_the_host(binding):
+    """Requests the fixed workspace cannot serve are turned down by host-side checks, before any CUDA call."""
+    b = binding
+    A, B, C = 1 << 20, 1 << 30, 1 << 40       # never dereferenced: the checks come before any launch
+    f = b.cyc_recurrence_matmul_splitk_static
+    big = 2048                                 # 2 * 2048 * 2048 * 4 bytes = 32 MiB > 8 MiB
+    assert 2 * big * big * 4 > b.CYC_STATIC_WORKSPACE_BYTES
+    assert f(big, big, 8192, b.CYC_BF16_F32, A, B, C, None, 0) == b.CYC_ERR_UNSUPPORTED
+    assert b"fixed workspace" in b.cyc_last_cuda_error()
+    assert f(256, 256, 512, b.CYC_BF16_F32, A, B, C, None, 0) == b.CYC_ERR_UNSUPPORTED       # k loop too short to cut
+    assert f(256, 256, 8192, b.CYC_F32, A, B, C, None, 0) == b.CYC_ERR_UNSUPPORTED           # fp32 has no split-K path
+    assert f(256, 256, 8192, b.CYC_BF16_F32, A, B, C, None, b.CYC_FLAG_FIXED_K_ORDER) == b.CYC_ERR_INVALID_ARG
+    assert f(256, 256, 8192, b.CYC_BF16_F32, None, B, C, None, 0) == b.CYC_ERR_INVALID_ARG

@@ -106,7 +106,32 @@ def test_exact_cases():
     del torch, binding
 
 
-def test_full_size_sampled_columns():
+def test_full_size_every_column():
+    """t2 at full size: the forward comparison with the oracle on all 4096 right-hand-side columns (every output of
+    X), the fp64 residual on one column of every 32-column CTA of the diagonal-tile kernel."""
+    import os
+    w = inputs.TRSM_WORKLOADS["t2"]
+    L, B = inputs.make_trsm_operands(w)
+    X = gpu_solve(L, B, w.tile)
+    assert X.shape == B.shape and np.isfinite(X).all()
+    threads = os.cpu_count() or 8
+    rcols = np.arange(0, w.m, 32) + (np.arange(w.m // 32) * 7) % 32      # one column per CTA, at varying offsets
+    R, S = otrsm.residual(L, B, X, rcols)
+    assert (np.abs(R) <= 1e-5 * S).all(), "residual %g of its scale" % float((np.abs(R) / S).max())
+    absL = np.abs(np.tril(np.nan_to_num(L))).astype(np.float64)
+    assert w.coupling == "dominant"
+    for c0 in range(0, w.m, 512):
+        cols = np.arange(c0, min(w.m, c0 + 512))
+        ref = otrsm.block_trsm(L, np.ascontiguousarray(B[:, cols]), w.tile, threads=threads)
+        err = np.abs(X[:, cols].astype(np.float64) - ref)
+        # the residual scale |B| + |L||X| of these columns (a library product: it is only the yardstick); with
+        # |L^-1| <= 2 in the infinity norm a column's error is at most twice its largest admissible residual
+        Sc = np.abs(B[:, cols]).astype(np.float64) + absL @ np.abs(X[:, cols]).astype(np.float64)
+        bound = 2e-5 * Sc.max(axis=0, keepdims=True)
+        assert (err <= bound).all(), "forward error %g of its bound (columns %d..)" % (float((err / bound).max()), c0)
+
+
+def test_quick_full_size_sampled_columns():
     w = inputs.TRSM_WORKLOADS["t2"]
     L, B = inputs.make_trsm_operands(w)
     X = gpu_solve(L, B, w.tile)

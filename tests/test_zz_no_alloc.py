@@ -5,8 +5,10 @@ handed the whole GPU to their own allocator at start-up, or they sit in a latenc
 that must never enter the driver's allocator.  For them the library carries a fixed workspace and
 an entry point that uses it instead of the stream-ordered pool.  This test calls that entry point
 through the C ABI twice in a row (different operands and shapes, so stale workspace contents would
-show) and compares with the ordinary entry point; it also checks that oversized requests are
-refused on the host.  Collected last on purpose (file name), and self-contained so that it also
+show) and compares with the ordinary entry point, and it checks the property in the name: after one
+warm-up call, free device memory and the library pool's size are the same before and after every
+call.  (That oversized requests are refused on the host is checked without a GPU, in
+tests/test_abi.py.)  Collected last on purpose (file name), and self-contained so that it also
 passes alone in a fresh process.
 """
 import numpy as np
@@ -62,15 +64,32 @@ def test_two_calls_in_a_row_match_the_ordinary_entry_point(dtype, col):
             assert (np.abs(got.astype(np.float64) - ref) <= 4e-3 * S).all(), "call %d vs oracle" % call
 
 
-def test_requests_beyond_the_fixed_workspace_are_refused_on_the_host():
+def _pool_bytes(b):
+    import ctypes
+    out = ctypes.c_int64(-1)
+    assert b.cyc_pool_reserved_bytes(ctypes.byref(out)) == b.CYC_OK
+    return out.value
+
+
+def test_calls_allocate_nothing():
+    """After one warm-up call on the device (which may load the library's device code, the moment the device receives
+    its copy of the fixed array), two further calls leave the free device memory and the library pool as they were."""
+    import torch
     from paper_2511_09987_b200 import binding as b
-    A, B, C = 1 << 20, 1 << 30, 1 << 40       # never dereferenced: the checks come before any launch
-    f = b.cyc_recurrence_matmul_splitk_static
-    big = 2048                                 # 2 * 2048 * 2048 * 4 bytes = 32 MiB > 8 MiB
-    assert 2 * big * big * 4 > b.CYC_STATIC_WORKSPACE_BYTES
-    assert f(big, big, 8192, b.CYC_BF16_F32, A, B, C, None, 0) == b.CYC_ERR_UNSUPPORTED
-    assert b"fixed workspace" in b.cyc_last_cuda_error()
-    assert f(256, 256, 512, b.CYC_BF16_F32, A, B, C, None, 0) == b.CYC_ERR_UNSUPPORTED       # k loop too short to cut
-    assert f(256, 256, 8192, b.CYC_F32, A, B, C, None, 0) == b.CYC_ERR_UNSUPPORTED           # fp32 has no split-K path
-    assert f(256, 256, 8192, b.CYC_BF16_F32, A, B, C, None, b.CYC_FLAG_FIXED_K_ORDER) == b.CYC_ERR_INVALID_ARG
-    assert f(256, 256, 8192, b.CYC_BF16_F32, None, B, C, None, 0) == b.CYC_ERR_INVALID_ARG
+    stream = torch.cuda.current_stream().cuda_stream
+    shapes = [(512, 256, 8192, 81), (300, 264, 4112, 82)]
+    ops = []
+    for M, N, K, seed in shapes:                      # every tensor exists before the first measurement
+        w, (A, B) = _operands("bf16", M, N, K, seed, False)
+        ops.append((M, N, K, _dev(A, "bf16"), _dev(B, "bf16"), torch.empty((M, N), dtype=torch.float32, device="cuda")))
+    M, N, K, dA, dB, dC = ops[0]
+    assert b.cyc_recurrence_matmul_splitk_static(M, N, K, b.CYC_BF16_F32, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), stream, 0) == b.CYC_OK
+    torch.cuda.synchronize()
+    for M, N, K, dA, dB, dC in ops:
+        free0, pool0 = torch.cuda.mem_get_info()[0], _pool_bytes(b)
+        rc = b.cyc_recurrence_matmul_splitk_static(M, N, K, b.CYC_BF16_F32, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), stream, 0)
+        assert rc == b.CYC_OK
+        torch.cuda.synchronize()
+        assert b.last_device_status() == b.CYC_OK
+        assert torch.cuda.mem_get_info()[0] == free0, "free device memory changed across the call"
+        assert _pool_bytes(b) == pool0, "the library's pool grew or shrank across the call"
