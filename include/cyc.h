@@ -298,7 +298,14 @@ const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64_t K, int d
  *                        one owner per C_ij; what CYC_FLAG_FIXED_K_ORDER always selects;
  *   "k_sliced"           the k range of a block is cut into slices held by different CTA
  *                        pairs at the same time (k partly in space) and the slices' partial
- *                        sums are added in increasing k by a second kernel.
+ *                        sums are added in increasing k by a second kernel;
+ *   "output_stationary+k_sliced_tail"
+ *                        output-stationary, except that the blocks left over after the last
+ *                        full round of CTA pairs (which would keep only some pairs busy for
+ *                        a whole k loop) are cut into k-slices spread over all pairs; for
+ *                        each strip of such a block the pair that finishes last adds the
+ *                        slices' partial sums in increasing k inside the same kernel
+ *                        (assumes a B200's 74 CTA pairs; never under CYC_FLAG_FIXED_K_ORDER).
  * NULL if the arguments are invalid.  Host only, makes no CUDA call. */
 const char* cyc_schedule_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
                              const void* C, unsigned flags);

@@ -77,6 +77,23 @@ static int cuda_fail(cudaError_t e, const char* what) {
         if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
     } while (0)
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while the kernel before it on the stream
+// is still running; each kernel launched this way executes griddepcontrol.wait before it touches global memory.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 static int elem_bytes(int dtype) { return dtype == CYC_F32 ? 4 : (dtype == CYC_BF16_F32 ? 2 : 1); }
 
 struct Problem {
@@ -336,9 +353,97 @@ static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
     auto kern = umma_recurrence_kernel<KIND, B_MN, BN, STAGES>;
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), Sm::TOTAL)) return rc_;
     const long long grid = p.num_tiles < sms ? p.num_tiles : sms;
-    kern<<<static_cast<unsigned>(grid), UMMA_THREADS, Sm::TOTAL, st>>>(tmA, tmB, p);
-    CYC_CUDA(cudaGetLastError());
+    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(grid), UMMA_THREADS, Sm::TOTAL, st, tmA, tmB, p));
     g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
+// ------------------------------------------------------------------ sliced tail of the two-SM kernel
+// When the tile count leaves a remainder of at most half the CTA pairs, the remainder tiles are cut into k-slices
+// that all pairs work on first (see PairParams).  Not under CYC_FLAG_FIXED_K_ORDER: the flag promises one owner per
+// C_ij.  S slices of at least 8 k-blocks each; S * remainder <= pairs.
+struct TailPlan {
+    int S = 0, tiles = 0, kb = 0;
+};
+static TailPlan plan_tail(const Problem& q, long long num_tiles, long long pairs) {
+    TailPlan tp;
+    if ((q.flags & CYC_FLAG_FIXED_K_ORDER) || num_tiles <= pairs) return tp;
+    const int bk = 128 / elem_bytes(q.dtype);
+    const long long nkb = (q.K + bk - 1) / bk;
+    const long long rem = num_tiles % pairs;
+    if (rem == 0 || rem * 2 > pairs || nkb < 16) return tp;
+    long long S = std::min<long long>({pairs / rem, nkb / 8, 4});
+    if (S < 2) return tp;
+    tp.kb = static_cast<int>((nkb + S - 1) / S);
+    tp.S = static_cast<int>((nkb + tp.kb - 1) / tp.kb);  // no empty slice
+    tp.tiles = static_cast<int>(rem);
+    if (tp.S < 2) tp = TailPlan();
+    return tp;
+}
+
+// Scratch of the sliced tail: partial-sum slots for up to one slice per CTA pair and one counter per 32-row strip.
+// The counters must be zero when a launch starts and the kernel leaves them zero, so the memory is kept for the
+// life of the process -- one scratch per (device, stream), because launches on one stream are ordered and launches on
+// different streams are not.  At most kTailScratchMax are created per device; beyond that a launch simply runs the
+// plain schedule.  A device-side timeout may leave counters non-zero: cyc_last_device_status marks every scratch
+// dirty and the next use clears it on its stream.
+struct TailScratch {
+    int dev = -1;
+    cudaStream_t stream = nullptr;
+    uint8_t* ws = nullptr;
+    int* counters = nullptr;
+    bool dirty = false;
+};
+constexpr int kTailScratchMax = 8;
+constexpr size_t kTailCounterBytes = static_cast<size_t>(kCtaPairs) * 8 * sizeof(int);
+static std::mutex g_tail_mu;
+static TailScratch g_tail_scratch[64];
+static int g_tail_scratch_count = 0;
+
+static void tail_scratch_mark_dirty() {
+    std::lock_guard<std::mutex> lk(g_tail_mu);
+    for (int i = 0; i < g_tail_scratch_count; ++i) g_tail_scratch[i].dirty = true;
+}
+
+// returns CYC_OK with *out = nullptr when no scratch can be had (the caller then runs the plain schedule)
+static int tail_scratch_for(cudaStream_t st, TailScratch** out) {
+    *out = nullptr;
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); return CYC_OK; }
+    std::lock_guard<std::mutex> lk(g_tail_mu);
+    TailScratch* found = nullptr;
+    int on_dev = 0;
+    for (int i = 0; i < g_tail_scratch_count; ++i) {
+        if (g_tail_scratch[i].dev != dev) continue;
+        ++on_dev;
+        if (g_tail_scratch[i].stream == st) found = &g_tail_scratch[i];
+    }
+    if (!found) {
+        // creating one allocates and clears memory: not while the stream is being captured into a graph
+        if (cap != cudaStreamCaptureStatusNone || on_dev >= kTailScratchMax || g_tail_scratch_count >= 64) return CYC_OK;
+        void* mem = nullptr;
+        const size_t bytes = static_cast<size_t>(kCtaPairs) * PAIR_TILE_BYTES + kTailCounterBytes;
+        if (cudaMalloc(&mem, bytes) != cudaSuccess) { cudaGetLastError(); return CYC_OK; }
+        if (cudaMemset(static_cast<uint8_t*>(mem) + static_cast<size_t>(kCtaPairs) * PAIR_TILE_BYTES, 0, kTailCounterBytes) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(mem);
+            return CYC_OK;
+        }
+        found = &g_tail_scratch[g_tail_scratch_count++];
+        found->dev = dev;
+        found->stream = st;
+        found->ws = static_cast<uint8_t*>(mem);
+        found->counters = reinterpret_cast<int*>(found->ws + static_cast<size_t>(kCtaPairs) * PAIR_TILE_BYTES);
+        found->dirty = false;
+    }
+    if (found->dirty) {
+        if (cap != cudaStreamCaptureStatusNone) return CYC_OK;
+        CYC_CUDA(cudaMemsetAsync(found->counters, 0, kTailCounterBytes, st));
+        found->dirty = false;
+    }
+    *out = found;
     return CYC_OK;
 }
 
@@ -382,8 +487,18 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws 
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), SMEM)) return rc_;
     const long long max_pairs = sms / 2;
     const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
-    kern<<<static_cast<unsigned>(2 * pairs), UMMA_THREADS, SMEM, st>>>(tmA, tmB, tmC, p);
-    CYC_CUDA(cudaGetLastError());
+    if (!ws && pairs <= kCtaPairs) {
+        const TailPlan tp = plan_tail(q, p.num_tiles, pairs);
+        if (tp.S > 1) {
+            TailScratch* sc = nullptr;
+            if (int rc_ = tail_scratch_for(st, &sc)) return rc_;
+            if (sc) {
+                p.tail_S = tp.S; p.tail_tiles = tp.tiles; p.tail_kb = tp.kb;
+                p.tail_ws = sc->ws; p.tail_counters = sc->counters;
+            }
+        }
+    }
+    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(2 * pairs), UMMA_THREADS, SMEM, st, tmA, tmB, tmC, p));
     g_launches.fetch_add(1);
     return CYC_OK;
 }
@@ -434,9 +549,8 @@ static int launch_splitk(const Problem& q, cudaStream_t st, int sms, void* ws, c
         const long long work = (vec4 ? plane / 4 : plane) * q.batch;
         long long blocks = (work + 127) / 128;  // short kernel: spread the work over as many SMs as possible
         if (blocks > 16ll * sms) blocks = 16ll * sms;
-        splitk_reduce_kernel<Out><<<static_cast<unsigned>(blocks), 128, 0, st>>>(static_cast<const Out*>(ws), static_cast<Out*>(q.C),
-                                                                                plane, q.sC, plan.S, q.batch, vec4);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = launch_pdl(splitk_reduce_kernel<Out>, static_cast<unsigned>(blocks), 128, 0, st, static_cast<const Out*>(ws),
+                                   static_cast<Out*>(q.C), plane, q.sC, plan.S, q.batch, vec4);
         if (e != cudaSuccess) rc = cuda_fail(e, "splitk_reduce_kernel launch");
         else g_launches.fetch_add(1);
     }
@@ -477,8 +591,7 @@ static int launch_pair_tall_cfg(const Problem& q, cudaStream_t st, int sms) {
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), TALL_SMEM_BYTES)) return rc_;
     const long long max_pairs = sms / 2;
     const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
-    kern<<<static_cast<unsigned>(2 * pairs), TALL_THREADS, TALL_SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
-    CYC_CUDA(cudaGetLastError());
+    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(2 * pairs), TALL_THREADS, TALL_SMEM_BYTES, st, tmA, tmB, tmC, p));
     g_launches.fetch_add(1);
     return CYC_OK;
 }
@@ -511,8 +624,7 @@ static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), X3_SMEM_BYTES)) return rc_;
     const long long max_pairs = sms / 2;
     const long long pairs = p.num_tiles < max_pairs ? p.num_tiles : max_pairs;
-    kern<<<static_cast<unsigned>(2 * pairs), X3_THREADS, X3_SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
-    CYC_CUDA(cudaGetLastError());
+    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(2 * pairs), X3_THREADS, X3_SMEM_BYTES, st, tmA, tmB, tmC, p));
     g_launches.fetch_add(1);
     return CYC_OK;
 }
@@ -600,8 +712,7 @@ static int trsm_diag(const TrsmPlan& t, long long b, unsigned mask) {
     p.rows = static_cast<int>(t.n - b * t.T < t.T ? t.n - b * t.T : t.T);
     p.mask = mask;
     const long long blocks = (t.m + TRSM_CW - 1) / TRSM_CW;
-    trsm_diag_kernel<<<static_cast<unsigned>(blocks), TRSM_THREADS, TRSM_SMEM_BYTES, t.st>>>(p);
-    CYC_CUDA(cudaGetLastError());
+    CYC_CUDA(launch_pdl(trsm_diag_kernel, static_cast<unsigned>(blocks), TRSM_THREADS, TRSM_SMEM_BYTES, t.st, p));
     g_launches.fetch_add(1);
     return CYC_OK;
 }
@@ -637,8 +748,7 @@ static int launch_fa2(long long batch, long long N, long long M, const void* Q, 
     if (int rc_ = status_word(&p.status)) return rc_;
     auto kern = fa2_kernel<D>;
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), Fa2Smem<D>::TOTAL)) return rc_;
-    kern<<<static_cast<unsigned>(batch * p.tiles_q), FA2_THREADS, Fa2Smem<D>::TOTAL, st>>>(tmQ, tmK, tmV, p);
-    CYC_CUDA(cudaGetLastError());
+    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(batch * p.tiles_q), FA2_THREADS, Fa2Smem<D>::TOTAL, st, tmQ, tmK, tmV, p));
     g_launches.fetch_add(1);
     return CYC_OK;
 }
@@ -1046,8 +1156,8 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
                 if (rc) break;
                 const long long work = pstride / 4;
                 long long blocks = std::min<long long>((work + 127) / 128, 16ll * di.sms);
-                splitk_reduce_kernel<float><<<static_cast<unsigned>(blocks), 128, 0, st>>>(W, W, pstride, pstride, planes, 1, 1);
-                cudaError_t e = cudaGetLastError();
+                cudaError_t e = launch_pdl(splitk_reduce_kernel<float>, static_cast<unsigned>(blocks), 128, 0, st, static_cast<const float*>(W), W,
+                                           pstride, pstride, planes, 1ll, 1);
                 if (e != cudaSuccess) { rc = cuda_fail(e, "splitk_reduce_kernel"); break; }
                 g_launches.fetch_add(1);
                 planes = 1;
@@ -1059,8 +1169,7 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
         d.lda = n; d.ldw = w; d.ldl = n;
         d.rows = static_cast<int>(w);
         d.zero_upper = in_place ? 0 : 1;
-        chol_diag_kernel<<<1, CHOL_THREADS, CHOL_SMEM_BYTES, st>>>(d);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = launch_pdl(chol_diag_kernel, 1u, CHOL_THREADS, CHOL_SMEM_BYTES, st, d);
         if (e != cudaSuccess) { rc = cuda_fail(e, "chol_diag_kernel"); break; }
         g_launches.fetch_add(1);
         if (below > 0) {
@@ -1072,8 +1181,7 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
             p.n = static_cast<int>(n); p.m = static_cast<int>(below);
             p.r0 = static_cast<int>(c0); p.rows = static_cast<int>(w);
             p.mask = planes ? ((1u << planes) - 1u) : 0u;
-            trsm_diag_kernel<<<static_cast<unsigned>((below + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, st>>>(p);
-            e = cudaGetLastError();
+            e = launch_pdl(trsm_diag_kernel, static_cast<unsigned>((below + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, st, p);
             if (e != cudaSuccess) { rc = cuda_fail(e, "trsm_diag_kernel"); break; }
             g_launches.fetch_add(1);
             if (!in_place) {  // zeros above the diagonal: the block row to the right of the diagonal tile
@@ -1105,6 +1213,7 @@ extern "C" int cyc_last_device_status(void* stream, int* out) {
     CYC_CUDA(cudaMemcpyFromSymbol(&word, g_device_status, sizeof word));
     if (word != 0) {
         const int zero = 0;
+        tail_scratch_mark_dirty();  // a kernel that gave up may have left strip counters of the sliced tail non-zero
         CYC_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero));
         snprintf(g_err, sizeof g_err, "device wait ran out (code 0x%x)", word);
     }
@@ -1132,7 +1241,13 @@ extern "C" const char* cyc_schedule_for(int64_t batch, int64_t M, int64_t N, int
     if (batch <= 0 || M <= 0 || N <= 0 || K <= 0) return nullptr;
     Problem q{batch, M, N, K, dtype, A, B, const_cast<void*>(C), M * K, K * N, M * N, flags};
     if (validate(q) != CYC_OK) return nullptr;
-    return choose(q) == FAM_UMMA_SPLITK ? "k_sliced" : "output_stationary";
+    const Family fam = choose(q);
+    if (fam == FAM_UMMA_SPLITK) return "k_sliced";
+    if (fam == FAM_UMMA_PAIR) {
+        const long long tiles = q.batch * ((q.M + 255) / 256) * ((q.N + 255) / 256);
+        if (plan_tail(q, tiles, kCtaPairs).S > 1) return "output_stationary+k_sliced_tail";
+    }
+    return "output_stationary";
 }
 
 extern "C" int64_t cyc_launch_count(void) { return g_launches.load(); }

@@ -126,6 +126,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     const int n0 = qt * FA2_BM;
     const int T = (p.M + FA2_BN - 1) / FA2_BN;  // key tiles
 
+    ptx::grid_launch_dependents();
     if (threadIdx.x == 0) {
         ptx::mbar_init(&ctl->q_full, 1);
         for (int s = 0; s < 2; ++s) {
@@ -156,6 +157,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; nothing it wrote is read before it ends
             ptx::mbar_arrive_expect_tx(&ctl->q_full, Sm::Q_BYTES);
 #pragma unroll
             for (int kb = 0; kb < D / 64; ++kb) ptx::tma_load_3d(sQ + kb * Sm::SLAB, &tmQ, &ctl->q_full, kb * 64, n0, b);

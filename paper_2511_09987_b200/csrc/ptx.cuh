@@ -15,6 +15,14 @@ __device__ __forceinline__ uint32_t lane_id() {
     return l;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// The library launches its kernels with programmatic stream serialisation: a kernel may be scheduled while the
+// kernel before it in the stream is still running.  grid_dependency_wait() returns once that kernel has completed and
+// its memory is visible -- nothing a previous kernel may have written (or may still read) is touched before it;
+// grid_launch_dependents() tells the scheduler that the NEXT kernel may start occupying SMs as they become free.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

@@ -5,6 +5,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "ptx.cuh"
+
 namespace cyc {
 
 // ws: [batch][S][plane] ; C: [batch] planes with stride sC ; plane = M*N elements.
@@ -13,6 +15,9 @@ namespace cyc {
 template <typename T>
 __global__ void __launch_bounds__(128) splitk_reduce_kernel(const T* ws, T* C, long long plane, long long sC, int S,
                                                             long long batch, int vec4) {
+    // launched with programmatic stream serialisation: only the launch itself overlaps the previous kernel
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
     const long long per_batch = vec4 ? plane / 4 : plane;
     const long long total = per_batch * batch;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;

@@ -22,6 +22,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "ptx.cuh"
+
 namespace cyc {
 
 struct TrsmDiagParams {
@@ -116,6 +118,9 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
     float(*Lt)[TRSM_LT_PITCH] = reinterpret_cast<float(*)[TRSM_LT_PITCH]>(Lb + TRSM_NBLK * TRSM_BLK);
     float* dinv = reinterpret_cast<float*>(Lt) + TRSM_SB * TRSM_LT_PITCH;
 
+    // launched with programmatic stream serialisation: only the launch itself overlaps the previous kernel
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c = blockIdx.x * TRSM_CW + lane;
     const bool col_ok = c < p.m;

@@ -153,6 +153,7 @@ umma_recurrence_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     const int lane = threadIdx.x & 31;
     const int num_kb = (p.K + BK - 1) / BK;
 
+    ptx::grid_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&ctl->full[s], 1);
@@ -183,6 +184,7 @@ umma_recurrence_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
+            ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; nothing it wrote is read before it ends
             for (long long t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
                 int b, tm, tn;
                 umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);

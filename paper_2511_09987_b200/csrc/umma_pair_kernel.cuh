@@ -34,7 +34,53 @@ struct PairParams {
     // to plane e of the output (a workspace that a second kernel adds up).  split_k = 1: the plain recurrence.
     int split_k = 1;
     int kb_per_slice = 0;
+    // Sliced tail (umma_pair_kernel only; never under the fixed-k-order flag): when the tile count is not a multiple
+    // of the number of CTA pairs, the last `tail_tiles` tiles of the list would occupy only some pairs for one more
+    // whole k loop.  Instead each of them is cut into `tail_S` k-slices of `tail_kb` k-blocks, the tail_tiles * tail_S
+    // slices go to different pairs as their FIRST work item, and for every 32-row strip of such a tile the warp that
+    // finishes its slice last adds the other slices' partial sums (parked in `tail_ws`) in increasing k and exports
+    // C.  Nobody waits for anybody: `tail_counters` (one per strip, zero between launches) tells a warp whether it
+    // is the last.
+    int tail_S = 0;
+    int tail_tiles = 0;
+    int tail_kb = 0;
+    void* tail_ws = nullptr;
+    int* tail_counters = nullptr;
 };
+
+// one item of a pair's work list: a tile (or one k-slice of a tail tile) with its k-block range
+struct PairWork {
+    long long tile;  // index into the tile list (for split_k: the (problem, slice) entry)
+    int kb0, nkb;
+    int slice;       // k-slice of a tail tile, or -1
+    int tail_index;  // which tail tile
+};
+
+// i-th work item of pair `pair` (of `num_pairs`); false when the pair's list is exhausted
+__device__ __forceinline__ bool pair_work_item(const PairParams& p, int num_kb, long long pair, long long num_pairs, int i, PairWork& w) {
+    long long full_tiles = p.num_tiles;
+    if (p.tail_S > 1) {
+        full_tiles = p.num_tiles - p.tail_tiles;
+        const long long units = static_cast<long long>(p.tail_tiles) * p.tail_S;
+        if (pair < units) {
+            if (i == 0) {
+                w.tail_index = static_cast<int>(pair / p.tail_S);
+                w.slice = static_cast<int>(pair - static_cast<long long>(w.tail_index) * p.tail_S);
+                w.tile = full_tiles + w.tail_index;
+                w.kb0 = w.slice * p.tail_kb;
+                w.nkb = min(p.tail_kb, num_kb - w.kb0);
+                return true;
+            }
+            --i;
+        }
+    }
+    w.tile = pair + static_cast<long long>(i) * num_pairs;
+    w.slice = -1;
+    w.tail_index = 0;
+    w.kb0 = 0;
+    w.nkb = num_kb;
+    return w.tile < full_tiles;
+}
 
 // k-block range [kb0, kb0 + nkb) of tile-list entry `e`, and the operand batch index it reads from
 __device__ __forceinline__ void pair_k_range(const PairParams& p, int num_kb, int e, int& b, int& kb0, int& nkb) {
@@ -51,6 +97,8 @@ constexpr int PAIR_STAGE_A = 128 * 128;
 constexpr int PAIR_STAGE_B = 128 * 128;
 constexpr int PAIR_STAGE_BYTES = PAIR_STAGE_A + PAIR_STAGE_B;
 constexpr int PAIR_STAGING_BYTES = 4 * 2 * 4096;  // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
+constexpr int PAIR_STRIP_BYTES = 32 * 256 * 4;     // partial sums of one 32-row strip of a 256 x 256 tile
+constexpr int PAIR_TILE_BYTES = 8 * PAIR_STRIP_BYTES;
 
 template <int STAGES>
 constexpr int pair_smem_bytes() { return STAGES * PAIR_STAGE_BYTES + PAIR_STAGING_BYTES + 1024 + 1024; }
@@ -80,6 +128,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const long long num_pairs = gridDim.x >> 1;
     const int num_kb = (p.K + BK - 1) / BK;
 
+    ptx::grid_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&ctl->full[s], 1);
@@ -114,10 +163,13 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             long long issued = 0;
             bool ok = true;
             const uint32_t full0 = ptx::mapa_u32(ptx::smem_u32(&ctl->full[0]), 0);  // the leader's full[] barriers
-            for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
+            ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; operands may not be read before it ends
+            PairWork w;
+            for (int item = 0; ok && pair_work_item(p, num_kb, pair, num_pairs, item, w); ++item) {
                 int e, tm, tn, b, kb0, nkb;
-                umma_tile_coord(t, p.tiles_m, p.tiles_n, e, tm, tn);
+                umma_tile_coord(w.tile, p.tiles_m, p.tiles_n, e, tm, tn);
                 pair_k_range(p, num_kb, e, b, kb0, nkb);
+                if (w.slice >= 0) { kb0 = w.kb0; nkb = w.nkb; }
                 const int m0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF;      // this CTA's 128 rows of cells
                 const int n0 = tn * PAIR_BN + static_cast<int>(rank) * PAIR_HALF;  // this CTA's half of the B tile
                 for (int kb = kb0; kb < kb0 + nkb; ++kb) {
@@ -158,15 +210,17 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t phase = 0;
             int local = 0;
             bool ok = true;
-            for (long long t = pair; t < p.num_tiles && ok; t += num_pairs, ++local) {
+            PairWork w;
+            for (; ok && pair_work_item(p, num_kb, pair, num_pairs, local, w); ++local) {
                 const int ab = local & 1;
                 const uint32_t acc_phase = (local >> 1) & 1;
                 if (!umma_wait(&ctl->acc_empty[ab], acc_phase ^ 1, ctl, p.status, 2)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * PAIR_BN);
                 int e, tm, tn, b, kb0, nkb;
-                umma_tile_coord(t, p.tiles_m, p.tiles_n, e, tm, tn);
+                umma_tile_coord(w.tile, p.tiles_m, p.tiles_n, e, tm, tn);
                 pair_k_range(p, num_kb, e, b, kb0, nkb);
+                if (w.slice >= 0) nkb = w.nkb;
                 for (int kb = 0; kb < nkb; ++kb) {  // the first k-block of the slice starts from zero
                     if (!umma_wait(&ctl->full[stage], phase, ctl, p.status, 3)) { ok = false; break; }
                     ptx::tc_fence_after();
@@ -191,29 +245,28 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------------------ epilogue: C_ij <- [i,k_end]_C (both CTAs)
         const int q = warp & 3;
         uint8_t* my_stage = staging + q * 8192;
+        const uint32_t lane_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
         int local = 0, sbuf = 0;
         bool ok = true;
-        for (long long t = pair; t < p.num_tiles && ok; t += num_pairs, ++local) {
+        PairWork w;
+        for (; ok && pair_work_item(p, num_kb, pair, num_pairs, local, w); ++local) {
             const int ab = local & 1;
             const uint32_t acc_phase = (local >> 1) & 1;
             int b, tm, tn;
-            umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);
+            umma_tile_coord(w.tile, p.tiles_m, p.tiles_n, b, tm, tn);
             if (!umma_wait(&ctl->acc_full[ab], acc_phase, ctl, p.status, 4)) { ok = false; break; }
             ptx::tc_fence_after();
             const int row0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF + q * 32;
             const int row = row0 + lane;
             Out* crow = static_cast<Out*>(p.C) + static_cast<long long>(b) * p.sC + static_cast<long long>(row) * p.N;
-#pragma unroll 1
-            for (int c0 = 0; c0 < PAIR_BN; c0 += 32) {
+            const int nchunks = min(PAIR_BN / 32, (p.N - tn * PAIR_BN + 31) / 32);  // 32-column pieces inside C
+            // one 32 x 32 piece of C (this lane's row, 32 consecutive columns starting at c0) leaves the SM
+            auto export_piece = [&](const uint32_t (&v)[32], int c0) {
                 const int col = tn * PAIR_BN + c0;
-                if (col >= p.N) break;  // uniform over the warp
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(ab * PAIR_BN + c0), v);
                 if (p.tma_store) {
                     uint8_t* buf = my_stage + sbuf * 4096;
                     if (lane == 0) ptx::tma_store_wait_read<1>();  // the store that last used this buffer has read it
                     __syncwarp();
-                    ptx::tmem_ld_wait();
                     // 32 rows x 128 B, 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
 #pragma unroll
                     for (int g = 0; g < 8; ++g)
@@ -225,18 +278,90 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         ptx::tma_store_commit();
                     }
                     sbuf ^= 1;
-                } else {
-                    ptx::tmem_ld_wait();
-                    if (row < p.M) {
+                } else if (row < p.M) {
 #pragma unroll
-                        for (int g = 0; g < 32; ++g)
-                            if (col + g < p.N) reinterpret_cast<uint32_t*>(crow)[col + g] = v[g];
+                    for (int g = 0; g < 32; ++g)
+                        if (col + g < p.N) reinterpret_cast<uint32_t*>(crow)[col + g] = v[g];
+                }
+            };
+            if (w.slice < 0) {
+                // whole tile: the tensor-memory read of the next piece is in flight while this one is staged and stored
+                uint32_t va[32], vb[32];
+                ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN), va);
+#pragma unroll 1
+                for (int c = 0; c < nchunks; c += 2) {
+                    ptx::tmem_ld_wait();
+                    if (c + 1 < nchunks) ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + (c + 1) * 32), vb);
+                    export_piece(va, c * 32);
+                    if (c + 1 < nchunks) {
+                        ptx::tmem_ld_wait();
+                        if (c + 2 < nchunks) ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + (c + 2) * 32), va);
+                        export_piece(vb, (c + 1) * 32);
                     }
                 }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(&ctl->acc_empty[ab], 0);
+                continue;
+            }
+            // k-slice of a tail tile: park this strip's partial sums (16-byte piece g of a lane's 32 values at
+            // (g * 32 + lane) * 16, so that one store instruction writes 512 contiguous bytes), give the accumulator
+            // back, then find out whether the other slices of the strip are already there
+            const int strip = static_cast<int>(rank) * 4 + q;
+            uint8_t* tile_ws = static_cast<uint8_t*>(p.tail_ws) + static_cast<size_t>(w.tail_index) * p.tail_S * PAIR_TILE_BYTES;
+            uint8_t* mine = tile_ws + static_cast<size_t>(w.slice) * PAIR_TILE_BYTES + strip * PAIR_STRIP_BYTES;
+#pragma unroll 1
+            for (int c = 0; c < nchunks; ++c) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + c * 32), v);
+                ptx::tmem_ld_wait();
+                uint4* dst = reinterpret_cast<uint4*>(mine + c * 4096);
+#pragma unroll
+                for (int g = 0; g < 8; ++g) dst[g * 32 + lane] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
             }
             ptx::tc_fence_before();
+            __threadfence();  // this lane's partial sums are out before the warp is counted
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(&ctl->acc_empty[ab], 0);
+            int arrived = 0;
+            if (lane == 0) {
+                ptx::mbar_arrive_cluster(&ctl->acc_empty[ab], 0);
+                arrived = atomicAdd(&p.tail_counters[w.tail_index * 8 + strip], 1);
+            }
+            arrived = __shfl_sync(0xffffffffu, arrived, 0);
+            if (arrived != p.tail_S - 1) continue;  // a later warp finishes this strip
+            // every slice of the strip has been parked: C_ij = their sum in increasing k (the slice at hand is read back
+            // like the others; the read of the next piece is in flight while this one is added)
+            __threadfence();
+            if (lane == 0) p.tail_counters[w.tail_index * 8 + strip] = 0;  // zero again for the next launch
+            const uint8_t* strip_ws = tile_ws + strip * PAIR_STRIP_BYTES;
+            const int pieces = nchunks * p.tail_S;
+            auto fetch = [&](int i, uint32_t (&o)[32]) {
+                const int c = i / p.tail_S, sl = i - c * p.tail_S;
+                const uint4* src = reinterpret_cast<const uint4*>(strip_ws + static_cast<size_t>(sl) * PAIR_TILE_BYTES + c * 4096);
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const uint4 x = __ldcg(src + g * 32 + lane);  // written by another SM: read through L2
+                    o[4 * g] = x.x; o[4 * g + 1] = x.y; o[4 * g + 2] = x.z; o[4 * g + 3] = x.w;
+                }
+            };
+            uint32_t cur[32], nxt[32], sum[32] = {};
+            fetch(0, cur);
+#pragma unroll 1
+            for (int i = 0; i < pieces; ++i) {
+                if (i + 1 < pieces) fetch(i + 1, nxt);
+                const int c = i / p.tail_S, sl = i - c * p.tail_S;
+#pragma unroll
+                for (int g = 0; g < 32; ++g) {
+                    Out x, y;
+                    memcpy(&x, &cur[g], 4);
+                    memcpy(&y, &sum[g], 4);
+                    y = sl == 0 ? x : y + x;
+                    memcpy(&sum[g], &y, 4);
+                }
+                if (sl == p.tail_S - 1) export_piece(sum, c * 32);
+#pragma unroll
+                for (int g = 0; g < 32; ++g) cur[g] = nxt[g];
+            }
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
         __syncwarp();

@@ -48,6 +48,7 @@ umma_pair_tall_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const long long num_pairs = gridDim.x >> 1;
     const int num_kb = (p.K + BK - 1) / BK;
 
+    ptx::grid_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&ctl->full[s], 1);
@@ -80,6 +81,7 @@ umma_pair_tall_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             long long issued = 0;
             bool ok = true;
             const uint32_t full0 = ptx::mapa_u32(ptx::smem_u32(&ctl->full[0]), 0);  // the leader's full[] barriers
+            ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; nothing it wrote is read before it ends
             for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
                 int b, tm, tn;
                 umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);

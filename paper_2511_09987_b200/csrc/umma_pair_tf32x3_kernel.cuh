@@ -80,6 +80,7 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const long long num_pairs = gridDim.x >> 1;
     const int num_kb = (p.K + BK - 1) / BK;
 
+    ptx::grid_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&ctl->full[s], 1);
@@ -114,6 +115,7 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
+            ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; nothing it wrote is read before it ends
             // A is streamed from HBM exactly once, and the ring is only three stages deep: a second cursor runs
             // X3_PREFETCH k-blocks ahead and asks L2 for the A tiles, so the copies into the ring hit L2
             long long pf_t = pair;

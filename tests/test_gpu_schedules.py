@@ -26,7 +26,7 @@ def _w(dtype, M, N, K, seed, col=False, fixed=False):
     return inputs.Workload("sched", dtype, M, N, K, seed, 1, col, fixed, ("uniform", -1.0, 1.0), ("normal", 1.0))
 
 
-INT8_CASES = [(130, 136, 160, True), (100, 272, 144, False), (260, 264, 272, True), (300, 520, 400, False), (515, 260, 130, True)]
+INT8_CASES = [(130, 136, 160, True), (100, 272, 144, False), (260, 264, 272, True), (300, 528, 400, False), (515, 260, 144, True)]
 
 
 @pytest.mark.parametrize("M,N,K,col", INT8_CASES)
@@ -58,7 +58,7 @@ def test_strict_fp32_kernel_equals_the_output_stationary_walker_bit_for_bit(M, N
     assert (np.abs(C.astype(np.float64) - ref) <= TOL["f32"] * S).all()
 
 
-@pytest.mark.parametrize("M,N,K", [(130, 136, 160), (260, 264, 272), (515, 260, 136)])
+@pytest.mark.parametrize("M,N,K", [(130, 136, 160), (260, 264, 272), (515, 264, 136)])
 def test_bf16_tensor_core_kernels_against_the_output_stationary_walker(M, N, K):
     from paper_2511_09987_b200 import binding
     w = _w("bf16", M, N, K, seed=80 + M)
@@ -85,6 +85,54 @@ def test_k_sliced_schedule_equals_the_walkers_for_int8():
     rows = np.array([0, 127, 128, 259])
     os_rows = oracle.walk("os_cannon", "i8", A[rows], B, b_col_major=True)
     assert (C[rows] == os_rows).all()
+
+
+TAIL_CASES = [
+    # dtype, batch, M, N, K, col   -- tile counts that leave a remainder of at most half the 74 CTA pairs
+    ("i8", 1, 2500, 2600, 2048, True),      # 10 x 11 = 110 tiles, remainder 36: two slices of 8 k-blocks
+    ("bf16", 1, 2500, 2344, 1032, False),   # 100 tiles, remainder 26; 17 k-blocks: slices of 9 and 8
+    ("i8", 3, 1280, 1536, 4096, False),     # 3 x 30 tiles, remainder 16: four slices of 8 k-blocks
+    ("bf16", 1, 2304, 2560, 1096, True),    # 90 tiles, remainder 16; 18 k-blocks, the last ragged: slices of 9
+]
+
+
+@pytest.mark.parametrize("dtype,batch,M,N,K,col", TAIL_CASES)
+def test_sliced_tail_every_output(dtype, batch, M, N, K, col):
+    """The leftover tiles of the last round are cut into k-slices spread over all CTA pairs and summed in increasing
+    k by whichever pair finishes a strip last: int8 must equal the walkers bit for bit, bf16 stay within tolerance, and
+    the result must not depend on which pair was last (two launches, two streams, identical bits)."""
+    import torch
+    from paper_2511_09987_b200 import binding
+    dist = ("int8",) if dtype == "i8" else ("uniform", -1.0, 1.0)
+    w = inputs.Workload("tail", dtype, M, N, K, 95 + batch, batch, col, False, dist, dist)
+    assert binding.kernel_for(batch, M, N, K, dtype, b_col_major=col) == "tcgen05_pair"
+    assert binding.schedule_for(batch, M, N, K, dtype, b_col_major=col) == "output_stationary+k_sliced_tail"
+    assert binding.schedule_for(batch, M, N, K, dtype, b_col_major=col, fixed_k_order=True) == "output_stationary"
+    A, B = inputs.make_operands(w)
+    C = gpu_run(w, A, B)
+    C2 = gpu_run(w, A, B)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        C3 = gpu_run(w, A, B)
+    assert C.tobytes() == C2.tobytes() == C3.tobytes()
+    C1 = gpu_run(w, A, B, fixed_k_order=True)          # one owner per output: the plain schedule
+    for b in range(batch):
+        Ab, Bb, Cb, C1b = (A, B, C, C1) if batch == 1 else (A[b], B[b], C[b], C1[b])
+        ref = oracle.collapsed(dtype, Ab, Bb, b_col_major=col, threads=16)
+        if dtype == "i8":
+            assert Cb.tobytes() == ref.tobytes()
+            assert C1b.tobytes() == ref.tobytes()
+        else:
+            S, _ = oracle.abs_sum_rows(dtype, Ab, Bb, b_col_major=col, threads=16)
+            assert (np.abs(Cb.astype(np.float64) - ref) <= TOL[dtype] * S).all()
+            assert (np.abs(C1b.astype(np.float64) - ref) <= TOL[dtype] * S).all()
+
+
+def test_headline_int8_configuration_uses_the_sliced_tail():
+    from paper_2511_09987_b200 import binding
+    assert binding.schedule_for(1, 4096, 4096, 4096, "i8", b_col_major=True) == "output_stationary+k_sliced_tail"
+    assert binding.schedule_for(1024, 256, 256, 256, "bf16") == "output_stationary"     # remainder 62 of 74: no slicing
+    assert binding.schedule_for(1, 8192, 8192, 8192, "bf16") == "output_stationary"     # tall tiles
 
 
 def test_caller_supplied_result_is_checked_before_it_reaches_a_kernel():

@@ -11,6 +11,8 @@ CASES = [
     # name, dtype, M, N, K, batch, col, fixed, launches
     ("3xtf32", "f32", 65536, 256, 256, 1, False, False, 3000),
     ("pair_int8", "i8", 4096, 4096, 1024, 1, True, False, 3000),
+    ("pair_int8_sliced_tail", "i8", 4096, 4096, 4096, 1, True, False, 2000),
+    ("pair_bf16_sliced_tail", "bf16", 2560, 2560, 1024, 1, False, False, 2000),
     ("pair_bf16_batched", "bf16", 256, 256, 256, 256, False, False, 3000),
     ("tall_bf16", "bf16", 4608, 4096, 6144, 1, False, False, 300),
     ("splitk_bf16", "bf16", 512, 512, 16384, 1, False, False, 3000),
