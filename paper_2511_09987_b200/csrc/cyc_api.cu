@@ -361,7 +361,7 @@ static int launch_umma_cfg(const Problem& q, cudaStream_t st, int sms) {
 // ------------------------------------------------------------------ sliced tail of the two-SM kernel
 // When the tile count leaves a remainder of at most half the CTA pairs, the remainder tiles are cut into k-slices
 // that all pairs work on first (see PairParams).  Not under CYC_FLAG_FIXED_K_ORDER: the flag promises one owner per
-// C_ij.  S slices of at least 8 k-blocks each; S * remainder <= pairs.
+// C_ij.  S slices (at most 4) of a minimum length each; S * remainder <= pairs.
 struct TailPlan {
     int S = 0, tiles = 0, kb = 0;
 };
@@ -371,8 +371,11 @@ static TailPlan plan_tail(const Problem& q, long long num_tiles, long long pairs
     const int bk = 128 / elem_bytes(q.dtype);
     const long long nkb = (q.K + bk - 1) / bk;
     const long long rem = num_tiles % pairs;
-    if (rem == 0 || rem * 2 > pairs || nkb < 16) return tp;
-    long long S = std::min<long long>({pairs / rem, nkb / 8, 4});
+    // bf16 and int8 only: measured on the fp32 (3xTF32) kernel, whose tiles are short, the parked slices cost more than
+    // the idle pairs (64 against 50 microseconds on the 65536 x 256 x 256 problem)
+    const long long min_kb = 8;  // a slice must amortise its own export
+    if (q.dtype == CYC_F32 || rem == 0 || rem * 2 > pairs || nkb < 2 * min_kb) return tp;
+    long long S = std::min<long long>({pairs / rem, nkb / min_kb, 4});
     if (S < 2) return tp;
     tp.kb = static_cast<int>((nkb + S - 1) / S);
     tp.S = static_cast<int>((nkb + tp.kb - 1) / tp.kb);  // no empty slice
@@ -599,11 +602,13 @@ static int launch_pair_tall_cfg(const Problem& q, cudaStream_t st, int sms) {
 template <bool B_MN>
 static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
     CUtensorMap tmA, tmB, tmC;
-    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, 32, PAIR_HALF);
+    // K-major tiles: rows of X3_BK fp32 (128 or 64 bytes) under the swizzle of that width
+    const CUtensorMapSwizzle ksw = X3_BK == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, q.batch, lda_of(q), q.sA, X3_BK, PAIR_HALF, ksw);
     if (rc) return rc;
     // fp32 B stored [K][N] feeds the MMA column-contiguous: 32-byte-chunk swizzle (see umma_smem_desc)
-    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, ldb_of(q), q.sB, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
-    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, ldb_of(q), q.sB, 32, PAIR_HALF);
+    if (B_MN) rc = make_map(&tmB, q.dtype, q.B, q.N, q.K, q.batch, ldb_of(q), q.sB, 32, X3_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+    else rc = make_map(&tmB, q.dtype, q.B, q.K, q.N, q.batch, ldb_of(q), q.sB, X3_BK, PAIR_HALF, ksw);
     if (rc) return rc;
     PairParams p;
     p.tma_store = (reinterpret_cast<uintptr_t>(q.C) % 16 == 0 && q.N % 4 == 0 && (q.batch == 1 || q.sC % 4 == 0)) ? 1 : 0;

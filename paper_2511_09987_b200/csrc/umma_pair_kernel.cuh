@@ -100,6 +100,69 @@ constexpr int PAIR_STAGING_BYTES = 4 * 2 * 4096;  // 4 epilogue warps x 2 buffer
 constexpr int PAIR_STRIP_BYTES = 32 * 256 * 4;     // partial sums of one 32-row strip of a 256 x 256 tile
 constexpr int PAIR_TILE_BYTES = 8 * PAIR_STRIP_BYTES;
 
+// k-slice of a tail tile, seen from the warp that owns 32-row strip `strip` (0..7 over the pair) of the tile: park
+// the strip's partial sums (16-byte piece g of a lane's 32 values at (g * 32 + lane) * 16, so that one store instruction
+// writes 512 contiguous bytes), give the accumulator at `acc_taddr` back, and find out whether the other slices of the
+// strip are already there.  If so, C_ij = the slices' sums added in increasing k (the slice at hand is read back like
+// the others; the read of the next piece is in flight while this one is added), handed piece by piece to
+// `export_piece(values, first column within the tile)`.
+template <typename Out, typename ExportFn>
+__device__ __forceinline__ void pair_tail_strip(const PairParams& p, const PairWork& w, int strip, uint32_t acc_taddr, int nchunks, int lane,
+                                                uint64_t* acc_empty, ExportFn&& export_piece) {
+    uint8_t* tile_ws = static_cast<uint8_t*>(p.tail_ws) + static_cast<size_t>(w.tail_index) * p.tail_S * PAIR_TILE_BYTES;
+    uint8_t* mine = tile_ws + static_cast<size_t>(w.slice) * PAIR_TILE_BYTES + strip * PAIR_STRIP_BYTES;
+#pragma unroll 1
+    for (int c = 0; c < nchunks; ++c) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(acc_taddr + static_cast<uint32_t>(c * 32), v);
+        ptx::tmem_ld_wait();
+        uint4* dst = reinterpret_cast<uint4*>(mine + c * 4096);
+#pragma unroll
+        for (int g = 0; g < 8; ++g) dst[g * 32 + lane] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+    }
+    ptx::tc_fence_before();
+    __threadfence();  // this lane's partial sums are out before the warp is counted
+    __syncwarp();
+    int arrived = 0;
+    if (lane == 0) {
+        ptx::mbar_arrive_cluster(acc_empty, 0);
+        arrived = atomicAdd(&p.tail_counters[w.tail_index * 8 + strip], 1);
+    }
+    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+    if (arrived != p.tail_S - 1) return;  // a later warp finishes this strip
+    __threadfence();
+    if (lane == 0) p.tail_counters[w.tail_index * 8 + strip] = 0;  // zero again for the next launch
+    const uint8_t* strip_ws = tile_ws + strip * PAIR_STRIP_BYTES;
+    const int pieces = nchunks * p.tail_S;
+    auto fetch = [&](int i, uint32_t (&o)[32]) {
+        const int c = i / p.tail_S, sl = i - c * p.tail_S;
+        const uint4* src = reinterpret_cast<const uint4*>(strip_ws + static_cast<size_t>(sl) * PAIR_TILE_BYTES + c * 4096);
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            const uint4 x = __ldcg(src + g * 32 + lane);  // written by another SM: read through L2
+            o[4 * g] = x.x; o[4 * g + 1] = x.y; o[4 * g + 2] = x.z; o[4 * g + 3] = x.w;
+        }
+    };
+    uint32_t cur[32], nxt[32], sum[32] = {};
+    fetch(0, cur);
+#pragma unroll 1
+    for (int i = 0; i < pieces; ++i) {
+        if (i + 1 < pieces) fetch(i + 1, nxt);
+        const int c = i / p.tail_S, sl = i - c * p.tail_S;
+#pragma unroll
+        for (int g = 0; g < 32; ++g) {
+            Out x, y;
+            memcpy(&x, &cur[g], 4);
+            memcpy(&y, &sum[g], 4);
+            y = sl == 0 ? x : y + x;
+            memcpy(&sum[g], &y, 4);
+        }
+        if (sl == p.tail_S - 1) export_piece(sum, c * 32);
+#pragma unroll
+        for (int g = 0; g < 32; ++g) cur[g] = nxt[g];
+    }
+}
+
 template <int STAGES>
 constexpr int pair_smem_bytes() { return STAGES * PAIR_STAGE_BYTES + PAIR_STAGING_BYTES + 1024 + 1024; }
 
@@ -304,64 +367,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (lane == 0) ptx::mbar_arrive_cluster(&ctl->acc_empty[ab], 0);
                 continue;
             }
-            // k-slice of a tail tile: park this strip's partial sums (16-byte piece g of a lane's 32 values at
-            // (g * 32 + lane) * 16, so that one store instruction writes 512 contiguous bytes), give the accumulator
-            // back, then find out whether the other slices of the strip are already there
-            const int strip = static_cast<int>(rank) * 4 + q;
-            uint8_t* tile_ws = static_cast<uint8_t*>(p.tail_ws) + static_cast<size_t>(w.tail_index) * p.tail_S * PAIR_TILE_BYTES;
-            uint8_t* mine = tile_ws + static_cast<size_t>(w.slice) * PAIR_TILE_BYTES + strip * PAIR_STRIP_BYTES;
-#pragma unroll 1
-            for (int c = 0; c < nchunks; ++c) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + c * 32), v);
-                ptx::tmem_ld_wait();
-                uint4* dst = reinterpret_cast<uint4*>(mine + c * 4096);
-#pragma unroll
-                for (int g = 0; g < 8; ++g) dst[g * 32 + lane] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-            }
-            ptx::tc_fence_before();
-            __threadfence();  // this lane's partial sums are out before the warp is counted
-            __syncwarp();
-            int arrived = 0;
-            if (lane == 0) {
-                ptx::mbar_arrive_cluster(&ctl->acc_empty[ab], 0);
-                arrived = atomicAdd(&p.tail_counters[w.tail_index * 8 + strip], 1);
-            }
-            arrived = __shfl_sync(0xffffffffu, arrived, 0);
-            if (arrived != p.tail_S - 1) continue;  // a later warp finishes this strip
-            // every slice of the strip has been parked: C_ij = their sum in increasing k (the slice at hand is read back
-            // like the others; the read of the next piece is in flight while this one is added)
-            __threadfence();
-            if (lane == 0) p.tail_counters[w.tail_index * 8 + strip] = 0;  // zero again for the next launch
-            const uint8_t* strip_ws = tile_ws + strip * PAIR_STRIP_BYTES;
-            const int pieces = nchunks * p.tail_S;
-            auto fetch = [&](int i, uint32_t (&o)[32]) {
-                const int c = i / p.tail_S, sl = i - c * p.tail_S;
-                const uint4* src = reinterpret_cast<const uint4*>(strip_ws + static_cast<size_t>(sl) * PAIR_TILE_BYTES + c * 4096);
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    const uint4 x = __ldcg(src + g * 32 + lane);  // written by another SM: read through L2
-                    o[4 * g] = x.x; o[4 * g + 1] = x.y; o[4 * g + 2] = x.z; o[4 * g + 3] = x.w;
-                }
-            };
-            uint32_t cur[32], nxt[32], sum[32] = {};
-            fetch(0, cur);
-#pragma unroll 1
-            for (int i = 0; i < pieces; ++i) {
-                if (i + 1 < pieces) fetch(i + 1, nxt);
-                const int c = i / p.tail_S, sl = i - c * p.tail_S;
-#pragma unroll
-                for (int g = 0; g < 32; ++g) {
-                    Out x, y;
-                    memcpy(&x, &cur[g], 4);
-                    memcpy(&y, &sum[g], 4);
-                    y = sl == 0 ? x : y + x;
-                    memcpy(&sum[g], &y, 4);
-                }
-                if (sl == p.tail_S - 1) export_piece(sum, c * 32);
-#pragma unroll
-                for (int g = 0; g < 32; ++g) cur[g] = nxt[g];
-            }
+            // k-slice of a tail tile
+            pair_tail_strip<Out>(p, w, static_cast<int>(rank) * 4 + q, lane_taddr + static_cast<uint32_t>(ab * PAIR_BN), nchunks, lane,
+                                 &ctl->acc_empty[ab], export_piece);
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
         __syncwarp();

@@ -13,26 +13,41 @@
 // buffer before the MMA thread may read it (the landed tile itself serves as the hi
 // part).  The split is element-wise, so it is indifferent to the swizzled tile layout.
 //
-// Barriers: full[s] (per CTA: its own 32 KB of copies), ready[s] (leader: 8 arrivals =
-// 4 split warps of each CTA), empty[s] (both, by the leader's multicast commit),
-// acc_full[a] (both), acc_empty[a] (leader, 8 arrivals).
+// Barriers: full[s] (per CTA: its own 32 KB of copies), ready[s] (leader: 8 arrivals = the
+// four split warps of the stage's turn in each CTA; the peer's arrive across the pair with a
+// CTA-scope release, which is enough because every split thread has already made its writes
+// visible to the async proxy and the tiles are read by the tensor cores only), empty[s]
+// (both, by the leader's multicast commit), acc_full[a] (both), acc_empty[a] (leader, 8).
 #pragma once
 #include "umma_pair_kernel.cuh"
 
 namespace cyc {
 
-constexpr int X3_SPLIT_SETS = 2;               // sets of four split warps, taking stages in turn
-constexpr int X3_THREADS = 192 + X3_SPLIT_SETS * 128;  // TMA, MMA, 4 epilogue warps, then the split warps
-constexpr int X3_STAGE_HI = 2 * 128 * 128;     // A (128 rows) + B half (128 columns), 128 bytes of k each
+#ifndef CYC_X3_SPLIT_SETS
+#define CYC_X3_SPLIT_SETS 1
+#endif
+constexpr int X3_SPLIT_WARPS = 8;                         // split warps per CTA
+constexpr int X3_SPLIT_SETS = CYC_X3_SPLIT_SETS;          // sets of split warps, taking stages in turn
+constexpr int X3_SET_WARPS = X3_SPLIT_WARPS / X3_SPLIT_SETS;
+constexpr int X3_THREADS = 192 + X3_SPLIT_WARPS * 32;     // TMA, MMA, 4 epilogue warps, then the split warps
+#ifndef CYC_X3_BK
+#define CYC_X3_BK 32
+#endif
+// A stage holds BK = 32 (or 16) values of k: A (128 rows) + B half (128 columns), BK * 4 bytes of k each, followed by their
+// lo parts.  The ring is 192 KB either way: three stages of 64 KB or six of 32 KB (64-byte swizzle).  Measured on the
+// 65536 x 256 x 256 problem: 49-52 microseconds with three stages, 61-62 with six -- the stage rate is set by the bytes
+// that cross shared memory per unit of k (TMA write, split read and write, operand reads of three MMAs), not by the depth.
+constexpr int X3_BK = CYC_X3_BK;
+constexpr int X3_STAGE_HI = 2 * 128 * X3_BK * 4;
 constexpr int X3_STAGE_BYTES = 2 * X3_STAGE_HI;  // hi parts followed by lo parts
-constexpr int X3_STAGES = 3;
-constexpr int X3_PREFETCH = 8;  // k-blocks of A requested from L2 ahead of the ring
+constexpr int X3_STAGES = 96 / X3_BK;
+constexpr int X3_PREFETCH = 256 / X3_BK;  // k-blocks of A requested from L2 ahead of the ring
 constexpr int X3_SMEM_BYTES = X3_STAGES * X3_STAGE_BYTES + PAIR_STAGING_BYTES + 1024 + 1024;
 
 struct X3Ctl {
-    uint64_t full[4];
-    uint64_t ready[4];
-    uint64_t empty[4];
+    uint64_t full[8];
+    uint64_t ready[8];
+    uint64_t empty[8];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint32_t tmem_base;
@@ -61,7 +76,7 @@ template <bool B_MN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(X3_THREADS, 1)
 umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                         const __grid_constant__ CUtensorMap tmC, const PairParams p) {
-    constexpr int BK = 32;   // fp32 elements per 128-byte swizzle row
+    constexpr int BK = X3_BK;  // fp32 elements of k per stage: one 128-byte (or 64-byte) swizzle row
     constexpr int UK = 8;    // k extent of one kind::tf32 MMA
     constexpr int CH = 32;   // B stored [K][N]: columns per 128-byte row
     constexpr uint32_t TMEM_COLS = 512;
@@ -84,7 +99,7 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&ctl->full[s], 1);
-            ptx::mbar_init(&ctl->ready[s], 8);  // four split warps of each CTA
+            ptx::mbar_init(&ctl->ready[s], 2 * X3_SET_WARPS);  // the split warps of the stage's turn, both CTAs
             ptx::mbar_init(&ctl->empty[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -118,26 +133,28 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; nothing it wrote is read before it ends
             // A is streamed from HBM exactly once, and the ring is only three stages deep: a second cursor runs
             // X3_PREFETCH k-blocks ahead and asks L2 for the A tiles, so the copies into the ring hit L2
-            long long pf_t = pair;
-            int pf_kb = 0;
+            int pf_item = 0, pf_kb = 0;
+            PairWork pw;
+            bool pf_more = pair_work_item(p, num_kb, pair, num_pairs, 0, pw);
             auto prefetch_next = [&]() {
-                if (pf_t >= p.num_tiles) return;
+                if (!pf_more) return;
                 int b, tm, tn;
-                umma_tile_coord(pf_t, p.tiles_m, p.tiles_n, b, tm, tn);
-                ptx::tma_prefetch_l2_3d(&tmA, pf_kb * BK, tm * 256 + static_cast<int>(rank) * PAIR_HALF, b);
-                if (++pf_kb == num_kb) { pf_kb = 0; pf_t += num_pairs; }
+                umma_tile_coord(pw.tile, p.tiles_m, p.tiles_n, b, tm, tn);
+                ptx::tma_prefetch_l2_3d(&tmA, (pw.kb0 + pf_kb) * BK, tm * 256 + static_cast<int>(rank) * PAIR_HALF, b);
+                if (++pf_kb == pw.nkb) { pf_kb = 0; pf_more = pair_work_item(p, num_kb, pair, num_pairs, ++pf_item, pw); }
             };
             for (int i = 0; i < X3_PREFETCH; ++i) prefetch_next();
-            for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
+            PairWork w;
+            for (int item = 0; ok && pair_work_item(p, num_kb, pair, num_pairs, item, w); ++item) {
                 int b, tm, tn;
-                umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);
+                umma_tile_coord(w.tile, p.tiles_m, p.tiles_n, b, tm, tn);
                 const int m0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF;
                 const int n0 = tn * PAIR_BN + static_cast<int>(rank) * PAIR_HALF;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = w.kb0; kb < w.kb0 + w.nkb; ++kb) {
                     prefetch_next();
                     if (!x3_wait(&ctl->empty[stage], phase ^ 1, ctl, p.status, 1)) { ok = false; break; }
                     uint8_t* sa = smem + stage * X3_STAGE_BYTES;
-                    uint8_t* sb = sa + 128 * 128;
+                    uint8_t* sb = sa + 128 * BK * 4;
                     ptx::mbar_arrive_expect_tx(&ctl->full[stage], X3_STAGE_HI);
                     ptx::tma_load_3d(sa, &tmA, &ctl->full[stage], kb * BK, m0, b);
                     if constexpr (!B_MN) {
@@ -170,25 +187,28 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             uint32_t phase = 0;
             int local = 0;
             bool ok = true;
-            for (long long t = pair; t < p.num_tiles && ok; t += num_pairs, ++local) {
+            PairWork w;
+            for (; ok && pair_work_item(p, num_kb, pair, num_pairs, local, w); ++local) {
                 const int ab = local & 1;
                 const uint32_t acc_phase = (local >> 1) & 1;
                 if (!x3_wait(&ctl->acc_empty[ab], acc_phase ^ 1, ctl, p.status, 2)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * PAIR_BN);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = 0; kb < w.nkb; ++kb) {  // the first k-block of a slice starts from zero
                     if (!x3_wait(&ctl->ready[stage], phase, ctl, p.status, 3)) { ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t sa = ptx::smem_u32(smem + stage * X3_STAGE_BYTES);
-                    const uint32_t sb = sa + 128 * 128;
+                    const uint32_t sb = sa + 128 * BK * 4;
 #pragma unroll
                     for (int k = 0; k < BK / UK; ++k) {
-                        const uint64_t a_hi = umma_smem_desc(sa + k * 32, 16, 1024);
-                        const uint64_t a_lo = umma_smem_desc(sa + X3_STAGE_HI + k * 32, 16, 1024);
+                        // K-major rows of BK * 4 bytes (128- or 64-byte swizzle), groups of 8 rows one after another
+                        constexpr uint32_t KSBO = 8 * BK * 4, KSW = BK == 32 ? 2 : 4;
+                        const uint64_t a_hi = umma_smem_desc(sa + k * 32, 16, KSBO, KSW);
+                        const uint64_t a_lo = umma_smem_desc(sa + X3_STAGE_HI + k * 32, 16, KSBO, KSW);
                         uint64_t b_hi, b_lo;
                         if constexpr (!B_MN) {
-                            b_hi = umma_smem_desc(sb + k * 32, 16, 1024);
-                            b_lo = umma_smem_desc(sb + X3_STAGE_HI + k * 32, 16, 1024);
+                            b_hi = umma_smem_desc(sb + k * 32, 16, KSBO, KSW);
+                            b_lo = umma_smem_desc(sb + X3_STAGE_HI + k * 32, 16, KSBO, KSW);
                         } else {
                             // B stored [K][N]: 128-byte rows of 32 columns, 32-byte chunks permuted over groups of
                             // 4 k-rows (512 B apart); the next 32 columns are BK*128 B further on
@@ -210,20 +230,24 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         // ------------------------------------------------------------ split warps: x -> (hi, lo)
         // the sets of four warps take stages in turn, so the fixed latencies of one stage's split
         // (wait, store drain, proxy fence) overlap with the other set's work
-        const int set = (warp - 6) >> 2;
-        const int tid = (threadIdx.x - 6 * 32) & 127;  // 0..127 within the set
-        constexpr int NT = 128;
+        const int set = (warp - 6) / X3_SET_WARPS;
+        constexpr int NT = 32 * X3_SET_WARPS;
+        const int tid = (threadIdx.x - 6 * 32) % NT;  // index within the set
         int stage = 0;
         uint32_t phase = 0;
         uint32_t turn = 0;
         bool ok = true;
-        for (long long t = pair; t < p.num_tiles && ok; t += num_pairs) {
-            for (int kb = 0; kb < num_kb; ++kb, ++turn) {
+        PairWork w;
+        for (int item = 0; ok && pair_work_item(p, num_kb, pair, num_pairs, item, w); ++item) {
+            for (int kb = 0; kb < w.nkb; ++kb, ++turn) {
+                // Every set observes every use of every stage, its own or not: a parity wait tells phase k from phase
+                // k + 1 only, and copies may land out of order, so a set that skipped the other set's turn could otherwise
+                // take the previous use of a stage for the one it is waiting for.
+                if (!x3_wait(&ctl->full[stage], phase, ctl, p.status, 5)) { ok = false; break; }
                 if (turn % X3_SPLIT_SETS != static_cast<uint32_t>(set)) {
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                     continue;
                 }
-                if (!x3_wait(&ctl->full[stage], phase, ctl, p.status, 5)) { ok = false; break; }
                 uint8_t* base = smem + stage * X3_STAGE_BYTES;
 #pragma unroll 1
                 for (int it0 = 0; it0 < X3_STAGE_HI / (NT * 16); it0 += 4) {
@@ -248,7 +272,10 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 }
                 ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive_cluster(&ctl->ready[stage], 0);
+                if (lane == 0) {
+                    if (rank == 0) ptx::mbar_arrive(&ctl->ready[stage]);
+                    else ptx::mbar_arrive_remote(&ctl->ready[stage], 0);
+                }
                 if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
         }
@@ -256,29 +283,27 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         // ------------------------------------------------------------ epilogue: C_ij <- [i,k_end]_C (both CTAs)
         const int q = warp & 3;
         uint8_t* my_stage = staging + q * 8192;
+        const uint32_t lane_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
         int local = 0, sbuf = 0;
         bool ok = true;
-        for (long long t = pair; t < p.num_tiles && ok; t += num_pairs, ++local) {
+        PairWork w;
+        for (; ok && pair_work_item(p, num_kb, pair, num_pairs, local, w); ++local) {
             const int ab = local & 1;
             const uint32_t acc_phase = (local >> 1) & 1;
             int b, tm, tn;
-            umma_tile_coord(t, p.tiles_m, p.tiles_n, b, tm, tn);
+            umma_tile_coord(w.tile, p.tiles_m, p.tiles_n, b, tm, tn);
             if (!x3_wait(&ctl->acc_full[ab], acc_phase, ctl, p.status, 4)) { ok = false; break; }
             ptx::tc_fence_after();
             const int row0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF + q * 32;
             const int row = row0 + lane;
             float* crow = static_cast<float*>(p.C) + static_cast<long long>(b) * p.sC + static_cast<long long>(row) * p.N;
-#pragma unroll 1
-            for (int c0 = 0; c0 < PAIR_BN; c0 += 32) {
+            const int nchunks = min(PAIR_BN / 32, (p.N - tn * PAIR_BN + 31) / 32);
+            auto export_piece = [&](const uint32_t (&v)[32], int c0) {
                 const int col = tn * PAIR_BN + c0;
-                if (col >= p.N) break;
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(ab * PAIR_BN + c0), v);
                 if (p.tma_store) {
                     uint8_t* buf = my_stage + sbuf * 4096;
                     if (lane == 0) ptx::tma_store_wait_read<1>();
                     __syncwarp();
-                    ptx::tmem_ld_wait();
 #pragma unroll
                     for (int g = 0; g < 8; ++g)
                         *reinterpret_cast<uint4*>(buf + lane * 128 + ((g ^ (lane & 7)) << 4)) = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
@@ -289,13 +314,24 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         ptx::tma_store_commit();
                     }
                     sbuf ^= 1;
-                } else {
-                    ptx::tmem_ld_wait();
-                    if (row < p.M) {
+                } else if (row < p.M) {
 #pragma unroll
-                        for (int g = 0; g < 32; ++g)
-                            if (col + g < p.N) reinterpret_cast<uint32_t*>(crow)[col + g] = v[g];
-                    }
+                    for (int g = 0; g < 32; ++g)
+                        if (col + g < p.N) reinterpret_cast<uint32_t*>(crow)[col + g] = v[g];
+                }
+            };
+            // the tensor-memory read of the next piece is in flight while this one is staged and stored
+            uint32_t va[32], vb[32];
+            ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN), va);
+#pragma unroll 1
+            for (int c = 0; c < nchunks; c += 2) {
+                ptx::tmem_ld_wait();
+                if (c + 1 < nchunks) ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + (c + 1) * 32), vb);
+                export_piece(va, c * 32);
+                if (c + 1 < nchunks) {
+                    ptx::tmem_ld_wait();
+                    if (c + 2 < nchunks) ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + (c + 2) * 32), va);
+                    export_piece(vb, (c + 1) * 32);
                 }
             }
             ptx::tc_fence_before();
