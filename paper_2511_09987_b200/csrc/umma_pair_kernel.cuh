@@ -125,7 +125,7 @@ __device__ __forceinline__ void pair_tail_strip(const PairParams& p, const PairW
     __syncwarp();
     int arrived = 0;
     if (lane == 0) {
-        ptx::mbar_arrive_cluster(acc_empty, 0);
+        ptx::mbar_arrive_remote(acc_empty, 0);
         arrived = atomicAdd(&p.tail_counters[w.tail_index * 8 + strip], 1);
     }
     arrived = __shfl_sync(0xffffffffu, arrived, 0);
@@ -364,7 +364,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive_cluster(&ctl->acc_empty[ab], 0);
+                if (lane == 0) ptx::mbar_arrive_remote(&ctl->acc_empty[ab], 0);
                 continue;
             }
             // k-slice of a tail tile

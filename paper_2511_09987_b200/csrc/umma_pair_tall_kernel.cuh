@@ -199,7 +199,7 @@ umma_pair_tall_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             }
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(&ctl->acc_empty[0], 0);
+            if (lane == 0) ptx::mbar_arrive_remote(&ctl->acc_empty[0], 0);
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
         __syncwarp();

@@ -336,7 +336,7 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             }
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(&ctl->acc_empty[ab], 0);
+            if (lane == 0) ptx::mbar_arrive_remote(&ctl->acc_empty[ab], 0);
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
         __syncwarp();
