@@ -748,7 +748,7 @@ static int launch_fa2(long long batch, long long N, long long M, const void* Q, 
     Fa2Params p;
     p.O = O;
     p.N = static_cast<int>(N); p.M = static_cast<int>(M);
-    p.tiles_q = static_cast<int>((N + FA2_BM - 1) / FA2_BM);
+    p.tiles_q = static_cast<int>((N + FA2_ROWS - 1) / FA2_ROWS);
     p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
     if (int rc_ = status_word(&p.status)) return rc_;
     auto kern = fa2_kernel<D>;
@@ -780,7 +780,39 @@ extern "C" int cyc_recurrence_matmul_batched(int64_t batch, int64_t M, int64_t N
 
 // Host-buffer evaluation.  Device buffers come from the library's pool; for large problems the rows of A and C (or the
 // problems of a batch) are cut into chunks so that the upload of chunk i+1, the kernel of chunk i and the download of
-// chunk i-1 overlap (two helper streams, ordered against the caller's stream by events).
+// chunk i-1 overlap (two helper streams, ordered against the caller's stream by events).  The helper streams and
+// events are created once per device and kept; a mutex serialises host-buffer calls on one device (they would share
+// the PCIe link anyway).
+constexpr int kHostChunksMax = 16;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t up = nullptr, down = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_down = nullptr, ev_up[kHostChunksMax] = {}, ev_done[kHostChunksMax] = {};
+    std::mutex mu;
+};
+static int host_pipe(HostPipe** out) {
+    static std::mutex mu;
+    static HostPipe pipes[64];
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    HostPipe& hp = pipes[dev];
+    if (!hp.ready) {
+        CYC_CUDA(cudaStreamCreateWithFlags(&hp.up, cudaStreamNonBlocking));
+        CYC_CUDA(cudaStreamCreateWithFlags(&hp.down, cudaStreamNonBlocking));
+        CYC_CUDA(cudaEventCreateWithFlags(&hp.ev_start, cudaEventDisableTiming));
+        CYC_CUDA(cudaEventCreateWithFlags(&hp.ev_down, cudaEventDisableTiming));
+        for (int c = 0; c < kHostChunksMax; ++c) {
+            CYC_CUDA(cudaEventCreateWithFlags(&hp.ev_up[c], cudaEventDisableTiming));
+            CYC_CUDA(cudaEventCreateWithFlags(&hp.ev_done[c], cudaEventDisableTiming));
+        }
+        hp.ready = true;
+    }
+    *out = &hp;
+    return CYC_OK;
+}
+
 extern "C" int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A_host,
                                           const void* B_host, void* C_host, void* stream, unsigned flags) {
     if (batch <= 0 || M <= 0 || N <= 0 || K <= 0 || !A_host || !B_host || !C_host) return CYC_ERR_INVALID_ARG;
@@ -795,6 +827,10 @@ extern "C" int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, i
     cudaMemPool_t pool;
     int rc = workspace_pool(&pool);
     if (rc) return rc;
+    HostPipe* hp = nullptr;
+    rc = host_pipe(&hp);
+    if (rc) return rc;
+    std::lock_guard<std::mutex> pipe_lock(hp->mu);
     uint8_t* d = nullptr;
     CYC_CUDA(cudaMallocFromPoolAsync(reinterpret_cast<void**>(&d), oc + nc, pool, st));
     const uint8_t* hA = static_cast<const uint8_t*>(A_host);
@@ -802,10 +838,12 @@ extern "C" int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, i
     uint8_t* hC = static_cast<uint8_t*>(C_host);
     cudaError_t e = cudaSuccess;
 
-    // chunks: rows of one problem (multiples of 512), or whole problems of a batch
+    // chunks: rows of one problem (multiples of 512), or whole problems of a batch; about 8 MB of traffic each, so
+    // that the first kernel starts early and the last download is short
     const bool by_rows = batch == 1;
     const long long units = by_rows ? M : batch;
-    long long nch = (na + nc) > (16u << 20) ? 4 : 1;
+    long long nch = static_cast<long long>((na + nc) / (8u << 20));
+    nch = std::max<long long>(1, std::min<long long>(nch, kHostChunksMax));
     long long per = (units + nch - 1) / nch;
     if (by_rows) per = (per + 511) / 512 * 512;
     if (per < 1) per = 1;
@@ -822,63 +860,38 @@ extern "C" int cyc_recurrence_matmul_host(int64_t batch, int64_t M, int64_t N, i
         if (!rc && (e = cudaMemcpyAsync(hC, d + oc, nc, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
             rc = cuda_fail(e, "cudaMemcpyAsync(device to host)");
     } else {
-        cudaStream_t up = nullptr, down = nullptr;
-        cudaEvent_t ev_start = nullptr, ev_up[8] = {}, ev_done[8] = {}, ev_down = nullptr;
         auto ok = [&](cudaError_t err, const char* what) {
             if (err != cudaSuccess && !rc) rc = cuda_fail(err, what);
             return rc == CYC_OK;
         };
-        ok(cudaStreamCreateWithFlags(&up, cudaStreamNonBlocking), "cudaStreamCreateWithFlags");
-        ok(cudaStreamCreateWithFlags(&down, cudaStreamNonBlocking), "cudaStreamCreateWithFlags");
-        ok(cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming), "cudaEventCreateWithFlags");
-        ok(cudaEventCreateWithFlags(&ev_down, cudaEventDisableTiming), "cudaEventCreateWithFlags");
-        for (long long c = 0; c < nch && !rc; ++c) {
-            ok(cudaEventCreateWithFlags(&ev_up[c], cudaEventDisableTiming), "cudaEventCreateWithFlags");
-            ok(cudaEventCreateWithFlags(&ev_done[c], cudaEventDisableTiming), "cudaEventCreateWithFlags");
-        }
-        if (!rc) {
-            // the helper streams start after whatever the caller's stream holds (the allocation included)
-            ok(cudaEventRecord(ev_start, st), "cudaEventRecord");
-            ok(cudaStreamWaitEvent(up, ev_start, 0), "cudaStreamWaitEvent");
-            ok(cudaStreamWaitEvent(down, ev_start, 0), "cudaStreamWaitEvent");
-            if (by_rows) ok(cudaMemcpyAsync(d + ob, hB, nb, cudaMemcpyHostToDevice, up), "cudaMemcpyAsync(B)");
-        }
+        // the helper streams start after whatever the caller's stream holds (the allocation included)
+        ok(cudaEventRecord(hp->ev_start, st), "cudaEventRecord");
+        ok(cudaStreamWaitEvent(hp->up, hp->ev_start, 0), "cudaStreamWaitEvent");
+        ok(cudaStreamWaitEvent(hp->down, hp->ev_start, 0), "cudaStreamWaitEvent");
+        if (by_rows && !rc) ok(cudaMemcpyAsync(d + ob, hB, nb, cudaMemcpyHostToDevice, hp->up), "cudaMemcpyAsync(B)");
         for (long long c = 0; c < nch && !rc; ++c) {
             const long long u0 = c * per, un = (u0 + per <= units ? per : units - u0);
-            // element offsets of this chunk in A, B, C
+            // byte offsets of this chunk in A, B, C
             const size_t a_off = static_cast<size_t>(u0) * (by_rows ? K : M * K) * eb, a_len = static_cast<size_t>(un) * (by_rows ? K : M * K) * eb;
             const size_t c_off = static_cast<size_t>(u0) * (by_rows ? N : M * N) * 4, c_len = static_cast<size_t>(un) * (by_rows ? N : M * N) * 4;
             const size_t b_off = by_rows ? 0 : static_cast<size_t>(u0) * K * N * eb, b_len = by_rows ? 0 : static_cast<size_t>(un) * K * N * eb;
-            ok(cudaMemcpyAsync(d + oa + a_off, hA + a_off, a_len, cudaMemcpyHostToDevice, up), "cudaMemcpyAsync(A chunk)");
-            if (b_len) ok(cudaMemcpyAsync(d + ob + b_off, hB + b_off, b_len, cudaMemcpyHostToDevice, up), "cudaMemcpyAsync(B chunk)");
-            ok(cudaEventRecord(ev_up[c], up), "cudaEventRecord");
-            ok(cudaStreamWaitEvent(st, ev_up[c], 0), "cudaStreamWaitEvent");
+            ok(cudaMemcpyAsync(d + oa + a_off, hA + a_off, a_len, cudaMemcpyHostToDevice, hp->up), "cudaMemcpyAsync(A chunk)");
+            if (b_len) ok(cudaMemcpyAsync(d + ob + b_off, hB + b_off, b_len, cudaMemcpyHostToDevice, hp->up), "cudaMemcpyAsync(B chunk)");
+            ok(cudaEventRecord(hp->ev_up[c], hp->up), "cudaEventRecord");
+            ok(cudaStreamWaitEvent(st, hp->ev_up[c], 0), "cudaStreamWaitEvent");
             if (!rc) {
                 Problem q{by_rows ? 1 : un, by_rows ? un : M, N, K, dtype, d + oa + a_off, d + ob + b_off, d + oc + c_off, (by_rows ? un : M) * K, K * N,
                           (by_rows ? un : M) * N, flags};
                 rc = dispatch(q, st);
             }
-            ok(cudaEventRecord(ev_done[c], st), "cudaEventRecord");
-            ok(cudaStreamWaitEvent(down, ev_done[c], 0), "cudaStreamWaitEvent");
-            ok(cudaMemcpyAsync(hC + c_off, d + oc + c_off, c_len, cudaMemcpyDeviceToHost, down), "cudaMemcpyAsync(C chunk)");
+            ok(cudaEventRecord(hp->ev_done[c], st), "cudaEventRecord");
+            ok(cudaStreamWaitEvent(hp->down, hp->ev_done[c], 0), "cudaStreamWaitEvent");
+            ok(cudaMemcpyAsync(hC + c_off, d + oc + c_off, c_len, cudaMemcpyDeviceToHost, hp->down), "cudaMemcpyAsync(C chunk)");
         }
         // the caller's stream continues (and the buffer is freed) only after the last download
-        if (down) {
-            if (ev_down && cudaEventRecord(ev_down, down) == cudaSuccess) cudaStreamWaitEvent(st, ev_down, 0);
-            else cudaStreamSynchronize(down);
-        }
-        if (up && rc) cudaStreamSynchronize(up);
-        cudaFreeAsync(d, st);
-        if ((e = cudaStreamSynchronize(st)) != cudaSuccess && !rc) rc = cuda_fail(e, "cudaStreamSynchronize");
-        if (up) { cudaStreamSynchronize(up); cudaStreamDestroy(up); }
-        if (down) { cudaStreamSynchronize(down); cudaStreamDestroy(down); }
-        if (ev_start) cudaEventDestroy(ev_start);
-        if (ev_down) cudaEventDestroy(ev_down);
-        for (int c = 0; c < 8; ++c) {
-            if (ev_up[c]) cudaEventDestroy(ev_up[c]);
-            if (ev_done[c]) cudaEventDestroy(ev_done[c]);
-        }
-        return rc;
+        if (cudaEventRecord(hp->ev_down, hp->down) == cudaSuccess) cudaStreamWaitEvent(st, hp->ev_down, 0);
+        else cudaStreamSynchronize(hp->down);
+        if (rc) { cudaStreamSynchronize(hp->up); cudaStreamSynchronize(hp->down); }
     }
     cudaFreeAsync(d, st);
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess && !rc) rc = cuda_fail(e, "cudaStreamSynchronize");
@@ -1015,7 +1028,7 @@ extern "C" int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t 
         snprintf(g_err, sizeof g_err, "flash attention: Q, K, V and O must be 16-byte aligned");
         return CYC_ERR_UNSUPPORTED;
     }
-    const long long tiles_q = (N + FA2_BM - 1) / FA2_BM;
+    const long long tiles_q = (N + FA2_ROWS - 1) / FA2_ROWS;
     if (N > 0x7fffffffll || M > 0x7fffffffll || batch * tiles_q > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
     DeviceInfo di;
     int rc = device_info(&di);
