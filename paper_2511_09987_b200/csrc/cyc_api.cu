@@ -752,6 +752,19 @@ static int launch_fa2(long long batch, long long N, long long M, const void* Q, 
     p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
     if (int rc_ = status_word(&p.status)) return rc_;
     auto kern = fa2_kernel<D>;
+    {
+        // the kernel redistributes the registers it was launched with among its warps and counts on 128 per thread
+        static std::atomic<int> checked{0};
+        if (!checked.load()) {
+            cudaFuncAttributes fa;
+            CYC_CUDA(cudaFuncGetAttributes(&fa, kern));
+            if (fa.numRegs < FA2_REGS_LAUNCH) {
+                snprintf(g_err, sizeof g_err, "flash attention kernel compiled to %d registers per thread, %d expected", fa.numRegs, FA2_REGS_LAUNCH);
+                return CYC_ERR_CUDA;
+            }
+            checked.store(1);
+        }
+    }
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), Fa2Smem<D>::TOTAL)) return rc_;
     CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(batch * p.tiles_q), FA2_THREADS, Fa2Smem<D>::TOTAL, st, tmQ, tmK, tmV, p));
     g_launches.fetch_add(1);

@@ -86,14 +86,15 @@ __device__ __forceinline__ float fa2_exp2(float x) {
 }
 
 // D[tmem] (+)= A[tmem] * B[smem], bf16 operands, one CTA
-__device__ __forceinline__ void fa2_umma_tmem_a(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void fa2_umma_tmem_a(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate, uint32_t leader) {
     asm volatile(
         "{\n"
-        ".reg .pred p;\n"
+        ".reg .pred p, q;\n"
         "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "setp.ne.b32 q, %5, 0;\n"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
         "}" ::"r"(tmem_d),
-        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
         : "memory");
 }
 // 32 lanes x 32 consecutive 32-bit columns from registers: thread t of the warp writes lane (base_lane + t)
@@ -109,6 +110,23 @@ __device__ __forceinline__ void fa2_tmem_st_32x32(uint32_t taddr, const uint32_t
         : "memory");
 }
 __device__ __forceinline__ void fa2_tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Register split.  The block is launched with 512 x 128 registers; the four warps that hold the producer and the MMA
+// issuer drop to 64 each and the keepers to 96, which lets the two groups of row threads grow to 176:
+// 2 * 128 * 176 + 128 * 96 + 128 * 64 = 65536 (no spills with this split).  (A split that asked for more than the launch holds would wait forever;
+// the host refuses to launch if the kernel was not compiled to 128 registers per thread.)
+constexpr int FA2_REGS_ROW = 176, FA2_REGS_KEEPER = 96, FA2_REGS_OTHER = 64, FA2_REGS_LAUNCH = 128;
+static_assert(FA2_REGS_ROW % 8 == 0 && FA2_REGS_KEEPER % 8 == 0 && FA2_REGS_OTHER % 8 == 0, "setmaxnreg takes multiples of 8");
+static_assert(2 * 128 * FA2_REGS_ROW + 128 * FA2_REGS_KEEPER + 128 * FA2_REGS_OTHER <= FA2_THREADS * FA2_REGS_LAUNCH, "register split");
+template <int N>
+__device__ __forceinline__ void fa2_regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void fa2_regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+__device__ __forceinline__ float fa2_max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 template <int D>
 __global__ void __launch_bounds__(FA2_THREADS, 1)
@@ -163,7 +181,9 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (warp == 12) {
+    if (warp >= 12) {
+      fa2_regs_dec<FA2_REGS_OTHER>();
+      if (warp == 12) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; nothing it wrote is read before it ends
@@ -209,38 +229,49 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
         }
         __syncwarp();
-    } else if (warp == 13) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+      } else if (warp == 13) {
+        // ------------------------------------------------------------ MMA issuer: the whole warp walks the loop (waits
+        // ------------------------------------------------------------ included), one elected lane issues
+        {
+            const uint32_t leader = ptx::elect_one();
             bool ok = fa2_wait(&ctl->q_full, 0, ctl, p.status, 2);
+            // The issuing thread shares its scheduler with busy row warps, and an MMA of this size runs for only 64 clocks:
+            // every instruction between two MMAs counts.  Descriptors are built once; a k-step only adds its byte offset
+            // (in 16-byte units) to the address field, which cannot carry out of its 14 bits below 256 KB.
+            uint64_t dQ[2], dK[2], dV[2];
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                dQ[x] = umma_smem_desc(ptx::smem_u32(sQ + x * Sm::Q_BYTES), 16, 1024);
+                dK[x] = umma_smem_desc(ptx::smem_u32(sKV + x * Sm::STAGE_BYTES), 16, 1024);
+                dV[x] = umma_smem_desc(ptx::smem_u32(sKV + x * Sm::STAGE_BYTES + Sm::K_BYTES), Sm::SLAB, 1024);
+            }
             // S_i(t) = Q_i K_t^T, both operands K-major, into the score buffer of query tile i
             auto issue_s = [&](int i, int t) {
-                const uint32_t aQ = ptx::smem_u32(sQ + i * Sm::Q_BYTES);
-                const uint32_t aK = ptx::smem_u32(sKV + (t & 1) * Sm::STAGE_BYTES);
+                const uint64_t q0 = dQ[i], k0 = dK[t & 1];
+                const uint32_t d_s = tmem_base + COL_S + i * FA2_BN;
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k >> 2) * Sm::SLAB + (k & 3) * 32;
-                    ptx::umma<KIND_BF16, 1>(tmem_base + COL_S + i * FA2_BN, umma_smem_desc(aQ + off, 16, 1024),
-                                            umma_smem_desc(aK + off, 16, 1024), IDESC_S, k != 0 ? 1u : 0u);
+                    constexpr uint32_t dummy = 0; (void)dummy;
+                    const uint64_t off = static_cast<uint64_t>(((k >> 2) * Sm::SLAB + (k & 3) * 32) >> 4);
+                    ptx::umma_elect<KIND_BF16>(d_s, q0 + off, k0 + off, IDESC_S, k != 0 ? 1u : 0u, leader);
                 }
-                ptx::umma_commit(&ctl->s_full[i]);
+                ptx::umma_commit_elect(&ctl->s_full[i], leader);
             };
             // o_i (+)= P_i(t) V_t : A = P in tensor memory (row = lane, two keys per 32-bit column, 16 keys = 8 columns
             // per MMA), B = V (MN-major: 128-byte rows of d, 8-key groups 1024 B apart, next 64 columns of d one slab on)
             auto issue_u = [&](int i, int t) {
-                const uint32_t aV = ptx::smem_u32(sKV + (t & 1) * Sm::STAGE_BYTES + Sm::K_BYTES);
+                const uint64_t v0 = dV[t & 1];
+                const uint32_t d_o = tmem_base + COL_O + i * D, a_p = tmem_base + COL_S + i * FA2_BN;
 #pragma unroll
-                for (int k = 0; k < FA2_BN / 16; ++k) {
-                    const uint64_t bdesc = umma_smem_desc(aV + k * (16 * 128), Sm::SLAB, 1024);
-                    fa2_umma_tmem_a(tmem_base + COL_O + i * D, tmem_base + COL_S + i * FA2_BN + k * 8, bdesc, IDESC_U, (t | k) != 0 ? 1u : 0u);
-                }
-                ptx::umma_commit(&ctl->pv_done[i]);
+                for (int k = 0; k < FA2_BN / 16; ++k)
+                    fa2_umma_tmem_a(d_o, a_p + k * 8, v0 + static_cast<uint64_t>((k * 16 * 128) >> 4), IDESC_U, (t | k) != 0 ? 1u : 0u, leader);
+                ptx::umma_commit_elect(&ctl->pv_done[i], leader);
             };
             if (ok) ok = fa2_wait(&ctl->k_full[0], 0, ctl, p.status, 4);
             if (ok) {
                 ptx::tc_fence_after();
                 for (int i = 0; i < ntq; ++i) issue_s(i, 0);
-                ptx::umma_commit(&ctl->k_empty[0]);
+                ptx::umma_commit_elect(&ctl->k_empty[0], leader);
             }
             for (int t = 0; t < T && ok; ++t) {
                 const int st = t & 1;
@@ -250,20 +281,22 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     if (!fa2_wait(&ctl->o_ready[i], t & 1, ctl, p.status, 5)) { ok = false; break; }
                     ptx::tc_fence_after();
                     issue_u(i, t);
-                    if (i == ntq - 1) ptx::umma_commit(&ctl->v_empty[st]);
+                    if (i == ntq - 1) ptx::umma_commit_elect(&ctl->v_empty[st], leader);
                     if (t + 1 < T) {
                         // the next scores of this query tile go to the buffer its P was just read from: the tensor core
                         // runs the MMAs of one thread in issue order
                         if (i == 0 && !fa2_wait(&ctl->k_full[(t + 1) & 1], ((t + 1) >> 1) & 1, ctl, p.status, 4)) { ok = false; break; }
                         ptx::tc_fence_after();
                         issue_s(i, t + 1);
-                        if (i == ntq - 1) ptx::umma_commit(&ctl->k_empty[(t + 1) & 1]);
+                        if (i == ntq - 1) ptx::umma_commit_elect(&ctl->k_empty[(t + 1) & 1], leader);
                     }
                 }
             }
         }
         __syncwarp();
+      }
     } else if (warp < 8) {
+        fa2_regs_inc<FA2_REGS_ROW>();
         // ------------------------------------------------------------ row threads: one per query row
         const int i = warp >> 2;                 // query tile
         const int q = warp & 3;                  // TMEM lane quarter this warp may access
@@ -276,22 +309,25 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (!fa2_wait(&ctl->s_full[i], t & 1, ctl, p.status, 7)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const int valid = min(FA2_BN, p.M - t * FA2_BN);  // keys of this tile that exist (< 128 only in the last)
-                // ---- pass 1: the row's maximum over the tile
-                float mx = -INFINITY;
+                // ---- the row's 128 scores, read once and kept in registers from the maximum to the exponentials
+                uint32_t v[FA2_BN];
 #pragma unroll
-                for (int c0 = 0; c0 < FA2_BN; c0 += 32) {
-                    uint32_t v[32];
-                    ptx::tmem_ld_32x32(s_addr + c0, v);
-                    ptx::tmem_ld_wait();
-                    if (valid < FA2_BN) {
+                for (int c0 = 0; c0 < FA2_BN; c0 += 32) ptx::tmem_ld_32x32(s_addr + c0, *reinterpret_cast<uint32_t(*)[32]>(&v[c0]));
+                ptx::tmem_ld_wait();
+                if (valid < FA2_BN) {
 #pragma unroll
-                        for (int g = 0; g < 32; ++g)
-                            if (c0 + g >= valid) v[g] = 0xff800000u;  // a key that does not exist: -inf, weight 0
-                    }
-#pragma unroll
-                    for (int g = 0; g < 32; ++g) mx = fmaxf(mx, __uint_as_float(v[g]));
+                    for (int g = 0; g < FA2_BN; ++g)
+                        if (g >= valid) v[g] = 0xff800000u;  // a key that does not exist: -inf, weight 0
                 }
-                const float m_t = mx * p.scale_log2;
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;  // four chains of three-input maxima
+#pragma unroll
+                for (int g = 0; g < FA2_BN; g += 8) {
+                    mx0 = fa2_max3(mx0, __uint_as_float(v[g]), __uint_as_float(v[g + 1]));
+                    mx1 = fa2_max3(mx1, __uint_as_float(v[g + 2]), __uint_as_float(v[g + 3]));
+                    mx2 = fa2_max3(mx2, __uint_as_float(v[g + 4]), __uint_as_float(v[g + 5]));
+                    mx3 = fa2_max3(mx3, __uint_as_float(v[g + 6]), __uint_as_float(v[g + 7]));
+                }
+                const float m_t = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
                 // ---- does the reference move?  (never at the first tile: o is overwritten there, not accumulated)
                 float f = 1.0f;
                 if (t == 0) {
@@ -307,35 +343,25 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     ctl->need[i][q] = any != 0u;
                     ptx::mbar_arrive(&ctl->corr_req[i]);  // the keeper of these rows can start while the exponentials run
                 }
-                // ---- pass 2: P_t = 2^(S scale - m_ref) as bf16, two keys per 32-bit word (the lower key in the lower
-                // ---- half), row sum in fp32.  P goes over columns 0-63 of the score buffer: words 0-31 (keys 0-63) are
-                // ---- stored once columns 0-63 have been read, words 32-63 after columns 64-127.
-                float lsum = 0.f;
+                // ---- P_t = 2^(S scale - m_ref) as bf16, two keys per 32-bit word (the lower key in the lower half), packed
+                // ---- in place (word g/2 <= g: nothing still needed is overwritten), row sum in fp32 on four chains; P goes
+                // ---- over columns 0-63 of the score buffer
+                float ls0 = 0.f, ls1 = 0.f, ls2 = 0.f, ls3 = 0.f;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t pk[32];
+                for (int g = 0; g < FA2_BN; g += 8) {
+                    float e[8];
 #pragma unroll
-                    for (int cc = 0; cc < 2; ++cc) {
-                        const int c0 = h * 64 + cc * 32;
-                        uint32_t v[32];
-                        ptx::tmem_ld_32x32(s_addr + c0, v);
-                        ptx::tmem_ld_wait();
-                        if (valid < FA2_BN) {
+                    for (int u = 0; u < 8; ++u) e[u] = fa2_exp2(fmaf(__uint_as_float(v[g + u]), p.scale_log2, -m_ref));
+                    ls0 += e[0] + e[1]; ls1 += e[2] + e[3]; ls2 += e[4] + e[5]; ls3 += e[6] + e[7];
 #pragma unroll
-                            for (int g = 0; g < 32; ++g)
-                                if (c0 + g >= valid) v[g] = 0xff800000u;
-                        }
-#pragma unroll
-                        for (int g = 0; g < 32; g += 2) {
-                            const float p0 = fa2_exp2(fmaf(__uint_as_float(v[g]), p.scale_log2, -m_ref));
-                            const float p1 = fa2_exp2(fmaf(__uint_as_float(v[g + 1]), p.scale_log2, -m_ref));
-                            lsum += p0 + p1;
-                            __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
-                            pk[cc * 16 + (g >> 1)] = *reinterpret_cast<uint32_t*>(&hh);
-                        }
+                    for (int u = 0; u < 8; u += 2) {
+                        __nv_bfloat162 hh = __floats2bfloat162_rn(e[u], e[u + 1]);
+                        v[(g + u) >> 1] = *reinterpret_cast<uint32_t*>(&hh);
                     }
-                    fa2_tmem_st_32x32(s_addr + h * 32, pk);
                 }
+                const float lsum = (ls0 + ls1) + (ls2 + ls3);
+                fa2_tmem_st_32x32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                fa2_tmem_st_32x32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
                 l += lsum;
                 fa2_tmem_st_wait();
                 ptx::tc_fence_before();
@@ -347,7 +373,8 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (lane == 0) ptx::mbar_arrive(&ctl->l_done[i]);
         }
         ptx::tc_fence_before();
-    } else if (warp < 12) {
+    } else {
+        fa2_regs_dec<FA2_REGS_KEEPER>();
         // ------------------------------------------------------------ output keepers: one thread per row, both query tiles
         const int q = warp & 3;
         const int r = q * 32 + lane;

@@ -183,6 +183,43 @@ __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t b
 #undef CYC_UMMA_ASM
 }
 
+// One lane of a converged warp, chosen by the hardware: 1 in that lane, 0 in the others.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        ".reg .pred P;\n"
+        "elect.sync _|P, 0xffffffff;\n"
+        "selp.u32 %0, 1, 0, P;\n"
+        "}"
+        : "=r"(pred));
+    return pred;
+}
+// The MMA and the commit as PREDICATED instructions of a converged warp (`leader` is 1 in exactly one lane).  When a
+// whole warp walks the issue loop, descriptors and addresses are warp-uniform values the compiler can keep in uniform
+// registers; inside an `if (lane == 0)` branch it cannot, and every MMA pays for moving its operands there -- about a
+// hundred clocks, more than a 128 x 128 x 16 MMA runs.
+template <int KIND>
+__device__ __forceinline__ void umma_elect(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate, uint32_t leader) {
+    if constexpr (KIND == 0)
+        asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+                     "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
+                     : "memory");
+    else if constexpr (KIND == 1)
+        asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n@q tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+                     "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
+                     : "memory");
+    else
+        asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n@q tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+                     "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
+                     : "memory");
+}
+__device__ __forceinline__ void umma_commit_elect(uint64_t* bar, uint32_t leader) {
+    asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(smem_u32(bar)),
+                 "r"(leader)
+                 : "memory");
+}
+
 // make the mbarrier track completion of all tcgen05 operations issued so far by this thread
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
