@@ -199,25 +199,36 @@ __device__ __forceinline__ uint32_t elect_one() {
 // whole warp walks the issue loop, descriptors and addresses are warp-uniform values the compiler can keep in uniform
 // registers; inside an `if (lane == 0)` branch it cannot, and every MMA pays for moving its operands there -- about a
 // hundred clocks, more than a 128 x 128 x 16 MMA runs.
-template <int KIND>
+template <int KIND, int CTAS = 1>
 __device__ __forceinline__ void umma_elect(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate, uint32_t leader) {
-    if constexpr (KIND == 0)
-        asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
-                     "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
-                     : "memory");
-    else if constexpr (KIND == 1)
-        asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n@q tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
-                     "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
-                     : "memory");
-    else
-        asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n@q tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
-                     "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)
-                     : "memory");
+#define CYC_UMMA_ELECT_ASM(GROUP, KSTR)                                                                                     \
+    asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n@q tcgen05.mma.cta_group::" GROUP ".kind::" KSTR \
+                 " [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),                                                                \
+                 "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(leader)                                          \
+                 : "memory")
+    if constexpr (CTAS == 1) {
+        if constexpr (KIND == 0) CYC_UMMA_ELECT_ASM("1", "f16");
+        else if constexpr (KIND == 1) CYC_UMMA_ELECT_ASM("1", "i8");
+        else CYC_UMMA_ELECT_ASM("1", "tf32");
+    } else {
+        if constexpr (KIND == 0) CYC_UMMA_ELECT_ASM("2", "f16");
+        else if constexpr (KIND == 1) CYC_UMMA_ELECT_ASM("2", "i8");
+        else CYC_UMMA_ELECT_ASM("2", "tf32");
+    }
+#undef CYC_UMMA_ELECT_ASM
 }
 __device__ __forceinline__ void umma_commit_elect(uint64_t* bar, uint32_t leader) {
     asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(smem_u32(bar)),
                  "r"(leader)
                  : "memory");
+}
+
+__device__ __forceinline__ void umma_commit_pair_elect(uint64_t* bar, uint16_t cta_mask, uint32_t leader) {
+    asm volatile(
+        "{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n}" ::"r"(
+            smem_u32(bar)),
+        "h"(cta_mask), "r"(leader)
+        : "memory");
 }
 
 // make the mbarrier track completion of all tcgen05 operations issued so far by this thread

@@ -223,8 +223,10 @@ umma_recurrence_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer: the whole warp walks the loop
+        // ------------------------------------------------------------ converged, one elected lane issues
+        {
+            const uint32_t leader = ptx::elect_one();
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -248,12 +250,12 @@ umma_recurrence_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                         if constexpr (!B_MN) bdesc = umma_smem_desc(sb + k * 32, 16, 1024);
                         // B, MN-major: 128-byte rows of j, 8 k-rows per 1024 B group (stride dim), next j chunk BK*128 B on (leading dim)
                         else bdesc = umma_smem_desc(sb + k * (UK * 128), BK * 128, 1024);
-                        ptx::umma<KIND, 1>(d_tmem, adesc, bdesc, IDESC, (kb | k) != 0 ? 1u : 0u);
+                        ptx::umma_elect<KIND, 1>(d_tmem, adesc, bdesc, IDESC, (kb | k) != 0 ? 1u : 0u, leader);
                     }
-                    ptx::umma_commit(&ctl->empty[stage]);  // stage reusable once these MMAs have read it
+                    ptx::umma_commit_elect(&ctl->empty[stage], leader);  // stage reusable once these MMAs have read it
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (ok) ptx::umma_commit(&ctl->acc_full[ab]);  // [i,k_end]_C complete for this tile
+                if (ok) ptx::umma_commit_elect(&ctl->acc_full[ab], leader);  // [i,k_end]_C complete for this tile
             }
         }
         __syncwarp();

@@ -267,8 +267,10 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA only): the whole warp walks
+        // ------------------------------------------------------------ the loop converged, one elected lane issues
+        if (rank == 0) {
+            const uint32_t leader = ptx::elect_one();
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -295,12 +297,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         uint64_t bdesc;
                         if constexpr (!B_MN) bdesc = umma_smem_desc(sb + k * 32, 16, 1024);
                         else bdesc = umma_smem_desc(sb + k * (UK * 128), BK * 128, 1024);
-                        ptx::umma<KIND, 2>(d_tmem, adesc, bdesc, IDESC, (kb | k) != 0 ? 1u : 0u);
+                        ptx::umma_elect<KIND, 2>(d_tmem, adesc, bdesc, IDESC, (kb | k) != 0 ? 1u : 0u, leader);
                     }
-                    ptx::umma_commit_pair(&ctl->empty[stage], 3);  // both CTAs may refill this stage
+                    ptx::umma_commit_pair_elect(&ctl->empty[stage], 3, leader);  // both CTAs may refill this stage
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (ok) ptx::umma_commit_pair(&ctl->acc_full[ab], 3);  // [i,k_end]_C complete in both CTAs
+                if (ok) ptx::umma_commit_pair_elect(&ctl->acc_full[ab], 3, leader);  // [i,k_end]_C complete in both CTAs
             }
         }
         __syncwarp();

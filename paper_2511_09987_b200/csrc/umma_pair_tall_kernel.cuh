@@ -121,7 +121,8 @@ umma_pair_tall_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+        if (rank == 0) {  // the whole warp walks the loop converged, one elected lane issues
+            const uint32_t leader = ptx::elect_one();
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -143,13 +144,13 @@ umma_pair_tall_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                         if constexpr (!B_MN) bdesc = umma_smem_desc(sb + k * 32, 16, 1024);
                         else bdesc = umma_smem_desc(sb + k * (UK * 128), BK * 128, 1024);
                         const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
-                        ptx::umma<KIND, 2>(tmem_base, a0, bdesc, IDESC, acc);            // rows   0..255 of the tile
-                        ptx::umma<KIND, 2>(tmem_base + PAIR_BN, a1, bdesc, IDESC, acc);  // rows 256..511 of the tile
+                        ptx::umma_elect<KIND, 2>(tmem_base, a0, bdesc, IDESC, acc, leader);            // rows   0..255 of the tile
+                        ptx::umma_elect<KIND, 2>(tmem_base + PAIR_BN, a1, bdesc, IDESC, acc, leader);  // rows 256..511 of the tile
                     }
-                    ptx::umma_commit_pair(&ctl->empty[stage], 3);
+                    ptx::umma_commit_pair_elect(&ctl->empty[stage], 3, leader);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (ok) ptx::umma_commit_pair(&ctl->acc_full[0], 3);
+                if (ok) ptx::umma_commit_pair_elect(&ctl->acc_full[0], 3, leader);
             }
         }
         __syncwarp();

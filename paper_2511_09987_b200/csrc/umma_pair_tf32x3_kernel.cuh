@@ -182,7 +182,8 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+        if (rank == 0) {  // the whole warp walks the loop converged, one elected lane issues
+            const uint32_t leader = ptx::elect_one();
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -215,14 +216,14 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                             b_hi = umma_smem_desc(sb + k * (UK * 128), BK * 128, 512, 1);
                             b_lo = umma_smem_desc(sb + X3_STAGE_HI + k * (UK * 128), BK * 128, 512, 1);
                         }
-                        ptx::umma<KIND_TF32, 2>(d_tmem, a_lo, b_hi, IDESC, (kb | k) != 0 ? 1u : 0u);
-                        ptx::umma<KIND_TF32, 2>(d_tmem, a_hi, b_lo, IDESC, 1u);
-                        ptx::umma<KIND_TF32, 2>(d_tmem, a_hi, b_hi, IDESC, 1u);
+                        ptx::umma_elect<KIND_TF32, 2>(d_tmem, a_lo, b_hi, IDESC, (kb | k) != 0 ? 1u : 0u, leader);
+                        ptx::umma_elect<KIND_TF32, 2>(d_tmem, a_hi, b_lo, IDESC, 1u, leader);
+                        ptx::umma_elect<KIND_TF32, 2>(d_tmem, a_hi, b_hi, IDESC, 1u, leader);
                     }
-                    ptx::umma_commit_pair(&ctl->empty[stage], 3);
+                    ptx::umma_commit_pair_elect(&ctl->empty[stage], 3, leader);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (ok) ptx::umma_commit_pair(&ctl->acc_full[ab], 3);
+                if (ok) ptx::umma_commit_pair_elect(&ctl->acc_full[ab], 3, leader);
             }
         }
         __syncwarp();
