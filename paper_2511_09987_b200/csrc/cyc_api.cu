@@ -9,6 +9,7 @@
 #include <mutex>
 #include <set>
 #include <utility>
+#include <vector>
 #include <type_traits>
 
 #include <cuda.h>
@@ -1122,10 +1123,83 @@ extern "C" int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A,
 }
 
 // ------------------------------------------------------------------ tiled Cholesky
-// Panel j (columns c0 .. c1 of L), left-looking: one recurrence-matmul launch forms W = L[c0:n, 0:c0] L[c0:c1, 0:c0]^T
-// (the SYRK sum of the diagonal tile in its first rows, the GEMM sums of the tiles below it in the rest); the diagonal
-// tile is factored by chol_diag_kernel; the tiles below are the rows of X L_jj^T = A[c1:n, c0:c1] - W, solved by
-// trsm_diag_kernel with the right-hand sides addressed as rows.
+// Panel j (columns c0 .. c1 of L), left-looking.  The sums over the panels already factored,
+//     W = L[c0:n, 0:c0] L[c0:c1, 0:c0]^T ,
+// are recurrence-matmul launches (k cut into slices that run as the batch dimension, then summed in increasing k); the
+// diagonal tile A_jj - W is factored by chol_diag_kernel (one SM); the tiles below are the rows of
+// X L_jj^T = A[c1:n, c0:c1] - W, solved by trsm_diag_kernel with the right-hand sides addressed as rows.
+// The paper describes the recurrence as a wavefront that widens down the column; on a GPU the narrow end of that
+// wavefront is the one-SM diagonal tile, so the work is laid on two streams:
+//   the caller's stream carries the chain  sum of the diagonal tile -> diagonal tile (j) -> solve of the block row just
+//   below it -> sum of the next diagonal tile -> diagonal tile (j+1) ...,
+//   a helper stream carries the bulk: solve of the remaining rows of panel j, then the sums of everything below the
+//   next diagonal tile -- which run while diagonal tile j+1 is being factored.
+// Events order the two; every launch below names the data it needs.
+struct CholAux {
+    bool ready = false;
+    cudaStream_t side = nullptr;
+    std::vector<cudaEvent_t> events;
+    std::mutex mu;  // one factorisation at a time per device uses the helper stream
+};
+static int chol_aux(CholAux** out, size_t events) {
+    static std::mutex mu;
+    static CholAux aux[64];
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    CholAux& a = aux[dev];
+    if (!a.ready) {
+        CYC_CUDA(cudaStreamCreateWithFlags(&a.side, cudaStreamNonBlocking));
+        a.ready = true;
+    }
+    while (a.events.size() < events) {
+        cudaEvent_t e = nullptr;
+        CYC_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        a.events.push_back(e);
+    }
+    *out = &a;
+    return CYC_OK;
+}
+
+// W (plane 0) = L[r0:r1, 0:c0] L[c0:c0+w, 0:c0]^T on stream `s`; planes of `pstride` floats starting at W.  The k range
+// is cut into up to CHOL_MAX_SLICES equal slices (one batched launch: few 256-row tiles, and the slices give every CTA
+// pair work) plus one launch for the remainder; the slices' partial sums are then added in increasing k into plane 0.
+constexpr int CHOL_MAX_SLICES = 8;        // sums below a diagonal tile: several 256-row tiles share the CTA pairs
+constexpr int CHOL_MAX_SLICES_DIAG = 64;  // sum of a diagonal tile: one tile, so every panel of k can be a slice of its own
+static int chol_product(cudaStream_t s, float* Lf, long long n, long long T, long long c0, long long w, long long r0, long long r1, float* W,
+                        long long pstride, unsigned flags, int max_slices) {
+    const long long rows = r1 - r0;
+    const long long kblocks = c0 / T, tiles_m = (rows + 255) / 256;
+    const long long smax = std::min<long long>({static_cast<long long>(max_slices), kblocks, std::max<long long>(1, kCtaPairs / tiles_m)});
+    // slices of ceil(kblocks / smax) panels, so that the remainder (one more launch) is shorter than a slice
+    const long long per = (kblocks + smax - 1) / smax, S = kblocks / per;
+    const long long kc = per * T, rem = c0 - S * kc;
+    const unsigned gflags = (flags & CYC_FLAG_FIXED_K_ORDER) | CYC_FLAG_B_COL_MAJOR;
+    Problem q{S, rows, w, kc, CYC_F32, Lf + r0 * n, Lf + c0 * n, W, kc, kc, pstride, gflags, n, n};
+    int rc = route(q, s);
+    if (rc) return rc;
+    int planes = static_cast<int>(S);
+    if (rem > 0) {
+        Problem r{1, rows, w, rem, CYC_F32, Lf + r0 * n + S * kc, Lf + c0 * n + S * kc, W + S * pstride, rows * n, w * n, pstride, gflags, n, n};
+        rc = route(r, s);
+        if (rc) return rc;
+        ++planes;
+    }
+    if (planes > 1) {
+        DeviceInfo di;
+        rc = device_info(&di);
+        if (rc) return rc;
+        const long long work = pstride / 4;
+        const long long blocks = std::min<long long>((work + 127) / 128, 16ll * di.sms);
+        cudaError_t e = launch_pdl(splitk_reduce_kernel<float>, static_cast<unsigned>(blocks), 128, 0, s, static_cast<const float*>(W), W, pstride,
+                                   pstride, planes, 1ll, 1);
+        if (e != cudaSuccess) return cuda_fail(e, "splitk_reduce_kernel");
+        g_launches.fetch_add(1);
+    }
+    return CYC_OK;
+}
+
 extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, void* L, void* stream, unsigned flags) {
     if (n <= 0 || tile < 0 || tile > CHOL_T_MAX || !A || !L) return CYC_ERR_INVALID_ARG;
     if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
@@ -1141,88 +1215,91 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
     float* Lf = static_cast<float*>(L);
     const long long T = tile ? tile : CHOL_T_MAX;
     const bool in_place = a0 == l0;
+    const long long panels = (n + T - 1) / T;
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(chol_diag_kernel), CHOL_SMEM_BYTES)) return rc_;
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel), TRSM_SMEM_BYTES)) return rc_;
-    // The k range of a panel's sums is cut into up to CHOL_MAX_SLICES equal slices (one batched launch: a panel has
-    // few 256-row tiles, and the slices give every CTA pair work) plus one launch for the remainder; the consumers
-    // add the slices' partial sums in increasing k.
-    constexpr int CHOL_MAX_SLICES = 8;
-    float* W = nullptr;
-    const long long plane = (n - T) * T;
+    CholAux* aux = nullptr;
+    if (int rc_ = chol_aux(&aux, static_cast<size_t>(3 * panels + 2))) return rc_;
+    std::lock_guard<std::mutex> aux_lock(aux->mu);
+    cudaStream_t side = aux->side;
+    auto ev = [&](long long j, int which) { return aux->events[static_cast<size_t>(3 * j + which)]; };  // 0: D(j), 1: near solve (j), 2: sums below (j)
+    cudaEvent_t ev_fork = aux->events[static_cast<size_t>(3 * panels)], ev_join = aux->events[static_cast<size_t>(3 * panels + 1)];
+
+    // workspace: planes of the diagonal tile's sums and planes of the sums below it (the two streams never share a plane)
+    const long long pd = (T * T + 3) / 4 * 4, pb = ((n - T) * T + 3) / 4 * 4;
+    float* Wd = nullptr;
+    float* Wb = nullptr;
     if (n > T) {
         cudaMemPool_t pool;
         int rc = workspace_pool(&pool);
         if (rc) return rc;
         void* ws = nullptr;
-        CYC_CUDA(cudaMallocFromPoolAsync(&ws, static_cast<size_t>(CHOL_MAX_SLICES + 1) * (plane + 4) * sizeof(float), pool, st));
-        W = static_cast<float*>(ws);
+        CYC_CUDA(cudaMallocFromPoolAsync(&ws, (static_cast<size_t>(CHOL_MAX_SLICES_DIAG + 1) * pd + static_cast<size_t>(CHOL_MAX_SLICES + 1) * pb) * sizeof(float), pool, st));
+        Wd = static_cast<float*>(ws);
+        Wb = Wd + (CHOL_MAX_SLICES_DIAG + 1) * pd;
     }
     int rc = CYC_OK;
-    for (long long c0 = 0; c0 < n && rc == CYC_OK; c0 += T) {
-        const long long c1 = std::min<long long>(n, c0 + T), w = c1 - c0, below = n - c1;
-        int planes = 0;
-        // this panel's planes lie back to back, each (n - c0) x w floats rounded up to a multiple of four
-        const long long pstride = ((n - c0) * w + 3) / 4 * 4;
+    auto ok = [&](cudaError_t e, const char* what) {
+        if (e != cudaSuccess && rc == CYC_OK) rc = cuda_fail(e, what);
+        return rc == CYC_OK;
+    };
+    // rows [r0, r1) of panel (c0, w): X L_jj^T = A - W, the right-hand sides addressed as rows
+    auto solve_rows = [&](cudaStream_t s, long long c0, long long w, long long c1, long long r0, long long r1, bool have_w, long long pstride) {
+        TrsmDiagParams p;
+        p.L = Lf;
+        p.B = Af + r0 * n + c0; p.X = Lf + r0 * n + c0; p.W = have_w ? Wb + (r0 - c1) * w : nullptr;
+        p.plane = pstride;
+        p.b_r = 1; p.b_c = n; p.x_r = 1; p.x_c = n; p.w_r = 1; p.w_c = w;
+        p.n = static_cast<int>(n); p.m = static_cast<int>(r1 - r0);
+        p.r0 = static_cast<int>(c0); p.rows = static_cast<int>(w);
+        p.mask = have_w ? 1u : 0u;
+        if (ok(launch_pdl(trsm_diag_kernel, static_cast<unsigned>((r1 - r0 + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, s, p), "trsm_diag_kernel"))
+            g_launches.fetch_add(1);
+    };
+
+    ok(cudaEventRecord(ev_fork, st), "cudaEventRecord");
+    ok(cudaStreamWaitEvent(side, ev_fork, 0), "cudaStreamWaitEvent");
+    for (long long j = 0; j < panels && rc == CYC_OK; ++j) {
+        const long long c0 = j * T, c1 = std::min<long long>(n, c0 + T), w = c1 - c0, c2 = std::min<long long>(n, c1 + T);
+        // ---- caller's stream: the sum of the diagonal tile (needs row block j of every earlier panel: the near solve of
+        // ---- panel j-1 is on this stream, the far solves of older panels were waited for with the sums below panel j-1)
         if (c0 > 0) {
-            const long long kblocks = c0 / T, tiles_m = (n - c0 + 255) / 256;
-            long long S = std::min<long long>({static_cast<long long>(CHOL_MAX_SLICES), kblocks, std::max<long long>(1, kCtaPairs / tiles_m)});
-            const long long kc = (kblocks / S) * T, rem = c0 - S * kc;
-            const unsigned gflags = (flags & CYC_FLAG_FIXED_K_ORDER) | CYC_FLAG_B_COL_MAJOR;
-            Problem q{S, n - c0, w, kc, CYC_F32, Lf + c0 * n, Lf + c0 * n, W, kc, kc, pstride, gflags, n, n};
-            rc = route(q, st);
+            rc = chol_product(st, Lf, n, T, c0, w, c0, c1, Wd, pd, flags, CHOL_MAX_SLICES_DIAG);
             if (rc) break;
-            planes = static_cast<int>(S);
-            if (rem > 0) {
-                Problem r{1, n - c0, w, rem, CYC_F32, Lf + c0 * n + S * kc, Lf + c0 * n + S * kc, W + S * pstride, (n - c0) * n, w * n, pstride,
-                          gflags, n, n};
-                rc = route(r, st);
-                if (rc) break;
-                ++planes;
-            }
-            if (planes > 1) {
-                // the slices' partial sums added in increasing k into the first plane, by all SMs at once, so that the
-                // two consumers (one CTA for the diagonal tile, few CTAs per solve) read a single plane
-                DeviceInfo di;
-                rc = device_info(&di);
-                if (rc) break;
-                const long long work = pstride / 4;
-                long long blocks = std::min<long long>((work + 127) / 128, 16ll * di.sms);
-                cudaError_t e = launch_pdl(splitk_reduce_kernel<float>, static_cast<unsigned>(blocks), 128, 0, st, static_cast<const float*>(W), W,
-                                           pstride, pstride, planes, 1ll, 1);
-                if (e != cudaSuccess) { rc = cuda_fail(e, "splitk_reduce_kernel"); break; }
-                g_launches.fetch_add(1);
-                planes = 1;
-            }
         }
         CholDiagParams d;
-        d.A = Af + c0 * n + c0; d.W = W; d.L = Lf + c0 * n + c0;
-        d.plane = pstride; d.planes = planes;
+        d.A = Af + c0 * n + c0; d.W = Wd; d.L = Lf + c0 * n + c0;
+        d.plane = pd; d.planes = c0 > 0 ? 1 : 0;
         d.lda = n; d.ldw = w; d.ldl = n;
         d.rows = static_cast<int>(w);
         d.zero_upper = in_place ? 0 : 1;
-        cudaError_t e = launch_pdl(chol_diag_kernel, 1u, CHOL_THREADS, CHOL_SMEM_BYTES, st, d);
-        if (e != cudaSuccess) { rc = cuda_fail(e, "chol_diag_kernel"); break; }
+        if (!ok(launch_pdl(chol_diag_kernel, 1u, CHOL_THREADS, CHOL_SMEM_BYTES, st, d), "chol_diag_kernel")) break;
         g_launches.fetch_add(1);
-        if (below > 0) {
-            TrsmDiagParams p;
-            p.L = Lf;
-            p.B = Af + c1 * n + c0; p.X = Lf + c1 * n + c0; p.W = planes ? W + w * w : nullptr;
-            p.plane = pstride;
-            p.b_r = 1; p.b_c = n; p.x_r = 1; p.x_c = n; p.w_r = 1; p.w_c = w;
-            p.n = static_cast<int>(n); p.m = static_cast<int>(below);
-            p.r0 = static_cast<int>(c0); p.rows = static_cast<int>(w);
-            p.mask = planes ? ((1u << planes) - 1u) : 0u;
-            e = launch_pdl(trsm_diag_kernel, static_cast<unsigned>((below + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, st, p);
-            if (e != cudaSuccess) { rc = cuda_fail(e, "trsm_diag_kernel"); break; }
-            g_launches.fetch_add(1);
-            if (!in_place) {  // zeros above the diagonal: the block row to the right of the diagonal tile
-                e = cudaMemset2DAsync(Lf + c0 * n + c1, static_cast<size_t>(n) * 4, 0, static_cast<size_t>(below) * 4, static_cast<size_t>(w), st);
-                if (e != cudaSuccess) { rc = cuda_fail(e, "cudaMemset2DAsync"); break; }
-            }
+        if (c1 >= n) break;
+        ok(cudaEventRecord(ev(j, 0), st), "cudaEventRecord");
+        const long long pstride_b = ((n - c1) * w + 3) / 4 * 4;
+        // ---- caller's stream: the block row just below the diagonal tile (needs its sums, formed on the helper stream)
+        if (c0 > 0) ok(cudaStreamWaitEvent(st, ev(j, 2), 0), "cudaStreamWaitEvent");
+        if (rc == CYC_OK) solve_rows(st, c0, w, c1, c1, c2, c0 > 0, pstride_b);
+        ok(cudaEventRecord(ev(j, 1), st), "cudaEventRecord");
+        // ---- helper stream: the remaining rows of the panel (need the diagonal tile; their sums are on this stream)
+        ok(cudaStreamWaitEvent(side, ev(j, 0), 0), "cudaStreamWaitEvent");
+        if (c2 < n && rc == CYC_OK) solve_rows(side, c0, w, c1, c2, n, c0 > 0, pstride_b);
+        if (!in_place)  // zeros above the diagonal: the block row to the right of the diagonal tile
+            ok(cudaMemset2DAsync(Lf + c0 * n + c1, static_cast<size_t>(n) * 4, 0, static_cast<size_t>(n - c1) * 4, static_cast<size_t>(w), side), "cudaMemset2DAsync");
+        // ---- helper stream: the sums below the NEXT diagonal tile (need block row j+1 of this panel: the near solve)
+        if (c2 < n && rc == CYC_OK) {
+            const long long w1 = c2 - c1, pstride_n = ((n - c2) * w1 + 3) / 4 * 4;
+            ok(cudaStreamWaitEvent(side, ev(j, 1), 0), "cudaStreamWaitEvent");
+            if (rc == CYC_OK) rc = chol_product(side, Lf, n, T, c1, w1, c2, n, Wb, pstride_n, flags, CHOL_MAX_SLICES);
+            ok(cudaEventRecord(ev(j + 1, 2), side), "cudaEventRecord");
         }
     }
-    if (W) {
-        cudaError_t e = cudaFreeAsync(W, st);
+    // the caller's stream continues only after the helper stream has finished
+    if (cudaEventRecord(ev_join, side) == cudaSuccess) cudaStreamWaitEvent(st, ev_join, 0);
+    else cudaStreamSynchronize(side);
+    if (Wd) {
+        cudaError_t e = cudaFreeAsync(Wd, st);
         if (e != cudaSuccess && rc == CYC_OK) rc = cuda_fail(e, "cudaFreeAsync");
     }
     return rc;
