@@ -13,8 +13,10 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcyc.so")
-NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
-              "-Xcompiler", "-fPIC", "--cudart", "static"]
+ARCH_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a"]
+COMPILE_FLAGS = [*ARCH_FLAGS, "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
+LINK_FLAGS = [*ARCH_FLAGS, "-shared", "-Xcompiler", "-fPIC", "--cudart", "static"]
+OBJ_DIR = os.path.join(HERE, "_build")
 
 
 def _nvcc() -> str:
@@ -41,11 +43,29 @@ def stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or stale():
+        from concurrent.futures import ThreadPoolExecutor
         cu = [s for s in sources() if s.endswith(".cu")]
+        os.makedirs(OBJ_DIR, exist_ok=True)
+        nvcc = _nvcc()
+
+        def compile_one(src):  # one translation unit per recurrence, compiled side by side
+            obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".%d.o" % os.getpid())
+            cmd = [nvcc, *COMPILE_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-c", "-o", obj, src]
+            out = subprocess.run(cmd, cwd=HERE, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+            return obj, out
+
+        with ThreadPoolExecutor(max_workers=min(len(cu), os.cpu_count() or 1)) as pool:
+            results = list(pool.map(compile_one, cu))
+        for obj, out in results:
+            if out.stdout and (verbose or out.returncode):
+                sys.stderr.write(out.stdout)
+            if out.returncode:
+                raise subprocess.CalledProcessError(out.returncode, out.args)
         tmp = LIB + ".tmp.%d" % os.getpid()
-        cmd = [_nvcc(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp, *cu]
-        subprocess.check_call(cmd, cwd=HERE)
+        subprocess.check_call([nvcc, *LINK_FLAGS, "-o", tmp, *[obj for obj, _ in results]], cwd=HERE)
         os.replace(tmp, LIB)
+        for obj, _ in results:
+            os.remove(obj)
     return LIB
 
 

@@ -1,0 +1,210 @@
+// Shared state and helpers of the library, and the status / introspection entry points.  See include/cyc.h.
+#include "api_internal.h"
+#include "ptx.cuh"
+
+namespace cyc {
+
+// raised by a kernel whose bounded wait ran out; one word per device (module scope)
+__device__ int g_device_status = 0;
+// Self-test of the bounded-wait path: one CTA waits on an mbarrier that nothing ever arrives on, with a
+// caller-chosen clock budget, and reports through the same status word and abort flag as the real kernels.
+__global__ void bounded_wait_selftest_kernel(long long budget_cycles, int* status) {
+    __shared__ uint64_t bar;
+    __shared__ volatile int abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(&bar, 0)) {
+            if (clock64() - t0 > budget_cycles) {
+                abort_flag = 1;
+                atomicExch(status, 0x7f0);
+                break;
+            }
+        }
+    } else {
+        // the other role polls the abort flag the way the kernels' roles do, with its own (larger) budget
+        const long long t0 = clock64();
+        while (!abort_flag && clock64() - t0 < 64 * budget_cycles) {}
+    }
+    __syncthreads();
+}
+std::atomic<long long> g_launches{0};
+thread_local char g_err[512] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_err, sizeof g_err, "%s: %s", what, cudaGetErrorString(e));
+    return CYC_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static int get_encoder(EncodeTiledFn* out) {
+    static std::mutex mu;
+    static EncodeTiledFn fn = nullptr;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        CYC_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr));
+        if (qr != cudaDriverEntryPointSuccess || !sym) {
+            snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled not available from the driver");
+            return CYC_ERR_CUDA;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    *out = fn;
+    return CYC_OK;
+}
+
+// rank-3 map over a [d2][d1][d0] array (d0 contiguous), box [1][box1][box0], 128-byte swizzle
+int make_map_raw(CUtensorMap* m, CUtensorMapDataType dt, int eb, const void* base, long long d0, long long d1, long long d2,
+                        long long pitch1_elems, long long pitch2_elems, int box0, int box1,
+                        CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn enc;
+    int rc = get_encoder(&enc);
+    if (rc) return rc;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d0), static_cast<cuuint64_t>(d1), static_cast<cuuint64_t>(d2)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch1_elems) * eb, static_cast<cuuint64_t>(pitch2_elems) * eb};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(box0), static_cast<cuuint32_t>(box1), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+        return CYC_ERR_CUDA;
+    }
+    return CYC_OK;
+}
+
+// operand map (A or B) in the problem's input type
+int make_map(CUtensorMap* m, int dtype, const void* base, long long d0, long long d1, long long d2, long long pitch1_elems,
+                    long long pitch2_elems, int box0, int box1, CUtensorMapSwizzle swizzle) {
+    const CUtensorMapDataType dt = dtype == CYC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                    : (dtype == CYC_BF16_F32 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
+    return make_map_raw(m, dt, elem_bytes(dtype), base, d0, d1, d2, pitch1_elems, pitch2_elems, box0, box1, swizzle);
+}
+
+int device_info(DeviceInfo* out) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(mu);
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    if (!cache[dev].known) {
+        CYC_CUDA(cudaDeviceGetAttribute(&cache[dev].sms, cudaDevAttrMultiProcessorCount, dev));
+        CYC_CUDA(cudaDeviceGetAttribute(&cache[dev].cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+        cache[dev].known = true;
+    }
+    *out = cache[dev];
+    return CYC_OK;
+}
+// Once per device: the address of the status word, and the opt-in to more than 48 KB of dynamic shared memory for a
+// kernel.  Both are remembered so that the per-call path makes neither runtime call again.
+int status_word(int** out) {
+    static std::mutex mu;
+    static int* addr[64] = {};
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!addr[dev]) CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&addr[dev]), g_device_status));
+    *out = addr[dev];
+    return CYC_OK;
+}
+
+int ensure_dynamic_smem(const void* kernel, int bytes) {
+    static std::mutex mu;
+    static std::set<std::pair<const void*, int>> done;
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(mu);
+    if (done.count({kernel, dev})) return CYC_OK;
+    CYC_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    done.insert({kernel, dev});
+    return CYC_OK;
+}
+// Workspace for partial sums and scratch: stream-ordered allocations from a pool the library owns (one per device),
+// so that repeated calls reuse the same memory without a synchronising cudaMalloc.
+int workspace_pool(cudaMemPool_t* out, bool create) {
+    static std::mutex mu;
+    static cudaMemPool_t pools[64] = {};
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!pools[dev] && create) {
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        CYC_CUDA(cudaMemPoolCreate(&pools[dev], &props));
+        unsigned long long keep = ~0ull;  // keep freed blocks for the next call instead of returning them to the driver
+        CYC_CUDA(cudaMemPoolSetAttribute(pools[dev], cudaMemPoolAttrReleaseThreshold, &keep));
+    }
+    *out = pools[dev];
+    return CYC_OK;
+}
+}  // namespace cyc
+
+using namespace cyc;
+
+extern "C" int cyc_pool_reserved_bytes(int64_t* out) {
+    if (!out) return CYC_ERR_INVALID_ARG;
+    *out = 0;
+    cudaMemPool_t pool = nullptr;
+    int rc = workspace_pool(&pool, /*create=*/false);
+    if (rc) return rc;
+    if (pool) {
+        unsigned long long bytes = 0;
+        CYC_CUDA(cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReservedMemCurrent, &bytes));
+        *out = static_cast<int64_t>(bytes);
+    }
+    return CYC_OK;
+}
+extern "C" int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles) {
+    if (budget_cycles < 1 || budget_cycles > (1ll << 24)) return CYC_ERR_INVALID_ARG;  // at most ~10 ms
+    int* status = nullptr;
+    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_device_status));
+    bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(budget_cycles, status);
+    CYC_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
+extern "C" int cyc_last_device_status(void* stream, int* out) {
+    CYC_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int word = 0;
+    CYC_CUDA(cudaMemcpyFromSymbol(&word, g_device_status, sizeof word));
+    if (word != 0) {
+        const int zero = 0;
+        tail_scratch_mark_dirty();  // a kernel that gave up may have left strip counters of the sliced tail non-zero
+        CYC_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero));
+        snprintf(g_err, sizeof g_err, "device wait ran out (code 0x%x)", word);
+    }
+    if (out) *out = word != 0 ? CYC_ERR_TIMEOUT : CYC_OK;
+    return CYC_OK;
+}
+extern "C" int64_t cyc_launch_count(void) { return g_launches.load(); }
+extern "C" const char* cyc_last_cuda_error(void) { return g_err; }
+
+extern "C" const char* cyc_status_string(int s) {
+    switch (s) {
+        case CYC_OK: return "ok";
+        case CYC_ERR_INVALID_ARG: return "invalid argument";
+        case CYC_ERR_UNSUPPORTED: return "unsupported";
+        case CYC_ERR_CUDA: return "CUDA error";
+        case CYC_ERR_TIMEOUT: return "device wait timed out";
+        default: return "unknown status";
+    }
+}
+extern "C" int cyc_version(void) { return 100; }

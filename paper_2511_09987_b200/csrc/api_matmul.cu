@@ -1,117 +1,21 @@
-// C ABI of the library: argument validation, kernel selection, tensor-map
-// construction and launches.  See include/cyc.h for the contract.
-#include <algorithm>
-#include <atomic>
-#include <cmath>
-#include <cstdint>
-#include <cstdio>
-#include <cstring>
-#include <mutex>
-#include <set>
-#include <utility>
-#include <vector>
-#include <type_traits>
-
-#include <cuda.h>
-#include <cuda_bf16.h>
-#include <cuda_runtime.h>
-
-#include "../../include/cyc.h"
+// The matrix-multiply recurrence: kernel selection, tensor-map construction, launches, and the entry points
+// cyc_recurrence_matmul, _batched, _host, _splitk_static, cyc_kernel_for and cyc_schedule_for.  See include/cyc.h.
+#include "api_internal.h"
 #include "simt_kernel.cuh"
 #include "umma_kernel.cuh"
 #include "umma_pair_kernel.cuh"
 #include "umma_pair_tall_kernel.cuh"
 #include "splitk_reduce_kernel.cuh"
 #include "umma_pair_tf32x3_kernel.cuh"
-#include "trsm_diag_kernel.cuh"
-#include "fa2_kernel.cuh"
-#include "scan_kernel.cuh"
-#include "chol_diag_kernel.cuh"
 
 namespace cyc {
-
-// raised by a kernel whose bounded wait ran out; one word per device (module scope)
-__device__ int g_device_status = 0;
 
 // Fixed workspace of cyc_recurrence_matmul_splitk_static: lives in every device that loads the library, from load
 // to exit.  In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.
 static __device__ __align__(256) unsigned char g_static_workspace[CYC_STATIC_WORKSPACE_BYTES];
 
-// Self-test of the bounded-wait path: one CTA waits on an mbarrier that nothing ever arrives on, with a
-// caller-chosen clock budget, and reports through the same status word and abort flag as the real kernels.
-__global__ void bounded_wait_selftest_kernel(long long budget_cycles, int* status) {
-    __shared__ uint64_t bar;
-    __shared__ volatile int abort_flag;
-    if (threadIdx.x == 0) {
-        ptx::mbar_init(&bar, 1);
-        abort_flag = 0;
-        ptx::fence_mbar_init();
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const long long t0 = clock64();
-        while (!ptx::mbar_try_wait(&bar, 0)) {
-            if (clock64() - t0 > budget_cycles) {
-                abort_flag = 1;
-                atomicExch(status, 0x7f0);
-                break;
-            }
-        }
-    } else {
-        // the other role polls the abort flag the way the kernels' roles do, with its own (larger) budget
-        const long long t0 = clock64();
-        while (!abort_flag && clock64() - t0 < 64 * budget_cycles) {}
-    }
-    __syncthreads();
-}
-
-static std::atomic<long long> g_launches{0};
-static thread_local char g_err[512] = "";
-
-static int cuda_fail(cudaError_t e, const char* what) {
-    snprintf(g_err, sizeof g_err, "%s: %s", what, cudaGetErrorString(e));
-    return CYC_ERR_CUDA;
-}
-#define CYC_CUDA(call)                                    \
-    do {                                                  \
-        cudaError_t e_ = (call);                          \
-        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
-    } while (0)
-
-// Launch with programmatic stream serialisation: the kernel may be scheduled while the kernel before it on the stream
-// is still running; each kernel launched this way executes griddepcontrol.wait before it touches global memory.
-template <typename... KArgs, typename... Args>
-static cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args&&... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid, 1, 1);
-    cfg.blockDim = dim3(block, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
-}
-
-static int elem_bytes(int dtype) { return dtype == CYC_F32 ? 4 : (dtype == CYC_BF16_F32 ? 2 : 1); }
-
-struct Problem {
-    long long batch, M, N, K;
-    int dtype;
-    const void *A, *B;
-    void* C;
-    long long sA, sB, sC;
-    unsigned flags;
-    long long lda = 0;  // row pitch of A in elements; 0 = dense (K).  Only internal callers set it (sub-blocks of L).
-    long long ldb = 0;  // pitch of B in elements (between rows k, or between columns j when stored [N][K]); 0 = dense
-};
-static long long lda_of(const Problem& q) { return q.lda ? q.lda : q.K; }
-static long long ldb_of(const Problem& q) { return q.ldb ? q.ldb : ((q.flags & CYC_FLAG_B_COL_MAJOR) ? q.K : q.N); }
-
 // host-side validation; no CUDA call
-static int validate(const Problem& q) {
+int validate(const Problem& q) {
     if (q.dtype != CYC_F32 && q.dtype != CYC_BF16_F32 && q.dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
     if (q.flags & ~(CYC_FLAG_FIXED_K_ORDER | CYC_FLAG_B_COL_MAJOR)) return CYC_ERR_INVALID_ARG;
     if (q.batch <= 0 || q.M <= 0 || q.N <= 0 || q.K <= 0) return CYC_ERR_INVALID_ARG;
@@ -131,7 +35,6 @@ static int validate(const Problem& q) {
 }
 
 enum Family { FAM_SIMT = 0, FAM_UMMA = 1, FAM_UMMA_3XTF32 = 2, FAM_UMMA_PAIR = 3, FAM_UMMA_TALL = 4, FAM_UMMA_SPLITK = 5 };
-constexpr long long kCtaPairs = 74;  // CTA pairs resident on a B200 (148 SMs); used by the tile-shape rule
 
 // the tensor-core kernels move tiles with TMA: 16-byte aligned bases and pitches
 static bool tma_ok(const Problem& q) {
@@ -184,7 +87,6 @@ static Family choose(const Problem& q) {
         return plan_split_k(q).S > 1 ? FAM_UMMA_SPLITK : FAM_UMMA_PAIR;
     return FAM_UMMA;
 }
-
 // ------------------------------------------------------------------ SIMT launch
 template <typename TIn, typename TAcc>
 static int launch_simt(const Problem& q, cudaStream_t st) {
@@ -225,108 +127,10 @@ static int launch_simt(const Problem& q, cudaStream_t st) {
     g_launches.fetch_add(1);
     return CYC_OK;
 }
-
-// ------------------------------------------------------------------ tensor maps
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static int get_encoder(EncodeTiledFn* out) {
-    static std::mutex mu;
-    static EncodeTiledFn fn = nullptr;
-    std::lock_guard<std::mutex> lk(mu);
-    if (!fn) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        CYC_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr));
-        if (qr != cudaDriverEntryPointSuccess || !sym) {
-            snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled not available from the driver");
-            return CYC_ERR_CUDA;
-        }
-        fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    *out = fn;
-    return CYC_OK;
-}
-
-// rank-3 map over a [d2][d1][d0] array (d0 contiguous), box [1][box1][box0], 128-byte swizzle
-static int make_map_raw(CUtensorMap* m, CUtensorMapDataType dt, int eb, const void* base, long long d0, long long d1, long long d2,
-                        long long pitch1_elems, long long pitch2_elems, int box0, int box1,
-                        CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
-    EncodeTiledFn enc;
-    int rc = get_encoder(&enc);
-    if (rc) return rc;
-    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d0), static_cast<cuuint64_t>(d1), static_cast<cuuint64_t>(d2)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch1_elems) * eb, static_cast<cuuint64_t>(pitch2_elems) * eb};
-    cuuint32_t box[3] = {static_cast<cuuint32_t>(box0), static_cast<cuuint32_t>(box1), 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = enc(m, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
-        return CYC_ERR_CUDA;
-    }
-    return CYC_OK;
-}
-
-// operand map (A or B) in the problem's input type
-static int make_map(CUtensorMap* m, int dtype, const void* base, long long d0, long long d1, long long d2, long long pitch1_elems,
-                    long long pitch2_elems, int box0, int box1, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
-    const CUtensorMapDataType dt = dtype == CYC_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
-                                                    : (dtype == CYC_BF16_F32 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8);
-    return make_map_raw(m, dt, elem_bytes(dtype), base, d0, d1, d2, pitch1_elems, pitch2_elems, box0, box1, swizzle);
-}
-
 // result map: C[batch][M][N] of 32-bit words, boxes of 32 rows x 32 columns (128 bytes)
 static int make_c_map(CUtensorMap* m, int dtype, void* C, long long M, long long N, long long batch, long long sC) {
     const CUtensorMapDataType dt = dtype == CYC_I8_I32 ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
     return make_map_raw(m, dt, 4, C, N, M, batch, N, sC, 32, 32);
-}
-
-struct DeviceInfo {
-    int sms = 0, cc_major = 0;
-    bool known = false;
-};
-static int device_info(DeviceInfo* out) {
-    static std::mutex mu;
-    static DeviceInfo cache[64];
-    int dev = 0;
-    CYC_CUDA(cudaGetDevice(&dev));
-    std::lock_guard<std::mutex> lk(mu);
-    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
-    if (!cache[dev].known) {
-        CYC_CUDA(cudaDeviceGetAttribute(&cache[dev].sms, cudaDevAttrMultiProcessorCount, dev));
-        CYC_CUDA(cudaDeviceGetAttribute(&cache[dev].cc_major, cudaDevAttrComputeCapabilityMajor, dev));
-        cache[dev].known = true;
-    }
-    *out = cache[dev];
-    return CYC_OK;
-}
-
-// Once per device: the address of the status word, and the opt-in to more than 48 KB of dynamic shared memory for a
-// kernel.  Both are remembered so that the per-call path makes neither runtime call again.
-static int status_word(int** out) {
-    static std::mutex mu;
-    static int* addr[64] = {};
-    int dev = 0;
-    CYC_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lk(mu);
-    if (!addr[dev]) CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&addr[dev]), g_device_status));
-    *out = addr[dev];
-    return CYC_OK;
-}
-
-static int ensure_dynamic_smem(const void* kernel, int bytes) {
-    static std::mutex mu;
-    static std::set<std::pair<const void*, int>> done;
-    int dev = 0;
-    CYC_CUDA(cudaGetDevice(&dev));
-    std::lock_guard<std::mutex> lk(mu);
-    if (done.count({kernel, dev})) return CYC_OK;
-    CYC_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-    done.insert({kernel, dev});
-    return CYC_OK;
 }
 
 // ------------------------------------------------------------------ tensor-core launch
@@ -404,7 +208,7 @@ static std::mutex g_tail_mu;
 static TailScratch g_tail_scratch[64];
 static int g_tail_scratch_count = 0;
 
-static void tail_scratch_mark_dirty() {
+void tail_scratch_mark_dirty() {
     std::lock_guard<std::mutex> lk(g_tail_mu);
     for (int i = 0; i < g_tail_scratch_count; ++i) g_tail_scratch[i].dirty = true;
 }
@@ -506,31 +310,7 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws 
     g_launches.fetch_add(1);
     return CYC_OK;
 }
-
 // ------------------------------------------------------------------ split-K
-// Workspace for the partial sums: stream-ordered allocations from a pool the library owns (one per device),
-// so that repeated calls reuse the same memory without a synchronising cudaMalloc.
-static int workspace_pool(cudaMemPool_t* out, bool create = true) {
-    static std::mutex mu;
-    static cudaMemPool_t pools[64] = {};
-    int dev = 0;
-    CYC_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lk(mu);
-    if (!pools[dev] && create) {
-        cudaMemPoolProps props = {};
-        props.allocType = cudaMemAllocationTypePinned;
-        props.handleTypes = cudaMemHandleTypeNone;
-        props.location.type = cudaMemLocationTypeDevice;
-        props.location.id = dev;
-        CYC_CUDA(cudaMemPoolCreate(&pools[dev], &props));
-        unsigned long long keep = ~0ull;  // keep freed blocks for the next call instead of returning them to the driver
-        CYC_CUDA(cudaMemPoolSetAttribute(pools[dev], cudaMemPoolAttrReleaseThreshold, &keep));
-    }
-    *out = pools[dev];
-    return CYC_OK;
-}
-
 // partial sums of plan.S k-slices into the workspace (CTA-pair kernel), then their sum in slice order into C.
 // `ws` = nullptr: the workspace comes from the library's pool for the duration of the two kernels.
 template <int KIND>
@@ -668,7 +448,7 @@ static int launch_umma(const Problem& q, cudaStream_t st) {
 }
 
 // kernel selection and launch for a validated problem (also used for the sub-problems the library builds itself)
-static int route(const Problem& q, cudaStream_t st) {
+int route(const Problem& q, cudaStream_t st) {
     switch (choose(q)) {
         case FAM_UMMA:
         case FAM_UMMA_PAIR:
@@ -684,97 +464,13 @@ static int route(const Problem& q, cudaStream_t st) {
     }
 }
 
-static int dispatch(const Problem& q, cudaStream_t st) {
+int dispatch(const Problem& q, cudaStream_t st) {
     int rc = validate(q);
     if (rc) return rc;
     return route(q, st);
 }
-
-// ------------------------------------------------------------------ block lower-triangular solve
-// X_i = TRSM(L_ii, B_i - sum_{j<i} GEMM(L_ij, X_j)).  The block rows are split recursively: solve the upper part,
-// form the partial sums of the lower part's rows over the solved block columns with one recurrence-matmul launch
-// (triangular space; written to the plane of this recursion level), solve the lower part.  A diagonal tile subtracts
-// the planes of every level that covered its rows (its end-of-row accumulator) and solves (diagonal space).
-struct TrsmPlan {
-    long long n, m, T;
-    const float* L;
-    const float* B;
-    float* X;
-    float* W;
-    long long plane;
-    unsigned flags;
-    cudaStream_t st;
-};
-
-static int trsm_diag(const TrsmPlan& t, long long b, unsigned mask) {
-    TrsmDiagParams p;
-    p.L = t.L;
-    p.B = t.B + b * t.T * t.m; p.X = t.X + b * t.T * t.m; p.W = t.W ? t.W + b * t.T * t.m : nullptr;  // first row of the tile
-    p.plane = t.plane;
-    p.b_r = p.x_r = p.w_r = t.m;
-    p.b_c = p.x_c = p.w_c = 1;
-    p.n = static_cast<int>(t.n); p.m = static_cast<int>(t.m);
-    p.r0 = static_cast<int>(b * t.T);
-    p.rows = static_cast<int>(t.n - b * t.T < t.T ? t.n - b * t.T : t.T);
-    p.mask = mask;
-    const long long blocks = (t.m + TRSM_CW - 1) / TRSM_CW;
-    CYC_CUDA(launch_pdl(trsm_diag_kernel, static_cast<unsigned>(blocks), TRSM_THREADS, TRSM_SMEM_BYTES, t.st, p));
-    g_launches.fetch_add(1);
-    return CYC_OK;
-}
-
-static int trsm_range(const TrsmPlan& t, long long b0, long long b1, unsigned mask, int level) {
-    if (b1 - b0 == 1) return trsm_diag(t, b0, mask);
-    const long long mid = b0 + (b1 - b0 + 1) / 2;
-    int rc = trsm_range(t, b0, mid, mask, level + 1);
-    if (rc) return rc;
-    const long long r0 = mid * t.T, r1 = b1 * t.T < t.n ? b1 * t.T : t.n, k0 = b0 * t.T, k1 = mid * t.T;
-    Problem q{1, r1 - r0, t.m, k1 - k0, CYC_F32, t.L + r0 * t.n + k0, t.X + k0 * t.m, t.W + level * t.plane + r0 * t.m,
-              (r1 - r0) * t.n, (k1 - k0) * t.m, (r1 - r0) * t.m, t.flags & CYC_FLAG_FIXED_K_ORDER, t.n};
-    rc = route(q, t.st);
-    if (rc) return rc;
-    return trsm_range(t, mid, b1, mask | (1u << level), level + 1);
-}
-
-// ------------------------------------------------------------------ FlashAttention-2 recurrence
-template <int D>
-static int launch_fa2(long long batch, long long N, long long M, const void* Q, const void* K, const void* V, float* O, cudaStream_t st) {
-    CUtensorMap tmQ, tmK, tmV;
-    int rc = make_map(&tmQ, CYC_BF16_F32, Q, D, N, batch, D, N * D, 64, FA2_BM);
-    if (rc) return rc;
-    rc = make_map(&tmK, CYC_BF16_F32, K, D, M, batch, D, M * D, 64, FA2_BN);
-    if (rc) return rc;
-    rc = make_map(&tmV, CYC_BF16_F32, V, D, M, batch, D, M * D, 64, FA2_BN);
-    if (rc) return rc;
-    Fa2Params p;
-    p.O = O;
-    p.N = static_cast<int>(N); p.M = static_cast<int>(M);
-    p.tiles_q = static_cast<int>((N + FA2_ROWS - 1) / FA2_ROWS);
-    p.scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
-    if (int rc_ = status_word(&p.status)) return rc_;
-    auto kern = fa2_kernel<D>;
-    {
-        // the kernel redistributes the registers it was launched with among its warps and counts on 128 per thread
-        static std::atomic<int> checked{0};
-        if (!checked.load()) {
-            cudaFuncAttributes fa;
-            CYC_CUDA(cudaFuncGetAttributes(&fa, kern));
-            if (fa.numRegs < FA2_REGS_LAUNCH) {
-                snprintf(g_err, sizeof g_err, "flash attention kernel compiled to %d registers per thread, %d expected", fa.numRegs, FA2_REGS_LAUNCH);
-                return CYC_ERR_CUDA;
-            }
-            checked.store(1);
-        }
-    }
-    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), Fa2Smem<D>::TOTAL)) return rc_;
-    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(batch * p.tiles_q), FA2_THREADS, Fa2Smem<D>::TOTAL, st, tmQ, tmK, tmV, p));
-    g_launches.fetch_add(1);
-    return CYC_OK;
-}
-
 }  // namespace cyc
 
-// ====================================================================== C ABI
 using namespace cyc;
 
 extern "C" int cyc_recurrence_matmul(int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B, void* C,
@@ -971,364 +667,6 @@ extern "C" int cyc_recurrence_matmul_splitk_static(int64_t M, int64_t N, int64_t
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return dtype == CYC_BF16_F32 ? launch_splitk<KIND_BF16>(q, st, di.sms, ws, plan) : launch_splitk<KIND_I8>(q, st, di.sms, ws, plan);
 }
-
-extern "C" int cyc_pool_reserved_bytes(int64_t* out) {
-    if (!out) return CYC_ERR_INVALID_ARG;
-    *out = 0;
-    cudaMemPool_t pool = nullptr;
-    int rc = workspace_pool(&pool, /*create=*/false);
-    if (rc) return rc;
-    if (pool) {
-        unsigned long long bytes = 0;
-        CYC_CUDA(cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReservedMemCurrent, &bytes));
-        *out = static_cast<int64_t>(bytes);
-    }
-    return CYC_OK;
-}
-
-extern "C" int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, const void* L, const void* B, void* X,
-                              void* stream, unsigned flags) {
-    if (n <= 0 || m <= 0 || tile < 0 || tile > TRSM_T_MAX || !L || !B || !X) return CYC_ERR_INVALID_ARG;
-    if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
-    if (flags & ~CYC_FLAG_FIXED_K_ORDER) return CYC_ERR_INVALID_ARG;
-    const uintptr_t l0 = reinterpret_cast<uintptr_t>(L), b0 = reinterpret_cast<uintptr_t>(B), x0 = reinterpret_cast<uintptr_t>(X);
-    if ((l0 | b0 | x0) % 4) return CYC_ERR_INVALID_ARG;
-    if (n > 0x7fffffffll || m > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
-    if (dtype != CYC_F32) return CYC_ERR_UNSUPPORTED;  // the solve is defined for fp32 only
-    const uintptr_t lbytes = static_cast<uintptr_t>(n) * n * 4, xbytes = static_cast<uintptr_t>(n) * m * 4;
-    if (x0 < l0 + lbytes && l0 < x0 + xbytes) return CYC_ERR_INVALID_ARG;                // X over L
-    if (x0 != b0 && x0 < b0 + xbytes && b0 < x0 + xbytes) return CYC_ERR_INVALID_ARG;    // X over B, other than in place
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    TrsmPlan t;
-    t.n = n; t.m = m; t.T = tile ? tile : TRSM_T_MAX;
-    t.L = static_cast<const float*>(L); t.B = static_cast<const float*>(B); t.X = static_cast<float*>(X);
-    t.W = nullptr; t.plane = n * m; t.flags = flags; t.st = st;
-    const long long nb = (n + t.T - 1) / t.T;
-    int levels = 0;
-    while ((1ll << levels) < nb) ++levels;
-    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel), TRSM_SMEM_BYTES)) return rc_;
-    if (levels) {
-        cudaMemPool_t pool;
-        int rc = workspace_pool(&pool);
-        if (rc) return rc;
-        void* ws = nullptr;
-        CYC_CUDA(cudaMallocFromPoolAsync(&ws, static_cast<size_t>(levels) * t.plane * sizeof(float), pool, st));
-        t.W = static_cast<float*>(ws);
-    }
-    int rc = trsm_range(t, 0, nb, 0u, 0);
-    if (t.W) {
-        cudaError_t e = cudaFreeAsync(t.W, st);
-        if (e != cudaSuccess && rc == CYC_OK) rc = cuda_fail(e, "cudaFreeAsync");
-    }
-    return rc;
-}
-
-extern "C" int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t d, int dtype, const void* Q, const void* K,
-                                   const void* V, void* O, void* stream, unsigned flags) {
-    if (batch <= 0 || N <= 0 || M <= 0 || d <= 0 || !Q || !K || !V || !O || flags != 0) return CYC_ERR_INVALID_ARG;
-    if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
-    const uintptr_t q0 = reinterpret_cast<uintptr_t>(Q), k0 = reinterpret_cast<uintptr_t>(K), v0 = reinterpret_cast<uintptr_t>(V),
-                    o0 = reinterpret_cast<uintptr_t>(O);
-    if ((q0 | k0 | v0) % 2 || o0 % 4) return CYC_ERR_INVALID_ARG;
-    const uintptr_t obytes = static_cast<uintptr_t>(batch) * N * d * 4, qbytes = static_cast<uintptr_t>(batch) * N * d * 2,
-                    kbytes = static_cast<uintptr_t>(batch) * M * d * 2;
-    if ((o0 < q0 + qbytes && q0 < o0 + obytes) || (o0 < k0 + kbytes && k0 < o0 + obytes) || (o0 < v0 + kbytes && v0 < o0 + obytes))
-        return CYC_ERR_INVALID_ARG;  // O over an input
-    if (dtype != CYC_BF16_F32 || (d != 64 && d != 128)) {
-        snprintf(g_err, sizeof g_err, "flash attention: bf16 inputs with head dimension 64 or 128 only");
-        return CYC_ERR_UNSUPPORTED;
-    }
-    if ((q0 | k0 | v0 | o0) % 16) {
-        snprintf(g_err, sizeof g_err, "flash attention: Q, K, V and O must be 16-byte aligned");
-        return CYC_ERR_UNSUPPORTED;
-    }
-    const long long tiles_q = (N + FA2_ROWS - 1) / FA2_ROWS;
-    if (N > 0x7fffffffll || M > 0x7fffffffll || batch * tiles_q > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
-    DeviceInfo di;
-    int rc = device_info(&di);
-    if (rc) return rc;
-    if (di.cc_major != 10) {
-        snprintf(g_err, sizeof g_err, "tensor-core kernels need an sm_100 device");
-        return CYC_ERR_UNSUPPORTED;
-    }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return d == 64 ? launch_fa2<64>(batch, N, M, Q, K, V, static_cast<float*>(O), st)
-                   : launch_fa2<128>(batch, N, M, Q, K, V, static_cast<float*>(O), st);
-}
-
-// tile of SUBS * 4096 elements: 16384 for long rows (the running value of one chain advances by at most 32 tiles per
-// descriptor round trip), 8192 when a row has at most 32 such tiles (its look-back never leaves one window; half the
-// shared memory per CTA, twice the CTAs per SM)
-static int scan_subs(long long n) { return (n + SCAN_SUBS_SHORT * SCAN_SUB - 1) / (SCAN_SUBS_SHORT * SCAN_SUB) <= SCAN_WINDOW ? SCAN_SUBS_SHORT : SCAN_SUBS; }
-
-template <typename T, int SUBS>
-static int launch_scan(long long rows, long long n, const void* A, long long sA, void* P, long long sP, cudaStream_t st) {
-    constexpr long long TILE = static_cast<long long>(SUBS) * SCAN_SUB;
-    ScanParams<T> p;
-    p.A = static_cast<const T*>(A);
-    p.P = static_cast<T*>(P);
-    p.n = n; p.strideA = sA; p.strideP = sP;
-    p.tiles_per_row = (n + TILE - 1) / TILE;
-    const long long tiles = rows * p.tiles_per_row;
-    p.total_tiles = tiles;
-    p.vec_ok = (reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(P) % 16 == 0 && (rows == 1 || (sA % 4 == 0 && sP % 4 == 0)))
-                   ? 1 : 0;
-    if (int rc_ = status_word(&p.status)) return rc_;
-    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(scan_kernel<T, SUBS>), static_cast<int>(TILE * sizeof(T)) + 128)) return rc_;
-    cudaMemPool_t pool;
-    int rc = workspace_pool(&pool);
-    if (rc) return rc;
-    void* ws = nullptr;
-    const size_t bytes = sizeof(ScanHeader) + static_cast<size_t>(tiles) * sizeof(unsigned long long);
-    CYC_CUDA(cudaMallocFromPoolAsync(&ws, bytes, pool, st));
-    p.header = static_cast<ScanHeader*>(ws);
-    p.desc = reinterpret_cast<unsigned long long*>(static_cast<unsigned char*>(ws) + sizeof(ScanHeader));
-    cudaError_t e = cudaMemsetAsync(ws, 0, bytes, st);  // counter, abort flag and every descriptor start at zero
-    if (e == cudaSuccess) {
-        // short rows need only their own quarters of the staging buffer: more CTAs fit an SM
-        const int quarters = static_cast<int>(std::min<long long>(SUBS, (n + SCAN_SUB - 1) / SCAN_SUB));
-        scan_kernel<T, SUBS><<<static_cast<unsigned>(tiles), SCAN_THREADS, quarters * SCAN_SUB * sizeof(T) + 128, st>>>(p);
-        e = cudaGetLastError();
-        if (e == cudaSuccess) g_launches.fetch_add(1);
-    }
-    const cudaError_t e2 = cudaFreeAsync(ws, st);
-    if (e != cudaSuccess) return cuda_fail(e, "scan_kernel");
-    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaFreeAsync");
-    return CYC_OK;
-}
-
-extern "C" int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A, int64_t strideA, void* P, int64_t strideP,
-                              void* stream, unsigned flags) {
-    if (rows <= 0 || n <= 0 || !A || !P || flags != 0 || strideA < 0 || strideP < 0) return CYC_ERR_INVALID_ARG;
-    if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32 && dtype != CYC_I32) return CYC_ERR_INVALID_ARG;
-    const long long sA = strideA ? strideA : n, sP = strideP ? strideP : n;
-    if (sA < n || sP < n) return CYC_ERR_INVALID_ARG;
-    const uintptr_t a0 = reinterpret_cast<uintptr_t>(A), p0 = reinterpret_cast<uintptr_t>(P);
-    if ((a0 | p0) % 4) return CYC_ERR_INVALID_ARG;
-    if (rows > (1ll << 40) || n > (1ll << 40)) return CYC_ERR_UNSUPPORTED;
-    const uintptr_t abytes = (static_cast<uintptr_t>(rows - 1) * sA + n) * 4, pbytes = (static_cast<uintptr_t>(rows - 1) * sP + n) * 4;
-    const bool in_place = a0 == p0 && sA == sP;
-    if (!in_place && a0 < p0 + pbytes && p0 < a0 + abytes) return CYC_ERR_INVALID_ARG;
-    if (dtype != CYC_F32 && dtype != CYC_I32) {
-        snprintf(g_err, sizeof g_err, "prefix sum: fp32 or int32 only");
-        return CYC_ERR_UNSUPPORTED;
-    }
-    const int subs = scan_subs(n);
-    const long long tiles_per_row = (n + subs * SCAN_SUB - 1) / (subs * SCAN_SUB);
-    if (tiles_per_row > 0x7fffffffll / rows) return CYC_ERR_UNSUPPORTED;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (subs == SCAN_SUBS_SHORT)
-        return dtype == CYC_F32 ? launch_scan<float, SCAN_SUBS_SHORT>(rows, n, A, sA, P, sP, st) : launch_scan<int, SCAN_SUBS_SHORT>(rows, n, A, sA, P, sP, st);
-    return dtype == CYC_F32 ? launch_scan<float, SCAN_SUBS>(rows, n, A, sA, P, sP, st) : launch_scan<int, SCAN_SUBS>(rows, n, A, sA, P, sP, st);
-}
-
-// ------------------------------------------------------------------ tiled Cholesky
-// Panel j (columns c0 .. c1 of L), left-looking.  The sums over the panels already factored,
-//     W = L[c0:n, 0:c0] L[c0:c1, 0:c0]^T ,
-// are recurrence-matmul launches (k cut into slices that run as the batch dimension, then summed in increasing k); the
-// diagonal tile A_jj - W is factored by chol_diag_kernel (one SM); the tiles below are the rows of
-// X L_jj^T = A[c1:n, c0:c1] - W, solved by trsm_diag_kernel with the right-hand sides addressed as rows.
-// The paper describes the recurrence as a wavefront that widens down the column; on a GPU the narrow end of that
-// wavefront is the one-SM diagonal tile, so the work is laid on two streams:
-//   the caller's stream carries the chain  sum of the diagonal tile -> diagonal tile (j) -> solve of the block row just
-//   below it -> sum of the next diagonal tile -> diagonal tile (j+1) ...,
-//   a helper stream carries the bulk: solve of the remaining rows of panel j, then the sums of everything below the
-//   next diagonal tile -- which run while diagonal tile j+1 is being factored.
-// Events order the two; every launch below names the data it needs.
-struct CholAux {
-    bool ready = false;
-    cudaStream_t side = nullptr;
-    std::vector<cudaEvent_t> events;
-    std::mutex mu;  // one factorisation at a time per device uses the helper stream
-};
-static int chol_aux(CholAux** out, size_t events) {
-    static std::mutex mu;
-    static CholAux aux[64];
-    int dev = 0;
-    CYC_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return CYC_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lk(mu);
-    CholAux& a = aux[dev];
-    if (!a.ready) {
-        CYC_CUDA(cudaStreamCreateWithFlags(&a.side, cudaStreamNonBlocking));
-        a.ready = true;
-    }
-    while (a.events.size() < events) {
-        cudaEvent_t e = nullptr;
-        CYC_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-        a.events.push_back(e);
-    }
-    *out = &a;
-    return CYC_OK;
-}
-
-// W (plane 0) = L[r0:r1, 0:c0] L[c0:c0+w, 0:c0]^T on stream `s`; planes of `pstride` floats starting at W.  The k range
-// is cut into up to CHOL_MAX_SLICES equal slices (one batched launch: few 256-row tiles, and the slices give every CTA
-// pair work) plus one launch for the remainder; the slices' partial sums are then added in increasing k into plane 0.
-constexpr int CHOL_MAX_SLICES = 8;        // sums below a diagonal tile: several 256-row tiles share the CTA pairs
-constexpr int CHOL_MAX_SLICES_DIAG = 64;  // sum of a diagonal tile: one tile, so every panel of k can be a slice of its own
-static int chol_product(cudaStream_t s, float* Lf, long long n, long long T, long long c0, long long w, long long r0, long long r1, float* W,
-                        long long pstride, unsigned flags, int max_slices) {
-    const long long rows = r1 - r0;
-    const long long kblocks = c0 / T, tiles_m = (rows + 255) / 256;
-    const long long smax = std::min<long long>({static_cast<long long>(max_slices), kblocks, std::max<long long>(1, kCtaPairs / tiles_m)});
-    // slices of ceil(kblocks / smax) panels, so that the remainder (one more launch) is shorter than a slice
-    const long long per = (kblocks + smax - 1) / smax, S = kblocks / per;
-    const long long kc = per * T, rem = c0 - S * kc;
-    const unsigned gflags = (flags & CYC_FLAG_FIXED_K_ORDER) | CYC_FLAG_B_COL_MAJOR;
-    Problem q{S, rows, w, kc, CYC_F32, Lf + r0 * n, Lf + c0 * n, W, kc, kc, pstride, gflags, n, n};
-    int rc = route(q, s);
-    if (rc) return rc;
-    int planes = static_cast<int>(S);
-    if (rem > 0) {
-        Problem r{1, rows, w, rem, CYC_F32, Lf + r0 * n + S * kc, Lf + c0 * n + S * kc, W + S * pstride, rows * n, w * n, pstride, gflags, n, n};
-        rc = route(r, s);
-        if (rc) return rc;
-        ++planes;
-    }
-    if (planes > 1) {
-        DeviceInfo di;
-        rc = device_info(&di);
-        if (rc) return rc;
-        const long long work = pstride / 4;
-        const long long blocks = std::min<long long>((work + 127) / 128, 16ll * di.sms);
-        cudaError_t e = launch_pdl(splitk_reduce_kernel<float>, static_cast<unsigned>(blocks), 128, 0, s, static_cast<const float*>(W), W, pstride,
-                                   pstride, planes, 1ll, 1);
-        if (e != cudaSuccess) return cuda_fail(e, "splitk_reduce_kernel");
-        g_launches.fetch_add(1);
-    }
-    return CYC_OK;
-}
-
-extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, void* L, void* stream, unsigned flags) {
-    if (n <= 0 || tile < 0 || tile > CHOL_T_MAX || !A || !L) return CYC_ERR_INVALID_ARG;
-    if (dtype != CYC_F32 && dtype != CYC_BF16_F32 && dtype != CYC_I8_I32) return CYC_ERR_INVALID_ARG;
-    if (flags & ~CYC_FLAG_FIXED_K_ORDER) return CYC_ERR_INVALID_ARG;
-    const uintptr_t a0 = reinterpret_cast<uintptr_t>(A), l0 = reinterpret_cast<uintptr_t>(L);
-    if ((a0 | l0) % 4) return CYC_ERR_INVALID_ARG;
-    if (n > 0x7fffffffll) return CYC_ERR_UNSUPPORTED;
-    if (dtype != CYC_F32) return CYC_ERR_UNSUPPORTED;  // the factorisation is defined for fp32 only
-    const uintptr_t bytes = static_cast<uintptr_t>(n) * n * 4;
-    if (a0 != l0 && a0 < l0 + bytes && l0 < a0 + bytes) return CYC_ERR_INVALID_ARG;  // overlap other than in place
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const float* Af = static_cast<const float*>(A);
-    float* Lf = static_cast<float*>(L);
-    const long long T = tile ? tile : CHOL_T_MAX;
-    const bool in_place = a0 == l0;
-    const long long panels = (n + T - 1) / T;
-    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(chol_diag_kernel), CHOL_SMEM_BYTES)) return rc_;
-    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel), TRSM_SMEM_BYTES)) return rc_;
-    CholAux* aux = nullptr;
-    if (int rc_ = chol_aux(&aux, static_cast<size_t>(3 * panels + 2))) return rc_;
-    std::lock_guard<std::mutex> aux_lock(aux->mu);
-    cudaStream_t side = aux->side;
-    auto ev = [&](long long j, int which) { return aux->events[static_cast<size_t>(3 * j + which)]; };  // 0: D(j), 1: near solve (j), 2: sums below (j)
-    cudaEvent_t ev_fork = aux->events[static_cast<size_t>(3 * panels)], ev_join = aux->events[static_cast<size_t>(3 * panels + 1)];
-
-    // workspace: planes of the diagonal tile's sums and planes of the sums below it (the two streams never share a plane)
-    const long long pd = (T * T + 3) / 4 * 4, pb = ((n - T) * T + 3) / 4 * 4;
-    float* Wd = nullptr;
-    float* Wb = nullptr;
-    if (n > T) {
-        cudaMemPool_t pool;
-        int rc = workspace_pool(&pool);
-        if (rc) return rc;
-        void* ws = nullptr;
-        CYC_CUDA(cudaMallocFromPoolAsync(&ws, (static_cast<size_t>(CHOL_MAX_SLICES_DIAG + 1) * pd + static_cast<size_t>(CHOL_MAX_SLICES + 1) * pb) * sizeof(float), pool, st));
-        Wd = static_cast<float*>(ws);
-        Wb = Wd + (CHOL_MAX_SLICES_DIAG + 1) * pd;
-    }
-    int rc = CYC_OK;
-    auto ok = [&](cudaError_t e, const char* what) {
-        if (e != cudaSuccess && rc == CYC_OK) rc = cuda_fail(e, what);
-        return rc == CYC_OK;
-    };
-    // rows [r0, r1) of panel (c0, w): X L_jj^T = A - W, the right-hand sides addressed as rows
-    auto solve_rows = [&](cudaStream_t s, long long c0, long long w, long long c1, long long r0, long long r1, bool have_w, long long pstride) {
-        TrsmDiagParams p;
-        p.L = Lf;
-        p.B = Af + r0 * n + c0; p.X = Lf + r0 * n + c0; p.W = have_w ? Wb + (r0 - c1) * w : nullptr;
-        p.plane = pstride;
-        p.b_r = 1; p.b_c = n; p.x_r = 1; p.x_c = n; p.w_r = 1; p.w_c = w;
-        p.n = static_cast<int>(n); p.m = static_cast<int>(r1 - r0);
-        p.r0 = static_cast<int>(c0); p.rows = static_cast<int>(w);
-        p.mask = have_w ? 1u : 0u;
-        if (ok(launch_pdl(trsm_diag_kernel, static_cast<unsigned>((r1 - r0 + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, s, p), "trsm_diag_kernel"))
-            g_launches.fetch_add(1);
-    };
-
-    ok(cudaEventRecord(ev_fork, st), "cudaEventRecord");
-    ok(cudaStreamWaitEvent(side, ev_fork, 0), "cudaStreamWaitEvent");
-    for (long long j = 0; j < panels && rc == CYC_OK; ++j) {
-        const long long c0 = j * T, c1 = std::min<long long>(n, c0 + T), w = c1 - c0, c2 = std::min<long long>(n, c1 + T);
-        // ---- caller's stream: the sum of the diagonal tile (needs row block j of every earlier panel: the near solve of
-        // ---- panel j-1 is on this stream, the far solves of older panels were waited for with the sums below panel j-1)
-        if (c0 > 0) {
-            rc = chol_product(st, Lf, n, T, c0, w, c0, c1, Wd, pd, flags, CHOL_MAX_SLICES_DIAG);
-            if (rc) break;
-        }
-        CholDiagParams d;
-        d.A = Af + c0 * n + c0; d.W = Wd; d.L = Lf + c0 * n + c0;
-        d.plane = pd; d.planes = c0 > 0 ? 1 : 0;
-        d.lda = n; d.ldw = w; d.ldl = n;
-        d.rows = static_cast<int>(w);
-        d.zero_upper = in_place ? 0 : 1;
-        if (!ok(launch_pdl(chol_diag_kernel, 1u, CHOL_THREADS, CHOL_SMEM_BYTES, st, d), "chol_diag_kernel")) break;
-        g_launches.fetch_add(1);
-        if (c1 >= n) break;
-        ok(cudaEventRecord(ev(j, 0), st), "cudaEventRecord");
-        const long long pstride_b = ((n - c1) * w + 3) / 4 * 4;
-        // ---- caller's stream: the block row just below the diagonal tile (needs its sums, formed on the helper stream)
-        if (c0 > 0) ok(cudaStreamWaitEvent(st, ev(j, 2), 0), "cudaStreamWaitEvent");
-        if (rc == CYC_OK) solve_rows(st, c0, w, c1, c1, c2, c0 > 0, pstride_b);
-        ok(cudaEventRecord(ev(j, 1), st), "cudaEventRecord");
-        // ---- helper stream: the remaining rows of the panel (need the diagonal tile; their sums are on this stream)
-        ok(cudaStreamWaitEvent(side, ev(j, 0), 0), "cudaStreamWaitEvent");
-        if (c2 < n && rc == CYC_OK) solve_rows(side, c0, w, c1, c2, n, c0 > 0, pstride_b);
-        if (!in_place)  // zeros above the diagonal: the block row to the right of the diagonal tile
-            ok(cudaMemset2DAsync(Lf + c0 * n + c1, static_cast<size_t>(n) * 4, 0, static_cast<size_t>(n - c1) * 4, static_cast<size_t>(w), side), "cudaMemset2DAsync");
-        // ---- helper stream: the sums below the NEXT diagonal tile (need block row j+1 of this panel: the near solve)
-        if (c2 < n && rc == CYC_OK) {
-            const long long w1 = c2 - c1, pstride_n = ((n - c2) * w1 + 3) / 4 * 4;
-            ok(cudaStreamWaitEvent(side, ev(j, 1), 0), "cudaStreamWaitEvent");
-            if (rc == CYC_OK) rc = chol_product(side, Lf, n, T, c1, w1, c2, n, Wb, pstride_n, flags, CHOL_MAX_SLICES);
-            ok(cudaEventRecord(ev(j + 1, 2), side), "cudaEventRecord");
-        }
-    }
-    // the caller's stream continues only after the helper stream has finished
-    if (cudaEventRecord(ev_join, side) == cudaSuccess) cudaStreamWaitEvent(st, ev_join, 0);
-    else cudaStreamSynchronize(side);
-    if (Wd) {
-        cudaError_t e = cudaFreeAsync(Wd, st);
-        if (e != cudaSuccess && rc == CYC_OK) rc = cuda_fail(e, "cudaFreeAsync");
-    }
-    return rc;
-}
-
-extern "C" int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles) {
-    if (budget_cycles < 1 || budget_cycles > (1ll << 24)) return CYC_ERR_INVALID_ARG;  // at most ~10 ms
-    int* status = nullptr;
-    CYC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_device_status));
-    bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(budget_cycles, status);
-    CYC_CUDA(cudaGetLastError());
-    g_launches.fetch_add(1);
-    return CYC_OK;
-}
-
-extern "C" int cyc_last_device_status(void* stream, int* out) {
-    CYC_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
-    int word = 0;
-    CYC_CUDA(cudaMemcpyFromSymbol(&word, g_device_status, sizeof word));
-    if (word != 0) {
-        const int zero = 0;
-        tail_scratch_mark_dirty();  // a kernel that gave up may have left strip counters of the sliced tail non-zero
-        CYC_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero));
-        snprintf(g_err, sizeof g_err, "device wait ran out (code 0x%x)", word);
-    }
-    if (out) *out = word != 0 ? CYC_ERR_TIMEOUT : CYC_OK;
-    return CYC_OK;
-}
-
 extern "C" const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
                                       const void* C, unsigned flags) {
     if (batch <= 0 || M <= 0 || N <= 0 || K <= 0) return nullptr;
@@ -1357,18 +695,3 @@ extern "C" const char* cyc_schedule_for(int64_t batch, int64_t M, int64_t N, int
     }
     return "output_stationary";
 }
-
-extern "C" int64_t cyc_launch_count(void) { return g_launches.load(); }
-extern "C" const char* cyc_last_cuda_error(void) { return g_err; }
-
-extern "C" const char* cyc_status_string(int s) {
-    switch (s) {
-        case CYC_OK: return "ok";
-        case CYC_ERR_INVALID_ARG: return "invalid argument";
-        case CYC_ERR_UNSUPPORTED: return "unsupported";
-        case CYC_ERR_CUDA: return "CUDA error";
-        case CYC_ERR_TIMEOUT: return "device wait timed out";
-        default: return "unknown status";
-    }
-}
-extern "C" int cyc_version(void) { return 100; }
