@@ -203,7 +203,7 @@ struct TailScratch {
     bool dirty = false;
 };
 constexpr int kTailScratchMax = 8;
-constexpr size_t kTailCounterBytes = static_cast<size_t>(kCtaPairs) * 8 * sizeof(int);
+constexpr size_t kTailCounterBytes = static_cast<size_t>(kCtaPairs) * PAIR_STRIPS * sizeof(int);
 static std::mutex g_tail_mu;
 static TailScratch g_tail_scratch[64];
 static int g_tail_scratch_count = 0;
@@ -259,7 +259,7 @@ static int tail_scratch_for(cudaStream_t st, TailScratch** out) {
 // `ws` != nullptr: split-K -- the kernel writes plan.S planes of partial sums per problem into ws
 template <int KIND, bool B_MN>
 static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws = nullptr, SplitPlan plan = SplitPlan()) {
-    constexpr int STAGES = 6;
+    constexpr int STAGES = PAIR_STAGES;
     constexpr int BK = 128 / UmmaTraits<KIND>::ELEM_BYTES;
     constexpr int CH = 128 / UmmaTraits<KIND>::ELEM_BYTES;
     constexpr int SMEM = pair_smem_bytes<STAGES>();
@@ -306,7 +306,7 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws 
             }
         }
     }
-    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(2 * pairs), UMMA_THREADS, SMEM, st, tmA, tmB, tmC, p));
+    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(2 * pairs), PAIR_THREADS, SMEM, st, tmA, tmB, tmC, p));
     g_launches.fetch_add(1);
     return CYC_OK;
 }

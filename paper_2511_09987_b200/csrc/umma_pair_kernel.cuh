@@ -96,25 +96,39 @@ constexpr int PAIR_HALF = 128;      // B columns (and A rows) held by one CTA
 constexpr int PAIR_STAGE_A = 128 * 128;
 constexpr int PAIR_STAGE_B = 128 * 128;
 constexpr int PAIR_STAGE_BYTES = PAIR_STAGE_A + PAIR_STAGE_B;
-constexpr int PAIR_STAGING_BYTES = 4 * 2 * 4096;  // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
-constexpr int PAIR_STRIP_BYTES = 32 * 256 * 4;     // partial sums of one 32-row strip of a 256 x 256 tile
-constexpr int PAIR_TILE_BYTES = 8 * PAIR_STRIP_BYTES;
+#ifndef CYC_PAIR_EPI_WARPS
+#define CYC_PAIR_EPI_WARPS 4
+#endif
+// Epilogue warps per CTA: four (one per tensor-memory lane quarter, 256 columns each) or eight (two per quarter, 128
+// columns each; the ring then has five stages instead of six, so that 64 KB of export staging fit).  Measured: eight
+// warps change nothing on the batched 256^3 problems (94.9 against 95.0-95.4 us: the export is not what bounds them) and
+// cost 4 % on int8 4096^3 (the sixth stage matters there), so four it is.
+constexpr int PAIR_EPI_WARPS = CYC_PAIR_EPI_WARPS;
+constexpr int PAIR_EPI_COLS = PAIR_BN * 4 / PAIR_EPI_WARPS;     // columns of a tile one epilogue warp exports
+constexpr int PAIR_THREADS = 64 + 32 * PAIR_EPI_WARPS;          // producer, MMA issuer, epilogue warps
+constexpr int PAIR_STAGES = PAIR_EPI_WARPS == 8 ? 5 : 6;
+constexpr int PAIR_STAGING_BYTES = PAIR_EPI_WARPS * 2 * 4096;   // per epilogue warp 2 buffers of 32 rows x 128 B
+constexpr int PAIR_STAGING_BYTES_4 = 4 * 2 * 4096;              // the kernels with four epilogue warps
+constexpr int PAIR_STRIPS = 2 * PAIR_EPI_WARPS;                 // strips of a tile: one per epilogue warp of the pair
+constexpr int PAIR_STRIP_BYTES = 32 * PAIR_EPI_COLS * 4;        // partial sums of one strip (32 rows x the warp's columns)
+constexpr int PAIR_TILE_BYTES = PAIR_STRIPS * PAIR_STRIP_BYTES; // = 256 KB
 
-// k-slice of a tail tile, seen from the warp that owns 32-row strip `strip` (0..7 over the pair) of the tile: park
+// k-slice of a tail tile, seen from the epilogue warp that owns strip `strip` of the tile (32 rows x `nchunks` pieces of 32
+// columns starting at column `col0`): park
 // the strip's partial sums (16-byte piece g of a lane's 32 values at (g * 32 + lane) * 16, so that one store instruction
 // writes 512 contiguous bytes), give the accumulator at `acc_taddr` back, and find out whether the other slices of the
 // strip are already there.  If so, C_ij = the slices' sums added in increasing k (the slice at hand is read back like
 // the others; the read of the next piece is in flight while this one is added), handed piece by piece to
-// `export_piece(values, first column within the tile)`.
+// `export_piece(values, first column within the tile)`.  (`ptx::mbar_arrive_remote` gives the accumulator back.)
 template <typename Out, typename ExportFn>
-__device__ __forceinline__ void pair_tail_strip(const PairParams& p, const PairWork& w, int strip, uint32_t acc_taddr, int nchunks, int lane,
+__device__ __forceinline__ void pair_tail_strip(const PairParams& p, const PairWork& w, int strip, uint32_t acc_taddr, int col0, int nchunks, int lane,
                                                 uint64_t* acc_empty, ExportFn&& export_piece) {
     uint8_t* tile_ws = static_cast<uint8_t*>(p.tail_ws) + static_cast<size_t>(w.tail_index) * p.tail_S * PAIR_TILE_BYTES;
     uint8_t* mine = tile_ws + static_cast<size_t>(w.slice) * PAIR_TILE_BYTES + strip * PAIR_STRIP_BYTES;
 #pragma unroll 1
     for (int c = 0; c < nchunks; ++c) {
         uint32_t v[32];
-        ptx::tmem_ld_32x32(acc_taddr + static_cast<uint32_t>(c * 32), v);
+        ptx::tmem_ld_32x32(acc_taddr + static_cast<uint32_t>(col0 + c * 32), v);
         ptx::tmem_ld_wait();
         uint4* dst = reinterpret_cast<uint4*>(mine + c * 4096);
 #pragma unroll
@@ -126,12 +140,12 @@ __device__ __forceinline__ void pair_tail_strip(const PairParams& p, const PairW
     int arrived = 0;
     if (lane == 0) {
         ptx::mbar_arrive_remote(acc_empty, 0);
-        arrived = atomicAdd(&p.tail_counters[w.tail_index * 8 + strip], 1);
+        arrived = atomicAdd(&p.tail_counters[w.tail_index * PAIR_STRIPS + strip], 1);
     }
     arrived = __shfl_sync(0xffffffffu, arrived, 0);
     if (arrived != p.tail_S - 1) return;  // a later warp finishes this strip
     __threadfence();
-    if (lane == 0) p.tail_counters[w.tail_index * 8 + strip] = 0;  // zero again for the next launch
+    if (lane == 0) p.tail_counters[w.tail_index * PAIR_STRIPS + strip] = 0;  // zero again for the next launch
     const uint8_t* strip_ws = tile_ws + strip * PAIR_STRIP_BYTES;
     const int pieces = nchunks * p.tail_S;
     auto fetch = [&](int i, uint32_t (&o)[32]) {
@@ -143,6 +157,7 @@ __device__ __forceinline__ void pair_tail_strip(const PairParams& p, const PairW
             o[4 * g] = x.x; o[4 * g + 1] = x.y; o[4 * g + 2] = x.z; o[4 * g + 3] = x.w;
         }
     };
+    if (pieces == 0) return;  // this warp's columns lie outside C
     uint32_t cur[32], nxt[32], sum[32] = {};
     fetch(0, cur);
 #pragma unroll 1
@@ -157,7 +172,7 @@ __device__ __forceinline__ void pair_tail_strip(const PairParams& p, const PairW
             y = sl == 0 ? x : y + x;
             memcpy(&sum[g], &y, 4);
         }
-        if (sl == p.tail_S - 1) export_piece(sum, c * 32);
+        if (sl == p.tail_S - 1) export_piece(sum, col0 + c * 32);
 #pragma unroll
         for (int g = 0; g < 32; ++g) cur[g] = nxt[g];
     }
@@ -167,7 +182,7 @@ template <int STAGES>
 constexpr int pair_smem_bytes() { return STAGES * PAIR_STAGE_BYTES + PAIR_STAGING_BYTES + 1024 + 1024; }
 
 template <int KIND, bool B_MN, int STAGES>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(UMMA_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PAIR_THREADS, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmC, const PairParams p) {
     using Tr = UmmaTraits<KIND>;
@@ -199,7 +214,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(&ctl->acc_full[a], 1);
-            ptx::mbar_init(&ctl->acc_empty[a], 8);
+            ptx::mbar_init(&ctl->acc_empty[a], 2 * PAIR_EPI_WARPS);
         }
         ctl->abort = 0;
         ptx::fence_mbar_init();
@@ -308,8 +323,10 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         __syncwarp();
     } else {
         // ------------------------------------------------------------ epilogue: C_ij <- [i,k_end]_C (both CTAs)
-        const int q = warp & 3;
-        uint8_t* my_stage = staging + q * 8192;
+        const int q = warp & 3;                                  // tensor-memory lane quarter this warp may read
+        const int ew = warp - 2;                                 // epilogue warp 0 .. PAIR_EPI_WARPS - 1
+        const int col_first = (ew >> 2) * PAIR_EPI_COLS;         // its columns of the tile: [col_first, col_first + PAIR_EPI_COLS)
+        uint8_t* my_stage = staging + ew * 8192;
         const uint32_t lane_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
         int local = 0, sbuf = 0;
         bool ok = true;
@@ -324,7 +341,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const int row0 = tm * 256 + static_cast<int>(rank) * PAIR_HALF + q * 32;
             const int row = row0 + lane;
             Out* crow = static_cast<Out*>(p.C) + static_cast<long long>(b) * p.sC + static_cast<long long>(row) * p.N;
-            const int nchunks = min(PAIR_BN / 32, (p.N - tn * PAIR_BN + 31) / 32);  // 32-column pieces inside C
+            // 32-column pieces of this warp's columns that lie inside C
+            const int nchunks = max(0, min(PAIR_EPI_COLS / 32, (p.N - tn * PAIR_BN - col_first + 31) / 32));
             // one 32 x 32 piece of C (this lane's row, 32 consecutive columns starting at c0) leaves the SM
             auto export_piece = [&](const uint32_t (&v)[32], int c0) {
                 const int col = tn * PAIR_BN + c0;
@@ -352,16 +370,17 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (w.slice < 0) {
                 // whole tile: the tensor-memory read of the next piece is in flight while this one is staged and stored
                 uint32_t va[32], vb[32];
-                ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN), va);
+                const uint32_t acc = lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + col_first);
+                if (nchunks > 0) ptx::tmem_ld_32x32(acc, va);
 #pragma unroll 1
                 for (int c = 0; c < nchunks; c += 2) {
                     ptx::tmem_ld_wait();
-                    if (c + 1 < nchunks) ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + (c + 1) * 32), vb);
-                    export_piece(va, c * 32);
+                    if (c + 1 < nchunks) ptx::tmem_ld_32x32(acc + static_cast<uint32_t>((c + 1) * 32), vb);
+                    export_piece(va, col_first + c * 32);
                     if (c + 1 < nchunks) {
                         ptx::tmem_ld_wait();
-                        if (c + 2 < nchunks) ptx::tmem_ld_32x32(lane_taddr + static_cast<uint32_t>(ab * PAIR_BN + (c + 2) * 32), va);
-                        export_piece(vb, (c + 1) * 32);
+                        if (c + 2 < nchunks) ptx::tmem_ld_32x32(acc + static_cast<uint32_t>((c + 2) * 32), va);
+                        export_piece(vb, col_first + (c + 1) * 32);
                     }
                 }
                 ptx::tc_fence_before();
@@ -370,8 +389,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 continue;
             }
             // k-slice of a tail tile
-            pair_tail_strip<Out>(p, w, static_cast<int>(rank) * 4 + q, lane_taddr + static_cast<uint32_t>(ab * PAIR_BN), nchunks, lane,
-                                 &ctl->acc_empty[ab], export_piece);
+            pair_tail_strip<Out>(p, w, static_cast<int>(rank) * PAIR_EPI_WARPS + ew, lane_taddr + static_cast<uint32_t>(ab * PAIR_BN), col_first, nchunks,
+                                 lane, &ctl->acc_empty[ab], export_piece);
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
         __syncwarp();

@@ -42,7 +42,7 @@ constexpr int X3_STAGE_HI = 2 * 128 * X3_BK * 4;
 constexpr int X3_STAGE_BYTES = 2 * X3_STAGE_HI;  // hi parts followed by lo parts
 constexpr int X3_STAGES = 96 / X3_BK;
 constexpr int X3_PREFETCH = 256 / X3_BK;  // k-blocks of A requested from L2 ahead of the ring
-constexpr int X3_SMEM_BYTES = X3_STAGES * X3_STAGE_BYTES + PAIR_STAGING_BYTES + 1024 + 1024;
+constexpr int X3_SMEM_BYTES = X3_STAGES * X3_STAGE_BYTES + PAIR_STAGING_BYTES_4 + 1024 + 1024;
 
 struct X3Ctl {
     uint64_t full[8];
@@ -86,7 +86,7 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* staging = smem + STAGES * X3_STAGE_BYTES;
-    X3Ctl* ctl = reinterpret_cast<X3Ctl*>(staging + PAIR_STAGING_BYTES);
+    X3Ctl* ctl = reinterpret_cast<X3Ctl*>(staging + PAIR_STAGING_BYTES_4);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
