@@ -19,6 +19,11 @@
  * function returns without synchronising.  The functions never throw, never
  * abort and are safe to call from several host threads.
  *
+ * Environment.  CYC_LOG=1 (read once per process): one line on stderr for every
+ * kernel selection of the matrix-multiply recurrence -- shape, dtype, flags,
+ * pitches and the kernel chosen (the names of cyc_kernel_for) -- including the
+ * tile products that the triangular solve and the Cholesky factorisation lay on it.
+ *
  * Layouts.  A is [M][K] row-major (K contiguous).  B is [K][N] row-major, or,
  * with CYC_FLAG_B_COL_MAJOR, stored as [N][K] (element B_kj at B[j*K + k]).
  * C is [M][N] row-major and is written completely (the recurrence starts from

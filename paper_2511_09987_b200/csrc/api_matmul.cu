@@ -1,5 +1,7 @@
 // The matrix-multiply recurrence: kernel selection, tensor-map construction, launches, and the entry points
 // cyc_recurrence_matmul, _batched, _host, _splitk_static, cyc_kernel_for and cyc_schedule_for.  See include/cyc.h.
+#include <cstdlib>
+
 #include "api_internal.h"
 #include "simt_kernel.cuh"
 #include "umma_kernel.cuh"
@@ -448,7 +450,30 @@ static int launch_umma(const Problem& q, cudaStream_t st) {
 }
 
 // kernel selection and launch for a validated problem (also used for the sub-problems the library builds itself)
+static const char* family_name(Family f) {
+    switch (f) {
+        case FAM_UMMA: return "tcgen05";
+        case FAM_UMMA_PAIR: return "tcgen05_pair";
+        case FAM_UMMA_TALL: return "tcgen05_pair_tall";
+        case FAM_UMMA_SPLITK: return "tcgen05_pair_splitk";
+        case FAM_UMMA_3XTF32: return "tcgen05_3xtf32";
+        default: return "simt";
+    }
+}
+
+// CYC_LOG=1 in the environment: one line on stderr per kernel selection (read once per process)
+static bool log_enabled() {
+    static const bool on = [] {
+        const char* v = getenv("CYC_LOG");
+        return v && *v && *v != '0';
+    }();
+    return on;
+}
+
 int route(const Problem& q, cudaStream_t st) {
+    if (log_enabled())
+        fprintf(stderr, "cyc: batch=%lld M=%lld N=%lld K=%lld dtype=%d flags=0x%x lda=%lld ldb=%lld -> %s\n", q.batch, q.M, q.N, q.K, q.dtype, q.flags,
+                lda_of(q), ldb_of(q), family_name(choose(q)));
     switch (choose(q)) {
         case FAM_UMMA:
         case FAM_UMMA_PAIR:
@@ -672,14 +697,7 @@ extern "C" const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64
     if (batch <= 0 || M <= 0 || N <= 0 || K <= 0) return nullptr;
     Problem q{batch, M, N, K, dtype, A, B, const_cast<void*>(C), M * K, K * N, M * N, flags};
     if (validate(q) != CYC_OK) return nullptr;
-    switch (choose(q)) {
-        case FAM_UMMA: return "tcgen05";
-        case FAM_UMMA_PAIR: return "tcgen05_pair";
-        case FAM_UMMA_TALL: return "tcgen05_pair_tall";
-        case FAM_UMMA_SPLITK: return "tcgen05_pair_splitk";
-        case FAM_UMMA_3XTF32: return "tcgen05_3xtf32";
-        default: return "simt";
-    }
+    return family_name(choose(q));
 }
 
 extern "C" const char* cyc_schedule_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
