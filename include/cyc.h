@@ -22,7 +22,16 @@
  * Environment.  CYC_LOG=1 (read once per process): one line on stderr for every
  * kernel selection of the matrix-multiply recurrence -- shape, dtype, flags,
  * pitches and the kernel chosen (the names of cyc_kernel_for) -- including the
- * tile products that the triangular solve and the Cholesky factorisation lay on it.
+ * tile products that the triangular solve and the Cholesky factorisation lay on it,
+ * and for every attention launch its grid (units, sliced tail).
+ *
+ * Device memory the library holds besides the caller's buffers: a 4-byte status word per
+ * device; a stream-ordered pool for split-K and solver workspaces (cyc_pool_reserved_bytes);
+ * the fixed array of cyc_recurrence_matmul_splitk_static; and, for schedules with a sliced
+ * tail, one scratch per (device, stream) -- 19.4 MB for the matrix multiply, 21.3 MB for
+ * attention, at most eight of each per device -- allocated the first time such a schedule
+ * runs on a stream and kept until the process exits (a stream beyond the eighth, or one that
+ * is being captured before it has a scratch, runs the schedule without a sliced tail).
  *
  * Layouts.  A is [M][K] row-major (K contiguous).  B is [K][N] row-major, or,
  * with CYC_FLAG_B_COL_MAJOR, stored as [N][K] (element B_kj at B[j*K + k]).

@@ -1,4 +1,6 @@
 // Shared state and helpers of the library, and the status / introspection entry points.  See include/cyc.h.
+#include <cstdlib>
+
 #include "api_internal.h"
 #include "ptx.cuh"
 
@@ -154,6 +156,81 @@ int workspace_pool(cudaMemPool_t* out, bool create) {
     *out = pools[dev];
     return CYC_OK;
 }
+// CYC_LOG=1 in the environment: one line on stderr per kernel selection (read once per process)
+bool log_enabled() {
+    static const bool on = [] {
+        const char* v = getenv("CYC_LOG");
+        return v && *v && *v != '0';
+    }();
+    return on;
+}
+
+// ------------------------------------------------------------------ scratch kept per (device, stream, purpose)
+struct KeptScratch {
+    int dev = -1;
+    cudaStream_t stream = nullptr;
+    int purpose = 0;
+    uint8_t* data = nullptr;
+    int* counters = nullptr;
+    size_t counter_bytes = 0;
+    bool dirty = false;
+};
+constexpr int kKeptScratchPerDevice = 8;  // per purpose
+constexpr int kKeptScratchMax = 128;
+static std::mutex g_scratch_mu;
+static KeptScratch g_scratch[kKeptScratchMax];
+static int g_scratch_count = 0;
+
+void kept_scratch_mark_dirty() {
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    for (int i = 0; i < g_scratch_count; ++i) g_scratch[i].dirty = true;
+}
+
+int kept_scratch_for(cudaStream_t st, int purpose, size_t data_bytes, size_t counter_bytes, uint8_t** data, int** counters) {
+    *data = nullptr;
+    *counters = nullptr;
+    int dev = 0;
+    CYC_CUDA(cudaGetDevice(&dev));
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); return CYC_OK; }
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    KeptScratch* found = nullptr;
+    int on_dev = 0;
+    for (int i = 0; i < g_scratch_count; ++i) {
+        if (g_scratch[i].dev != dev || g_scratch[i].purpose != purpose) continue;
+        ++on_dev;
+        if (g_scratch[i].stream == st) found = &g_scratch[i];
+    }
+    if (!found) {
+        // creating one allocates and clears memory: not while the stream is being captured into a graph
+        if (cap != cudaStreamCaptureStatusNone || on_dev >= kKeptScratchPerDevice || g_scratch_count >= kKeptScratchMax) return CYC_OK;
+        const size_t data_padded = (data_bytes + 255) & ~static_cast<size_t>(255);
+        void* mem = nullptr;
+        if (cudaMalloc(&mem, data_padded + counter_bytes) != cudaSuccess) { cudaGetLastError(); return CYC_OK; }
+        if (cudaMemset(static_cast<uint8_t*>(mem) + data_padded, 0, counter_bytes) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(mem);
+            return CYC_OK;
+        }
+        found = &g_scratch[g_scratch_count++];
+        found->dev = dev;
+        found->stream = st;
+        found->purpose = purpose;
+        found->data = static_cast<uint8_t*>(mem);
+        found->counters = reinterpret_cast<int*>(found->data + data_padded);
+        found->counter_bytes = counter_bytes;
+        found->dirty = false;
+    }
+    if (found->dirty) {
+        if (cap != cudaStreamCaptureStatusNone) return CYC_OK;
+        CYC_CUDA(cudaMemsetAsync(found->counters, 0, found->counter_bytes, st));
+        found->dirty = false;
+    }
+    *data = found->data;
+    *counters = found->counters;
+    return CYC_OK;
+}
+
 }  // namespace cyc
 
 using namespace cyc;
@@ -187,7 +264,7 @@ extern "C" int cyc_last_device_status(void* stream, int* out) {
     CYC_CUDA(cudaMemcpyFromSymbol(&word, g_device_status, sizeof word));
     if (word != 0) {
         const int zero = 0;
-        tail_scratch_mark_dirty();  // a kernel that gave up may have left strip counters of the sliced tail non-zero
+        kept_scratch_mark_dirty();  // a kernel that gave up may have left arrival counters of a sliced tail non-zero
         CYC_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero));
         snprintf(g_err, sizeof g_err, "device wait ran out (code 0x%x)", word);
     }

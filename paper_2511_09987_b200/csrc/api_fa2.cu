@@ -5,8 +5,23 @@
 namespace cyc {
 
 // ------------------------------------------------------------------ FlashAttention-2 recurrence
+// Scratch of the sliced tail: at most one part per SM, eight warps of row threads per part, sized for the larger head dimension.
+constexpr int kFa2MaxSms = 160;
+constexpr size_t kFa2TailDataBytes = static_cast<size_t>(kFa2MaxSms) * 8 * fa2_tail_slot_floats(128) * sizeof(float);
+constexpr size_t kFa2TailCounterBytes = static_cast<size_t>(kFa2MaxSms / 2) * 8 * sizeof(int);
+
+// How many parts each unit of the grid's last, partial round is cut into (0 = no tail): the parts of that round must
+// fit the SMs at once, every part keeps at least two key tiles, at most FA2_TAIL_MAX_PARTS.
+static int fa2_tail_parts(long long units, long long key_tiles, int sms) {
+    if (sms > kFa2MaxSms) return 0;
+    const long long rem = units % sms;
+    if (rem == 0) return 0;
+    const long long parts = std::min<long long>({sms / rem, key_tiles / 2, FA2_TAIL_MAX_PARTS});
+    return parts >= 2 ? static_cast<int>(parts) : 0;
+}
+
 template <int D>
-static int launch_fa2(long long batch, long long N, long long M, const void* Q, const void* K, const void* V, float* O, cudaStream_t st) {
+static int launch_fa2(long long batch, long long N, long long M, const void* Q, const void* K, const void* V, float* O, cudaStream_t st, int sms) {
     CUtensorMap tmQ, tmK, tmV;
     int rc = make_map(&tmQ, CYC_BF16_F32, Q, D, N, batch, D, N * D, 64, FA2_BM);
     if (rc) return rc;
@@ -35,7 +50,29 @@ static int launch_fa2(long long batch, long long N, long long M, const void* Q, 
         }
     }
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), Fa2Smem<D>::TOTAL)) return rc_;
-    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(batch * p.tiles_q), FA2_THREADS, Fa2Smem<D>::TOTAL, st, tmQ, tmK, tmV, p));
+    const long long units = batch * p.tiles_q;
+    long long ctas = units;
+    p.full_units = static_cast<int>(units);
+    p.tail_parts = 0;
+    p.tail_ws = nullptr;
+    p.tail_counters = nullptr;
+    if (const int parts = fa2_tail_parts(units, (M + FA2_BN - 1) / FA2_BN, sms)) {
+        uint8_t* data = nullptr;
+        int* counters = nullptr;
+        if (int rc_ = kept_scratch_for(st, SCRATCH_ATTENTION_TAIL, kFa2TailDataBytes, kFa2TailCounterBytes, &data, &counters)) return rc_;
+        if (data) {
+            const long long rem = units % sms;
+            p.full_units = static_cast<int>(units - rem);
+            p.tail_parts = parts;
+            p.tail_ws = reinterpret_cast<float*>(data);
+            p.tail_counters = counters;
+            ctas = p.full_units + rem * parts;
+        }
+    }
+    if (log_enabled())
+        fprintf(stderr, "cyc: attention batch=%lld N=%lld M=%lld d=%d -> fa2 units=%lld tail_units=%lld tail_parts=%d ctas=%lld\n", batch, N, M, D, units,
+                units - p.full_units, p.tail_parts, ctas);
+    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(ctas), FA2_THREADS, Fa2Smem<D>::TOTAL, st, tmQ, tmK, tmV, p));
     g_launches.fetch_add(1);
     return CYC_OK;
 }
@@ -72,6 +109,6 @@ extern "C" int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t 
         return CYC_ERR_UNSUPPORTED;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return d == 64 ? launch_fa2<64>(batch, N, M, Q, K, V, static_cast<float*>(O), st)
-                   : launch_fa2<128>(batch, N, M, Q, K, V, static_cast<float*>(O), st);
+    return d == 64 ? launch_fa2<64>(batch, N, M, Q, K, V, static_cast<float*>(O), st, di.sms)
+                   : launch_fa2<128>(batch, N, M, Q, K, V, static_cast<float*>(O), st, di.sms);
 }

@@ -82,9 +82,18 @@ struct DeviceInfo {
     bool known = false;
 };
 int device_info(DeviceInfo* out);
+bool log_enabled();                                       // CYC_LOG=1 in the environment
 int status_word(int** out);                               // device address of the status word, cached per device
 int ensure_dynamic_smem(const void* kernel, int bytes);   // opt-in to large dynamic shared memory, once per (kernel, device)
 int workspace_pool(cudaMemPool_t* out, bool create = true);  // the library's stream-ordered pool on the current device
-void tail_scratch_mark_dirty();                           // after a device-side timeout: clear the sliced-tail counters before reuse
+// Scratch kept for the life of the process, one per (device, stream, purpose): `data_bytes` of partial results and
+// `counter_bytes` of arrival counters that are zero when a launch starts and that the kernel leaves zero.  Launches on
+// one stream are ordered, launches on different streams are not, hence one scratch per stream; at most eight are made
+// per device and purpose.  *data stays nullptr (and the call returns CYC_OK) when none can be had -- the stream is being
+// captured and has no scratch yet, the limit is reached, or the allocation failed -- and the caller then runs a
+// schedule that needs none.  A purpose always asks for the same sizes.
+enum ScratchPurpose { SCRATCH_MATMUL_TAIL = 0, SCRATCH_ATTENTION_TAIL = 1 };
+int kept_scratch_for(cudaStream_t st, int purpose, size_t data_bytes, size_t counter_bytes, uint8_t** data, int** counters);
+void kept_scratch_mark_dirty();  // after a device-side timeout counters may be non-zero: the next use of each scratch clears them
 
 }  // namespace cyc

@@ -191,71 +191,10 @@ static TailPlan plan_tail(const Problem& q, long long num_tiles, long long pairs
     return tp;
 }
 
-// Scratch of the sliced tail: partial-sum slots for up to one slice per CTA pair and one counter per 32-row strip.
-// The counters must be zero when a launch starts and the kernel leaves them zero, so the memory is kept for the
-// life of the process -- one scratch per (device, stream), because launches on one stream are ordered and launches on
-// different streams are not.  At most kTailScratchMax are created per device; beyond that a launch simply runs the
-// plain schedule.  A device-side timeout may leave counters non-zero: cyc_last_device_status marks every scratch
-// dirty and the next use clears it on its stream.
-struct TailScratch {
-    int dev = -1;
-    cudaStream_t stream = nullptr;
-    uint8_t* ws = nullptr;
-    int* counters = nullptr;
-    bool dirty = false;
-};
-constexpr int kTailScratchMax = 8;
+// Scratch of the sliced tail: partial-sum slots for up to one slice per CTA pair and one counter per 32-row strip,
+// kept per (device, stream) by kept_scratch_for.
+constexpr size_t kTailDataBytes = static_cast<size_t>(kCtaPairs) * PAIR_TILE_BYTES;
 constexpr size_t kTailCounterBytes = static_cast<size_t>(kCtaPairs) * PAIR_STRIPS * sizeof(int);
-static std::mutex g_tail_mu;
-static TailScratch g_tail_scratch[64];
-static int g_tail_scratch_count = 0;
-
-void tail_scratch_mark_dirty() {
-    std::lock_guard<std::mutex> lk(g_tail_mu);
-    for (int i = 0; i < g_tail_scratch_count; ++i) g_tail_scratch[i].dirty = true;
-}
-
-// returns CYC_OK with *out = nullptr when no scratch can be had (the caller then runs the plain schedule)
-static int tail_scratch_for(cudaStream_t st, TailScratch** out) {
-    *out = nullptr;
-    int dev = 0;
-    CYC_CUDA(cudaGetDevice(&dev));
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); return CYC_OK; }
-    std::lock_guard<std::mutex> lk(g_tail_mu);
-    TailScratch* found = nullptr;
-    int on_dev = 0;
-    for (int i = 0; i < g_tail_scratch_count; ++i) {
-        if (g_tail_scratch[i].dev != dev) continue;
-        ++on_dev;
-        if (g_tail_scratch[i].stream == st) found = &g_tail_scratch[i];
-    }
-    if (!found) {
-        // creating one allocates and clears memory: not while the stream is being captured into a graph
-        if (cap != cudaStreamCaptureStatusNone || on_dev >= kTailScratchMax || g_tail_scratch_count >= 64) return CYC_OK;
-        void* mem = nullptr;
-        const size_t bytes = static_cast<size_t>(kCtaPairs) * PAIR_TILE_BYTES + kTailCounterBytes;
-        if (cudaMalloc(&mem, bytes) != cudaSuccess) { cudaGetLastError(); return CYC_OK; }
-        if (cudaMemset(static_cast<uint8_t*>(mem) + static_cast<size_t>(kCtaPairs) * PAIR_TILE_BYTES, 0, kTailCounterBytes) != cudaSuccess) {
-            cudaGetLastError();
-            cudaFree(mem);
-            return CYC_OK;
-        }
-        found = &g_tail_scratch[g_tail_scratch_count++];
-        found->dev = dev;
-        found->stream = st;
-        found->ws = static_cast<uint8_t*>(mem);
-        found->counters = reinterpret_cast<int*>(found->ws + static_cast<size_t>(kCtaPairs) * PAIR_TILE_BYTES);
-        found->dirty = false;
-    }
-    if (found->dirty) {
-        if (cap != cudaStreamCaptureStatusNone) return CYC_OK;
-        CYC_CUDA(cudaMemsetAsync(found->counters, 0, kTailCounterBytes, st));
-        found->dirty = false;
-    }
-    *out = found;
-    return CYC_OK;
-}
 
 // ------------------------------------------------------------------ two-SM tensor-core launch
 // `ws` != nullptr: split-K -- the kernel writes plan.S planes of partial sums per problem into ws
@@ -300,11 +239,12 @@ static int launch_pair_cfg(const Problem& q, cudaStream_t st, int sms, void* ws 
     if (!ws && pairs <= kCtaPairs) {
         const TailPlan tp = plan_tail(q, p.num_tiles, pairs);
         if (tp.S > 1) {
-            TailScratch* sc = nullptr;
-            if (int rc_ = tail_scratch_for(st, &sc)) return rc_;
-            if (sc) {
+            uint8_t* data = nullptr;
+            int* counters = nullptr;
+            if (int rc_ = kept_scratch_for(st, SCRATCH_MATMUL_TAIL, kTailDataBytes, kTailCounterBytes, &data, &counters)) return rc_;
+            if (data) {
                 p.tail_S = tp.S; p.tail_tiles = tp.tiles; p.tail_kb = tp.kb;
-                p.tail_ws = sc->ws; p.tail_counters = sc->counters;
+                p.tail_ws = data; p.tail_counters = counters;
             }
         }
     }
@@ -459,15 +399,6 @@ static const char* family_name(Family f) {
         case FAM_UMMA_3XTF32: return "tcgen05_3xtf32";
         default: return "simt";
     }
-}
-
-// CYC_LOG=1 in the environment: one line on stderr per kernel selection (read once per process)
-static bool log_enabled() {
-    static const bool on = [] {
-        const char* v = getenv("CYC_LOG");
-        return v && *v && *v != '0';
-    }();
-    return on;
 }
 
 int route(const Problem& q, cudaStream_t st) {

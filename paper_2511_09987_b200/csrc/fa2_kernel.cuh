@@ -19,6 +19,13 @@
 // the recurrence's result does not depend on which reference is used (the same factor multiplies o and l), the
 // exponentials stay below 2^8 in bf16 / fp32, and the rescale of o, a read-modify-write of tensor memory, becomes rare.
 // Exponentials are 2^x on the scores scaled by alpha*log2(e).  bf16 inputs, fp32 output.  Every wait is bounded.
+//
+// Sliced tail.  The grid's last, partial round of CTAs would leave most SMs idle for a whole pass over the keys.  The
+// host may therefore cut each (problem, 256 queries) unit of that round into 2 to 4 parts by key range, one CTA each.
+// A part keeps its own (m, l, o); the recurrence is associative in these triples,
+//   (m, l, o) = (max(m_a, m_b), l_a 2^(m_a-m) + l_b 2^(m_b-m), o_a 2^(m_a-m) + o_b 2^(m_b-m)),
+// so each warp of row threads writes its 32 rows' triple to scratch, counts itself in, and the last part to arrive for
+// those rows folds all parts together in part order (the same bits whichever part arrives last) and writes O.
 #pragma once
 #include <cstdint>
 #include <cuda.h>
@@ -40,7 +47,15 @@ struct Fa2Params {
     int tiles_q;       // ceil(N / 256)
     float scale_log2;  // alpha * log2(e)
     int* status;       // device status word
+    // sliced tail: CTAs [0, full_units) take a whole unit each; after them come tail_parts CTAs per remaining unit
+    int full_units;      // = batch * tiles_q when there is no tail
+    int tail_parts;      // 0 (no tail) or 2..4
+    float* tail_ws;      // [tail unit][part][query tile][row warp] slots of fa2_tail_slot_floats(D) floats
+    int* tail_counters;  // [tail unit][query tile][warp], zero between launches
 };
+constexpr int FA2_TAIL_MAX_PARTS = 4;
+// the partial state of one warp's 32 rows: 32 x D of o, then 32 m, then 32 l
+__host__ __device__ constexpr int fa2_tail_slot_floats(int d) { return 32 * d + 64; }
 
 struct Fa2Ctl {
     uint64_t q_full;
@@ -146,9 +161,18 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     Fa2Ctl* ctl = reinterpret_cast<Fa2Ctl*>(sKV + 2 * Sm::STAGE_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x / p.tiles_q, qt = blockIdx.x - b * p.tiles_q;
+    // which unit (problem, 256 queries) and which key tiles [kt0, kt0 + T) of it this CTA walks
+    int unit = blockIdx.x, part = -1, kt0 = 0;
+    int T = (p.M + FA2_BN - 1) / FA2_BN;
+    if (static_cast<int>(blockIdx.x) >= p.full_units) {
+        const int x = blockIdx.x - p.full_units;
+        unit = p.full_units + x / p.tail_parts;
+        part = x - (unit - p.full_units) * p.tail_parts;
+        kt0 = static_cast<int>(static_cast<long long>(T) * part / p.tail_parts);
+        T = static_cast<int>(static_cast<long long>(T) * (part + 1) / p.tail_parts) - kt0;
+    }
+    const int b = unit / p.tiles_q, qt = unit - b * p.tiles_q;
     const int n0 = qt * FA2_ROWS;
-    const int T = (p.M + FA2_BN - 1) / FA2_BN;          // key tiles
     const int ntq = (n0 + FA2_BM < p.N) ? 2 : 1;        // query tiles of this CTA that hold rows of the problem
 
     ptx::grid_launch_dependents();
@@ -205,13 +229,13 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 ptx::mbar_arrive_expect_tx(&ctl->k_full[st], Sm::K_BYTES);
 #pragma unroll
                 for (int kb = 0; kb < D / 64; ++kb)
-                    ptx::tma_load_3d(sK + kb * Sm::SLAB, &tmK, &ctl->k_full[st], kb * 64, t * FA2_BN, b);  // keys x 64 of d
+                    ptx::tma_load_3d(sK + kb * Sm::SLAB, &tmK, &ctl->k_full[st], kb * 64, (kt0 + t) * FA2_BN, b);  // keys x 64 of d
                 ++issued_k;
                 if (!fa2_wait(&ctl->v_empty[st], ph ^ 1, ctl, p.status, 8)) { ok = false; break; }
                 ptx::mbar_arrive_expect_tx(&ctl->v_full[st], Sm::V_BYTES);
 #pragma unroll
                 for (int kb = 0; kb < D / 64; ++kb)
-                    ptx::tma_load_3d(sV + kb * Sm::SLAB, &tmV, &ctl->v_full[st], kb * 64, t * FA2_BN, b);  // keys x d-chunk kb
+                    ptx::tma_load_3d(sV + kb * Sm::SLAB, &tmV, &ctl->v_full[st], kb * 64, (kt0 + t) * FA2_BN, b);  // keys x d-chunk kb
                 ++issued_v;
             }
             if (!ok) {
@@ -308,7 +332,7 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             for (int t = 0; t < T && ok; ++t) {
                 if (!fa2_wait(&ctl->s_full[i], t & 1, ctl, p.status, 7)) { ok = false; break; }
                 ptx::tc_fence_after();
-                const int valid = min(FA2_BN, p.M - t * FA2_BN);  // keys of this tile that exist (< 128 only in the last)
+                const int valid = min(FA2_BN, p.M - (kt0 + t) * FA2_BN);  // keys of this tile that exist (< 128 only in the last)
                 // ---- the row's 128 scores, read once and kept in registers from the maximum to the exponentials
                 uint32_t v[FA2_BN];
 #pragma unroll
@@ -368,9 +392,86 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&ctl->p_ready[i]);
             }
-            ctl->row_l[i][r] = l;
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&ctl->l_done[i]);
+            if (part < 0) {
+                ctl->row_l[i][r] = l;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&ctl->l_done[i]);
+            } else if (ok && fa2_wait(&ctl->pv_done[i], (T - 1) & 1, ctl, p.status, 13)) {
+                // ---- a part of a sliced unit: its (m, l, o) for these 32 rows go to scratch; the last part to arrive folds
+                // ---- all parts in part order.  (The row threads do this, not the keepers: they are idle by now, both query
+                // ---- tiles proceed at once, and they have the registers to keep a whole round of loads in flight.)
+                ptx::tc_fence_after();
+                const uint32_t o_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + COL_O + i * D;
+                // slot of part k; within it piece j (four columns) of lane t sits at float (j * 32 + t) * 4, so that a warp
+                // writes and reads 512 contiguous bytes at a time
+                constexpr int SLOT = fa2_tail_slot_floats(D);
+                const int tu = unit - p.full_units, w = i * 4 + q;
+                float* slots = p.tail_ws + (static_cast<size_t>(tu) * p.tail_parts * 8 + w) * SLOT;
+                float* mine = slots + static_cast<size_t>(part) * 8 * SLOT;
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t v[32];
+                    ptx::tmem_ld_32x32(o_addr + c0, v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int g = 0; g < 32; g += 4)
+                        *reinterpret_cast<float4*>(mine + (((c0 + g) >> 2) * 32 + lane) * 4) =
+                            make_float4(__uint_as_float(v[g]), __uint_as_float(v[g + 1]), __uint_as_float(v[g + 2]), __uint_as_float(v[g + 3]));
+                }
+                mine[32 * D + lane] = m_ref;
+                mine[32 * D + 32 + lane] = l;
+                __threadfence();
+                __syncwarp();
+                int arrived = 0;
+                if (lane == 0) arrived = atomicAdd(&p.tail_counters[tu * 8 + w], 1);
+                arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                if (arrived == p.tail_parts - 1) {
+                    if (lane == 0) p.tail_counters[tu * 8 + w] = 0;  // every part has arrived: zero again for the next launch
+                    __threadfence();
+                    float a[FA2_TAIL_MAX_PARTS], m = -INFINITY, lsum = 0.f;
+#pragma unroll
+                    for (int k = 0; k < FA2_TAIL_MAX_PARTS; ++k) {
+                        a[k] = -INFINITY;
+                        if (k < p.tail_parts) a[k] = __ldcg(slots + static_cast<size_t>(k) * 8 * SLOT + 32 * D + lane);
+                        m = fmaxf(m, a[k]);
+                    }
+#pragma unroll
+                    for (int k = 0; k < FA2_TAIL_MAX_PARTS; ++k) {
+                        a[k] = fa2_exp2(a[k] - m);  // 0 for a part that does not exist
+                        if (k < p.tail_parts)
+                            lsum = __fadd_rn(lsum, __fmul_rn(__ldcg(slots + static_cast<size_t>(k) * 8 * SLOT + 32 * D + 32 + lane), a[k]));
+                    }
+                    const float inv = 1.0f / lsum;
+                    const int row = n0 + i * FA2_BM + r;
+                    float* dst = p.O + (static_cast<long long>(b) * p.N + row) * D;
+#pragma unroll
+                    for (int c0 = 0; c0 < D; c0 += 32) {
+                        float4 x[FA2_TAIL_MAX_PARTS][8];  // all loads of 32 columns in flight at once
+#pragma unroll
+                        for (int k = 0; k < FA2_TAIL_MAX_PARTS; ++k)
+                            if (k < p.tail_parts) {
+#pragma unroll
+                                for (int g = 0; g < 8; ++g)
+                                    x[k][g] = __ldcg(reinterpret_cast<const float4*>(slots + static_cast<size_t>(k) * 8 * SLOT + (((c0 >> 2) + g) * 32 + lane) * 4));
+                            }
+                        if (row < p.N) {
+#pragma unroll
+                            for (int g = 0; g < 8; ++g) {
+                                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                                for (int k = 0; k < FA2_TAIL_MAX_PARTS; ++k)
+                                    if (k < p.tail_parts) {
+                                        acc.x = __fadd_rn(acc.x, __fmul_rn(x[k][g].x, a[k]));
+                                        acc.y = __fadd_rn(acc.y, __fmul_rn(x[k][g].y, a[k]));
+                                        acc.z = __fadd_rn(acc.z, __fmul_rn(x[k][g].z, a[k]));
+                                        acc.w = __fadd_rn(acc.w, __fmul_rn(x[k][g].w, a[k]));
+                                    }
+                                *reinterpret_cast<float4*>(dst + c0 + g * 4) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                            }
+                        }
+                    }
+                }
+            }
         }
         ptx::tc_fence_before();
     } else {
@@ -404,14 +505,14 @@ fa2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (lane == 0) ptx::mbar_arrive(&ctl->o_ready[i]);
             }
         }
-        // ---- O = o / l
-        for (int i = 0; i < ntq && ok; ++i) {
+        // ---- O = o / l (the parts of a sliced unit are folded by their row threads instead)
+        for (int i = 0; i < ntq && ok && part < 0; ++i) {
             if (!fa2_wait(&ctl->pv_done[i], (T - 1) & 1, ctl, p.status, 11)) { ok = false; break; }
             if (!fa2_wait(&ctl->l_done[i], 0, ctl, p.status, 12)) { ok = false; break; }
             ptx::tc_fence_after();
             const int row = n0 + i * FA2_BM + r;
-            const float inv = 1.0f / ctl->row_l[i][r];
             float* dst = p.O + (static_cast<long long>(b) * p.N + row) * D;
+            const float inv = 1.0f / ctl->row_l[i][r];
 #pragma unroll
             for (int c0 = 0; c0 < D; c0 += 32) {
                 uint32_t v[32];
