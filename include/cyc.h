@@ -267,12 +267,12 @@ int cyc_prefix_sum(int64_t rows, int64_t n, int dtype, const void* A, int64_t st
  *   flags  0, or CYC_FLAG_FIXED_K_ORDER: the SYRK / GEMM sums then run as per-element fp32
  *          fused-multiply-add chains in increasing k (bit-reproducible, slower); without it they
  *          may run on the tensor cores (fp32 split into TF32 parts).
- * A matrix that is not positive definite yields NaN from the square root of a non-positive
- * pivot, as the recurrence does; it is not an error.  The SYRK / GEMM sums are evaluated by the
+ * A matrix that is not positive definite yields NaN (or infinities) from the square root of a
+ * non-positive pivot, as the recurrence does; it is not an error.  The SYRK / GEMM sums are evaluated by the
  * same kernels as cyc_recurrence_matmul (both operands sub-blocks of L with row pitch n) into a
  * workspace of (n - T) * T * 4 bytes from the library's stream-ordered pool; everything
- * else is fp32 with IEEE square roots; divisions by a pivot are multiplications by its correctly
- * rounded reciprocal.
+ * else is fp32; L_kk and the divisions by it are products with 1 / sqrt(pivot), computed to
+ * about 1e-7 relative (hardware reciprocal square root and one Newton step).
  * Asynchronous on `stream`; the caller owns A and L; errors as for cyc_recurrence_matmul.
  */
 int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, void* L, void* stream, unsigned flags);

@@ -150,32 +150,43 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
         trsm_cp_async_commit();
     }
 
-    // right-hand side of the tile: B_ii - Xa, Xa = the partial-sum planes in increasing level.  Eight rows per warp
-    // at a time, all their loads in flight together.
-    for (int rb = 0; rb < TRSM_T_MAX; rb += 8 * TRSM_WARPS) {
-        float v[8], xa[8];
-        long long at[8];
-        bool ok[8];
+    // right-hand side of the tile: B_ii - Xa, Xa = the partial-sum planes in increasing level.  A thread holds its
+    // sixteen rows (one column) at once, so that the loads of a whole plane -- two planes at a time -- are in flight
+    // together: the planes come from DRAM, and this prologue is all latency.
+    {
+        constexpr int RPT = TRSM_T_MAX / TRSM_WARPS;  // rows per thread
+        float v[RPT], xa[RPT];
+        unsigned okm = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = rb + TRSM_WARPS * i + warp;
-            ok[i] = r < p.rows && col_ok;
-            at[i] = r * p.w_r + c * p.w_c;
-            v[i] = ok[i] ? __ldg(p.B + r * p.b_r + c * p.b_c) : 0.f;
+        for (int i = 0; i < RPT; ++i) {
+            const int r = TRSM_WARPS * i + warp;
+            const bool ok = r < p.rows && col_ok;
+            okm |= static_cast<unsigned>(ok) << i;
+            v[i] = ok ? __ldg(p.B + r * p.b_r + c * p.b_c) : 0.f;
             xa[i] = 0.f;
         }
+        const long long wcol = c * p.w_c;
         unsigned mk = p.mask;
-        for (int l = 0; mk; ++l, mk >>= 1) {
-            if (!(mk & 1u)) continue;
-            const float* Wl = p.W + l * p.plane;
-            float w[8];
+        while (mk) {
+            const int l0 = __ffs(mk) - 1;
+            mk &= mk - 1;
+            const int l1 = mk ? __ffs(mk) - 1 : -1;
+            if (l1 >= 0) mk &= mk - 1;
+            const float* W0 = p.W + l0 * p.plane + wcol;
+            const float* W1 = p.W + (l1 >= 0 ? l1 : l0) * p.plane + wcol;
+            float w0[RPT], w1[RPT];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) w[i] = ok[i] ? __ldg(Wl + at[i]) : 0.f;
+            for (int i = 0; i < RPT; ++i) {
+                const bool ok = (okm >> i) & 1u;
+                const long long at = (TRSM_WARPS * i + warp) * p.w_r;
+                w0[i] = ok ? __ldg(W0 + at) : 0.f;
+                w1[i] = (ok && l1 >= 0) ? __ldg(W1 + at) : 0.f;
+            }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) xa[i] += w[i];
+            for (int i = 0; i < RPT; ++i) xa[i] = (xa[i] + w0[i]) + w1[i];
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) Xs[rb + TRSM_WARPS * i + warp][lane] = v[i] - xa[i];
+        for (int i = 0; i < RPT; ++i) Xs[TRSM_WARPS * i + warp][lane] = v[i] - xa[i];
     }
 
     // Diagonal block s prepared for the column sweep: every row r scaled by 1 / L_rr (so that the sweep needs no

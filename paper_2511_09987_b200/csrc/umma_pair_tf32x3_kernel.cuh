@@ -13,11 +13,11 @@
 // buffer before the MMA thread may read it (the landed tile itself serves as the hi
 // part).  The split is element-wise, so it is indifferent to the swizzled tile layout.
 //
-// Barriers: full[s] (per CTA: its own 32 KB of copies), ready[s] (leader: 8 arrivals = the
-// four split warps of the stage's turn in each CTA; the peer's arrive across the pair with a
-// CTA-scope release, which is enough because every split thread has already made its writes
-// visible to the async proxy and the tiles are read by the tensor cores only), empty[s]
-// (both, by the leader's multicast commit), acc_full[a] (both), acc_empty[a] (leader, 8).
+// Barriers: full[s] (per CTA: its own 32 KB of copies), ready[l] (leader: the split warps of
+// the stage's turn in each CTA; the peer's arrive across the pair with a CTA-scope release,
+// which is enough because every split thread has already made its writes visible to the async
+// proxy and the tiles are read by the tensor cores only), empty[s] and lo_empty[l] (both, by
+// the leader's multicast commits), acc_full[a] (both), acc_empty[a] (leader, 8).
 #pragma once
 #include "umma_pair_kernel.cuh"
 
@@ -33,21 +33,30 @@ constexpr int X3_THREADS = 192 + X3_SPLIT_WARPS * 32;     // TMA, MMA, 4 epilogu
 #ifndef CYC_X3_BK
 #define CYC_X3_BK 32
 #endif
-// A stage holds BK = 32 (or 16) values of k: A (128 rows) + B half (128 columns), BK * 4 bytes of k each, followed by their
-// lo parts.  The ring is 192 KB either way: three stages of 64 KB or six of 32 KB (64-byte swizzle).  Measured on the
-// 65536 x 256 x 256 problem: 49-52 microseconds with three stages, 61-62 with six -- the stage rate is set by the bytes
-// that cross shared memory per unit of k (TMA write, split read and write, operand reads of three MMAs), not by the depth.
+// A stage holds BK = 32 (or 16) values of k: A (128 rows) + B half (128 columns), BK * 4 bytes of k each.  Two rings share
+// 192 KB: the landed fp32 tiles (read by the MMAs as the hi parts) and the lo parts the split warps derive from them.  A
+// landed tile is held from the copy's issue to the end of its MMAs, a lo tile only from the split to the end of the MMAs,
+// so the first ring is the deeper one (four and two stages of 32 KB; three and three were 49-52 microseconds on the
+// 65536 x 256 x 256 problem).  Six and six stages of 16 KB (BK = 16, 64-byte swizzle) measured 61-62: what counts is the
+// bytes in flight, not the number of stages.
 constexpr int X3_BK = CYC_X3_BK;
 constexpr int X3_STAGE_HI = 2 * 128 * X3_BK * 4;
-constexpr int X3_STAGE_BYTES = 2 * X3_STAGE_HI;  // hi parts followed by lo parts
-constexpr int X3_STAGES = 96 / X3_BK;
+#ifndef CYC_X3_RAW_STAGES
+#define CYC_X3_RAW_STAGES (128 / CYC_X3_BK)
+#endif
+#ifndef CYC_X3_LO_STAGES
+#define CYC_X3_LO_STAGES (64 / CYC_X3_BK)
+#endif
+constexpr int X3_RAW_STAGES = CYC_X3_RAW_STAGES, X3_LO_STAGES = CYC_X3_LO_STAGES;
+static_assert(X3_RAW_STAGES <= 8 && X3_LO_STAGES <= 8 && X3_LO_STAGES <= X3_RAW_STAGES, "ring sizes");
 constexpr int X3_PREFETCH = 256 / X3_BK;  // k-blocks of A requested from L2 ahead of the ring
-constexpr int X3_SMEM_BYTES = X3_STAGES * X3_STAGE_BYTES + PAIR_STAGING_BYTES_4 + 1024 + 1024;
+constexpr int X3_SMEM_BYTES = (X3_RAW_STAGES + X3_LO_STAGES) * X3_STAGE_HI + PAIR_STAGING_BYTES_4 + 1024 + 1024;
 
 struct X3Ctl {
-    uint64_t full[8];
-    uint64_t ready[8];
-    uint64_t empty[8];
+    uint64_t full[8];      // landed-tile ring: copies done
+    uint64_t empty[8];     // landed-tile ring: MMAs done
+    uint64_t ready[8];     // lo ring: split done
+    uint64_t lo_empty[8];  // lo ring: MMAs done
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint32_t tmem_base;
@@ -81,11 +90,12 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     constexpr int CH = 32;   // B stored [K][N]: columns per 128-byte row
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t IDESC = umma_instr_desc(1, 2, B_MN, 256, PAIR_BN);
-    constexpr int STAGES = X3_STAGES;
+    constexpr int STAGES = X3_RAW_STAGES, LSTAGES = X3_LO_STAGES;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint8_t* staging = smem + STAGES * X3_STAGE_BYTES;
+    uint8_t* smem_lo = smem + STAGES * X3_STAGE_HI;
+    uint8_t* staging = smem_lo + LSTAGES * X3_STAGE_HI;
     X3Ctl* ctl = reinterpret_cast<X3Ctl*>(staging + PAIR_STAGING_BYTES_4);
 
     const int warp = threadIdx.x >> 5;
@@ -99,8 +109,11 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(&ctl->full[s], 1);
-            ptx::mbar_init(&ctl->ready[s], 2 * X3_SET_WARPS);  // the split warps of the stage's turn, both CTAs
             ptx::mbar_init(&ctl->empty[s], 1);
+        }
+        for (int l = 0; l < LSTAGES; ++l) {
+            ptx::mbar_init(&ctl->ready[l], 2 * X3_SET_WARPS);  // the split warps of the stage's turn, both CTAs
+            ptx::mbar_init(&ctl->lo_empty[l], 1);
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(&ctl->acc_full[a], 1);
@@ -153,7 +166,7 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 for (int kb = w.kb0; kb < w.kb0 + w.nkb; ++kb) {
                     prefetch_next();
                     if (!x3_wait(&ctl->empty[stage], phase ^ 1, ctl, p.status, 1)) { ok = false; break; }
-                    uint8_t* sa = smem + stage * X3_STAGE_BYTES;
+                    uint8_t* sa = smem + stage * X3_STAGE_HI;
                     uint8_t* sb = sa + 128 * BK * 4;
                     ptx::mbar_arrive_expect_tx(&ctl->full[stage], X3_STAGE_HI);
                     ptx::tma_load_3d(sa, &tmA, &ctl->full[stage], kb * BK, m0, b);
@@ -184,8 +197,8 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (rank == 0) {  // the whole warp walks the loop converged, one elected lane issues
             const uint32_t leader = ptx::elect_one();
-            int stage = 0;
-            uint32_t phase = 0;
+            int stage = 0, lstage = 0;
+            uint32_t lphase = 0;
             int local = 0;
             bool ok = true;
             PairWork w;
@@ -196,32 +209,36 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * PAIR_BN);
                 for (int kb = 0; kb < w.nkb; ++kb) {  // the first k-block of a slice starts from zero
-                    if (!x3_wait(&ctl->ready[stage], phase, ctl, p.status, 3)) { ok = false; break; }
+                    if (!x3_wait(&ctl->ready[lstage], lphase, ctl, p.status, 3)) { ok = false; break; }
                     ptx::tc_fence_after();
-                    const uint32_t sa = ptx::smem_u32(smem + stage * X3_STAGE_BYTES);
+                    const uint32_t sa = ptx::smem_u32(smem + stage * X3_STAGE_HI);
                     const uint32_t sb = sa + 128 * BK * 4;
+                    const uint32_t la = ptx::smem_u32(smem_lo + lstage * X3_STAGE_HI);
+                    const uint32_t lb = la + 128 * BK * 4;
 #pragma unroll
                     for (int k = 0; k < BK / UK; ++k) {
                         // K-major rows of BK * 4 bytes (128- or 64-byte swizzle), groups of 8 rows one after another
                         constexpr uint32_t KSBO = 8 * BK * 4, KSW = BK == 32 ? 2 : 4;
                         const uint64_t a_hi = umma_smem_desc(sa + k * 32, 16, KSBO, KSW);
-                        const uint64_t a_lo = umma_smem_desc(sa + X3_STAGE_HI + k * 32, 16, KSBO, KSW);
+                        const uint64_t a_lo = umma_smem_desc(la + k * 32, 16, KSBO, KSW);
                         uint64_t b_hi, b_lo;
                         if constexpr (!B_MN) {
                             b_hi = umma_smem_desc(sb + k * 32, 16, KSBO, KSW);
-                            b_lo = umma_smem_desc(sb + X3_STAGE_HI + k * 32, 16, KSBO, KSW);
+                            b_lo = umma_smem_desc(lb + k * 32, 16, KSBO, KSW);
                         } else {
                             // B stored [K][N]: 128-byte rows of 32 columns, 32-byte chunks permuted over groups of
                             // 4 k-rows (512 B apart); the next 32 columns are BK*128 B further on
                             b_hi = umma_smem_desc(sb + k * (UK * 128), BK * 128, 512, 1);
-                            b_lo = umma_smem_desc(sb + X3_STAGE_HI + k * (UK * 128), BK * 128, 512, 1);
+                            b_lo = umma_smem_desc(lb + k * (UK * 128), BK * 128, 512, 1);
                         }
                         ptx::umma_elect<KIND_TF32, 2>(d_tmem, a_lo, b_hi, IDESC, (kb | k) != 0 ? 1u : 0u, leader);
                         ptx::umma_elect<KIND_TF32, 2>(d_tmem, a_hi, b_lo, IDESC, 1u, leader);
                         ptx::umma_elect<KIND_TF32, 2>(d_tmem, a_hi, b_hi, IDESC, 1u, leader);
                     }
                     ptx::umma_commit_pair_elect(&ctl->empty[stage], 3, leader);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    ptx::umma_commit_pair_elect(&ctl->lo_empty[lstage], 3, leader);
+                    if (++stage == STAGES) stage = 0;
+                    if (++lstage == LSTAGES) { lstage = 0; lphase ^= 1; }
                 }
                 if (ok) ptx::umma_commit_pair_elect(&ctl->acc_full[ab], 3, leader);
             }
@@ -234,22 +251,28 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         const int set = (warp - 6) / X3_SET_WARPS;
         constexpr int NT = 32 * X3_SET_WARPS;
         const int tid = (threadIdx.x - 6 * 32) % NT;  // index within the set
-        int stage = 0;
-        uint32_t phase = 0;
+        int stage = 0, lstage = 0;
+        uint32_t phase = 0, lphase = 0;
         uint32_t turn = 0;
         bool ok = true;
         PairWork w;
+        auto advance = [&]() {
+            if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            if (++lstage == LSTAGES) { lstage = 0; lphase ^= 1; }
+        };
         for (int item = 0; ok && pair_work_item(p, num_kb, pair, num_pairs, item, w); ++item) {
             for (int kb = 0; kb < w.nkb; ++kb, ++turn) {
                 // Every set observes every use of every stage, its own or not: a parity wait tells phase k from phase
                 // k + 1 only, and copies may land out of order, so a set that skipped the other set's turn could otherwise
                 // take the previous use of a stage for the one it is waiting for.
                 if (!x3_wait(&ctl->full[stage], phase, ctl, p.status, 5)) { ok = false; break; }
+                if (!x3_wait(&ctl->lo_empty[lstage], lphase ^ 1, ctl, p.status, 6)) { ok = false; break; }
                 if (turn % X3_SPLIT_SETS != static_cast<uint32_t>(set)) {
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    advance();
                     continue;
                 }
-                uint8_t* base = smem + stage * X3_STAGE_BYTES;
+                const uint8_t* base = smem + stage * X3_STAGE_HI;
+                uint8_t* lo_base = smem_lo + lstage * X3_STAGE_HI;
 #pragma unroll 1
                 for (int it0 = 0; it0 < X3_STAGE_HI / (NT * 16); it0 += 4) {
                     uint4 v[4];
@@ -268,16 +291,16 @@ umma_pair_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                             lo[e] = ((x[e] & 0x7F800000u) == 0x7F800000u) ? 0u : tf32_round(__float_as_uint(r));
                         }
                         const int off = (tid + NT * (it0 + u)) * 16;
-                        *reinterpret_cast<uint4*>(base + X3_STAGE_HI + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                        *reinterpret_cast<uint4*>(lo_base + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                     }
                 }
                 ptx::fence_proxy_async_smem();  // generic-proxy writes -> visible to the tensor core's reads
                 __syncwarp();
                 if (lane == 0) {
-                    if (rank == 0) ptx::mbar_arrive(&ctl->ready[stage]);
-                    else ptx::mbar_arrive_remote(&ctl->ready[stage], 0);
+                    if (rank == 0) ptx::mbar_arrive(&ctl->ready[lstage]);
+                    else ptx::mbar_arrive_remote(&ctl->ready[lstage], 0);
                 }
-                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                advance();
             }
         }
     } else {
