@@ -12,9 +12,10 @@
 // The lower triangle of the tile is brought into shared memory once, as 32 x 32 blocks (cp.async; 144 KB for a full
 // tile).  The tile is then processed in sub-blocks of 32 rows, with one step of look-ahead so that the sequential part
 // overlaps the bulk of the arithmetic:
-//   solve(s)     warp 0: the 32 x 32 triangle of sub-block s by a column sweep in registers, rows pre-scaled by the
-//                reciprocal of their diagonal entry: x_r = s_r / L_rr - sum_{k<r} (L_rk / L_rr) x_k
-//   trailing(s)  twelve other warps, at the same time: rows below sub-block s  -=  L[rows][sub-block s-1] * x_(s-1)
+//   solve(s)     warps 0-3 (eight columns each, four lanes per column): the 32 x 32 triangle of sub-block s by a
+//                column sweep in registers, rows pre-scaled by the reciprocal of their diagonal entry:
+//                x_r = s_r / L_rr - sum_{k<r} (L_rk / L_rr) x_k
+//   trailing(s)  the twelve other warps, at the same time: rows below sub-block s  -=  L[rows][sub-block s-1] * x_(s-1)
 //                (a warp takes 16 rows x 32 columns, a 4 x 4 patch per lane)
 //   next(s+1)    two warps: rows of sub-block s+1  -=  L[rows][sub-block s] * x_s; eight warps prepare its triangle
 // Every row receives its updates in increasing column order.  Entries of L above the diagonal are never used.
@@ -219,42 +220,52 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
 
     for (int s = 0; s < nsb; ++s) {
         const int s0 = s * TRSM_SB;
-        if (warp == 0) {
-            // ---- solve(s): x_r = (s_r - sum_{k<r} L_rk x_k) / L_rr evaluated as s_r/L_rr - sum_k (L_rk/L_rr) x_k
-            float sv[TRSM_SB];
+        if (warp < 4) {
+            // ---- solve(s): x_r = (s_r - sum_{k<r} L_rk x_k) / L_rr evaluated as s_r/L_rr - sum_k (L_rk/L_rr) x_k.
+            // ---- Four warps, one per scheduler, eight columns each; a column is shared by four lanes that hold eight
+            // ---- consecutive rows each, so a step of the sweep is one shuffle (x_k from the lane that owns row k)
+            // ---- and eight multiply-adds per lane -- a quarter of the instructions a single warp would issue, and
+            // ---- the dependent chain of 32 steps is the shuffle and one multiply-add long.  The multipliers of step
+            // ---- k + 4 are fetched while step k is applied: the other warps keep shared memory busy.
+            const int cl = 8 * warp + (lane >> 2), q = lane & 3;   // column of the CTA's 32; row group
+            constexpr int AHEAD = 4;
+            float sv[8];
 #pragma unroll
-            for (int r = 0; r < TRSM_SB; ++r) sv[r] = Xs[s0 + r][lane] * dinv[r];
-            float4 lnext[TRSM_SB / 4];  // column k+1 of the triangle (row k+1 of Lt), fetched while column k is applied
+            for (int i = 0; i < 8; ++i) sv[i] = Xs[s0 + 8 * q + i][cl] * dinv[8 * q + i];
+            float4 la[AHEAD][2];   // Lt[k][8 q .. 8 q + 7] for the next steps
 #pragma unroll
-            for (int g = 0; g < TRSM_SB / 4; ++g) lnext[g] = *reinterpret_cast<const float4*>(&Lt[0][4 * g]);
+            for (int a = 0; a < AHEAD; ++a) {
+                la[a][0] = *reinterpret_cast<const float4*>(&Lt[a][8 * q]);
+                la[a][1] = *reinterpret_cast<const float4*>(&Lt[a][8 * q + 4]);
+            }
 #pragma unroll
             for (int k = 0; k < TRSM_SB; ++k) {
-                float4 l[TRSM_SB / 4];
-#pragma unroll
-                for (int g = 0; g < TRSM_SB / 4; ++g) l[g] = lnext[g];
-                if (k + 1 < TRSM_SB) {
-#pragma unroll
-                    for (int g = (k + 2) / 4; g < TRSM_SB / 4; ++g) lnext[g] = *reinterpret_cast<const float4*>(&Lt[k + 1][4 * g]);
+                const float4 l0 = la[k % AHEAD][0], l1 = la[k % AHEAD][1];
+                if (k + AHEAD < TRSM_SB) {
+                    la[k % AHEAD][0] = *reinterpret_cast<const float4*>(&Lt[k + AHEAD][8 * q]);
+                    la[k % AHEAD][1] = *reinterpret_cast<const float4*>(&Lt[k + AHEAD][8 * q + 4]);
                 }
-                const float xk = sv[k];
+                const float xk = __shfl_sync(0xffffffffu, sv[k & 7], (lane & ~3) | (k >> 3));
+                // only rows r > k take part (a finished row must not meet an infinite or NaN x_k): all eight rows of
+                // the lanes past the owner of row k, the rows after it in the owner itself
+                const bool past = q > (k >> 3), from = q >= (k >> 3);
+                const float lv[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
 #pragma unroll
-                for (int g = (k + 1) / 4; g < TRSM_SB / 4; ++g) {  // entries with r <= k are zero in Lt and skipped here
-                    if (4 * g + 0 > k) sv[4 * g + 0] = fmaf(-l[g].x, xk, sv[4 * g + 0]);
-                    if (4 * g + 1 > k) sv[4 * g + 1] = fmaf(-l[g].y, xk, sv[4 * g + 1]);
-                    if (4 * g + 2 > k) sv[4 * g + 2] = fmaf(-l[g].z, xk, sv[4 * g + 2]);
-                    if (4 * g + 3 > k) sv[4 * g + 3] = fmaf(-l[g].w, xk, sv[4 * g + 3]);
-                }
+                for (int i = 0; i < 8; ++i)
+                    if (i > (k & 7) ? from : past) sv[i] = fmaf(-lv[i], xk, sv[i]);
             }
+            const int c = blockIdx.x * TRSM_CW + cl;
 #pragma unroll
-            for (int r = 0; r < TRSM_SB; ++r) {
-                Xs[s0 + r][lane] = sv[r];
-                if (s0 + r < p.rows && col_ok) p.X[(s0 + r) * p.x_r + c * p.x_c] = sv[r];
+            for (int i = 0; i < 8; ++i) {
+                const int r = s0 + 8 * q + i;
+                Xs[r][cl] = sv[i];
+                if (r < p.rows && c < p.m) p.X[r * p.x_r + c * p.x_c] = sv[i];
             }
-        } else if ((warp & 3) != 0 && s >= 1 && s + 1 < nsb) {
-            // ---- trailing(s): rows below sub-block s, sixteen per warp at a time, with x of sub-block s-1.  Twelve
-            // warps: those that share warp 0's scheduler stay out of its way.
+        } else if (s >= 1 && s + 1 < nsb) {
+            // ---- trailing(s): rows below sub-block s, sixteen per warp at a time, with x of sub-block s-1: the other
+            // ---- twelve warps
             const int tasks = (nsb - s - 1) * (TRSM_SB / 16);
-            for (int g = warp - 1 - (warp >> 2); g < tasks; g += 12) {
+            for (int g = warp - 4; g < tasks; g += 12) {
                 const int t = s0 + TRSM_SB + 16 * g;  // first tile row of the task
                 trsm_apply<4>(Lb + trsm_block(t >> 5, s - 1) + (t & 31) * TRSM_SB, &Xs[s0 - TRSM_SB], &Xs[t], lane);
             }
