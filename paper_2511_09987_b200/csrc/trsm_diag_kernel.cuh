@@ -16,8 +16,8 @@
 //                column sweep in registers, rows pre-scaled by the reciprocal of their diagonal entry:
 //                x_r = s_r / L_rr - sum_{k<r} (L_rk / L_rr) x_k
 //   trailing(s)  the twelve other warps, at the same time: rows below sub-block s  -=  L[rows][sub-block s-1] * x_(s-1)
-//                (a warp takes 16 rows x 32 columns, a 4 x 4 patch per lane)
-//   next(s+1)    two warps: rows of sub-block s+1  -=  L[rows][sub-block s] * x_s; eight warps prepare its triangle
+//                (a warp takes 16 rows x 32 columns, a lane one column of them)
+//   next(s+1)    eight warps: rows of sub-block s+1  -=  L[rows][sub-block s] * x_s; the other eight prepare its triangle
 // Every row receives its updates in increasing column order.  Entries of L above the diagonal are never used.
 #pragma once
 #include <cstdint>
@@ -63,38 +63,36 @@ __device__ __forceinline__ void trsm_cp_async_wait() { asm volatile("cp.async.wa
 // block (bi, bj), bj <= bi, of the tile's lower triangle; element (r, k) of a block at [r * 32 + k]
 __device__ __forceinline__ int trsm_block(int bi, int bj) { return (bi * (bi + 1) / 2 + bj) * TRSM_BLK; }
 
-// One warp:  xdst[0..4R)[0..32)  -=  Lrows[0..4R)[0..32) . xsrc[0..32)[0..32)
-// (Lrows: 4R consecutive rows of one 32 x 32 block; xsrc: the 32 solved rows; xdst: the 4R rows to update).
-// Each lane owns an R x 4 patch (rows R*(lane/8).., columns 4*(lane%8)..): the eight lanes that share a row group read
-// the same address of L (broadcast), the eight column groups read one contiguous 128-byte row of x.
-template <int R>
+// One warp:  xdst[0..ROWS)[0..32)  -=  Lrows[0..ROWS)[0..32) . xsrc[0..32)[0..32)
+// (Lrows: ROWS consecutive rows of one 32 x 32 block; xsrc: the 32 solved rows; xdst: the ROWS rows to update).
+// Lane = column: a lane keeps its column of x in registers and walks down the rows; the entries of L are the same
+// address in every lane (one 16-byte broadcast per four values of k), so a multiply-add costs a quarter of the
+// shared-memory traffic of a register patch per lane, and every access of x is a conflict-free row.
+template <int ROWS>
 __device__ __forceinline__ void trsm_apply(const float* __restrict__ lrows, float (*xsrc)[TRSM_CW], float (*xdst)[TRSM_CW], int lane) {
-    const int tr = lane >> 3, tc = lane & 7;
-    float acc[R][4] = {};
-#pragma unroll 2
-    for (int k = 0; k < TRSM_SB; k += 4) {
-        float4 xv[4];
+    float xr[TRSM_SB];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) xv[j] = *reinterpret_cast<const float4*>(&xsrc[k + j][4 * tc]);
+    for (int k = 0; k < TRSM_SB; ++k) xr[k] = xsrc[k][lane];
+    static_assert(ROWS % 4 == 0, "rows are taken four at a time");
+#pragma unroll 1
+    for (int i = 0; i < ROWS; i += 4) {   // four rows at a time: four independent chains of multiply-adds
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int i = 0; i < R; ++i) {
-            const float4 l = *reinterpret_cast<const float4*>(lrows + (R * tr + i) * TRSM_SB + k);
-            acc[i][0] = fmaf(l.x, xv[0].x, acc[i][0]); acc[i][1] = fmaf(l.x, xv[0].y, acc[i][1]);
-            acc[i][2] = fmaf(l.x, xv[0].z, acc[i][2]); acc[i][3] = fmaf(l.x, xv[0].w, acc[i][3]);
-            acc[i][0] = fmaf(l.y, xv[1].x, acc[i][0]); acc[i][1] = fmaf(l.y, xv[1].y, acc[i][1]);
-            acc[i][2] = fmaf(l.y, xv[1].z, acc[i][2]); acc[i][3] = fmaf(l.y, xv[1].w, acc[i][3]);
-            acc[i][0] = fmaf(l.z, xv[2].x, acc[i][0]); acc[i][1] = fmaf(l.z, xv[2].y, acc[i][1]);
-            acc[i][2] = fmaf(l.z, xv[2].z, acc[i][2]); acc[i][3] = fmaf(l.z, xv[2].w, acc[i][3]);
-            acc[i][0] = fmaf(l.w, xv[3].x, acc[i][0]); acc[i][1] = fmaf(l.w, xv[3].y, acc[i][1]);
-            acc[i][2] = fmaf(l.w, xv[3].z, acc[i][2]); acc[i][3] = fmaf(l.w, xv[3].w, acc[i][3]);
+        for (int k = 0; k < TRSM_SB; k += 4) {
+            float4 l[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) l[r] = *reinterpret_cast<const float4*>(lrows + (i + r) * TRSM_SB + k);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc[r] = fmaf(l[r].x, xr[k], acc[r]);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc[r] = fmaf(l[r].y, xr[k + 1], acc[r]);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc[r] = fmaf(l[r].z, xr[k + 2], acc[r]);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc[r] = fmaf(l[r].w, xr[k + 3], acc[r]);
         }
-    }
 #pragma unroll
-    for (int i = 0; i < R; ++i) {
-        float4* dst = reinterpret_cast<float4*>(&xdst[R * tr + i][4 * tc]);
-        float4 cur = *dst;
-        cur.x -= acc[i][0]; cur.y -= acc[i][1]; cur.z -= acc[i][2]; cur.w -= acc[i][3];
-        *dst = cur;
+        for (int r = 0; r < 4; ++r) xdst[i + r][lane] -= acc[r];
     }
 }
 
@@ -267,17 +265,16 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
             const int tasks = (nsb - s - 1) * (TRSM_SB / 16);
             for (int g = warp - 4; g < tasks; g += 12) {
                 const int t = s0 + TRSM_SB + 16 * g;  // first tile row of the task
-                trsm_apply<4>(Lb + trsm_block(t >> 5, s - 1) + (t & 31) * TRSM_SB, &Xs[s0 - TRSM_SB], &Xs[t], lane);
+                trsm_apply<16>(Lb + trsm_block(t >> 5, s - 1) + (t & 31) * TRSM_SB, &Xs[s0 - TRSM_SB], &Xs[t], lane);
             }
         }
         if (s + 1 < nsb) trsm_wait_pending(nsb - 2 - s);  // column block s+1
         __syncthreads();  // x of sub-block s final; rows below it carry every update up to x of s-1
         if (s + 1 < nsb) {
-            // ---- next(s+1): the 32 rows of the next sub-block with x of sub-block s (warps 1 and 2, sixteen rows each:
-            // every warp that takes part reads all of x, so few warps with large patches cost the least shared-memory
-            // bandwidth); its triangle is prepared by warps 8-15 meanwhile
-            if (warp == 1 || warp == 2)
-                trsm_apply<4>(Lb + trsm_block(s + 1, s) + (16 * (warp - 1)) * TRSM_SB, &Xs[s0], &Xs[s0 + TRSM_SB + 16 * (warp - 1)], lane);
+            // ---- next(s+1): the 32 rows of the next sub-block with x of sub-block s (warps 0-7, four rows each: this
+            // ---- step is on the critical path, so it is spread thin); its triangle is prepared by warps 8-15 meanwhile
+            if (warp < TRSM_WARPS / 2)
+                trsm_apply<4>(Lb + trsm_block(s + 1, s) + (4 * warp) * TRSM_SB, &Xs[s0], &Xs[s0 + TRSM_SB + 4 * warp], lane);
             build_lt(s + 1);
             __syncthreads();
         }
