@@ -79,6 +79,30 @@ def test_exact_and_closed_form_cases():
     assert (a == b).all()
 
 
+def test_sliced_tail_is_reproducible_and_per_stream():
+    """Units cut by key range and folded by whichever part arrives last: the same bits every time, on any stream (each
+    stream has its own scratch), and from two streams at once."""
+    import torch
+    from paper_2511_09987_b200 import binding
+    w = AW("parts", 3, 300, 900, 64, seed=54)   # 6 units, 8 key tiles: 4 parts each
+    Q, K, V = inputs.make_attention_operands(w)
+    first = gpu_attention(Q, K, V)
+    for _ in range(5):
+        assert (gpu_attention(Q, K, V) == first).all()
+    dQ, dK, dV = (torch.from_numpy(np.ascontiguousarray(x)).view(torch.bfloat16).cuda() for x in (Q, K, V))
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = []
+    for rep in range(4):
+        for st in (s1, s2):
+            with torch.cuda.stream(st):
+                outs.append(binding.flash_attention(dQ, dK, dV))
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == binding.CYC_OK
+    for o in outs:
+        assert (o.cpu().numpy() == first).all()
+
+
 def test_full_size_every_query_row():
     """a2 at full size: every query row of every problem (all 32 x 4096 x 128 outputs) against the oracle."""
     import os
