@@ -24,6 +24,21 @@ struct TrsmPlan {
     cudaStream_t st;
 };
 
+// One launch of the diagonal-space kernel over `columns` right-hand-side columns: 32 columns per CTA, or 8 when 32 would
+// occupy at most a quarter of the SMs (the CTA's chain of dependent steps is as long either way, its arithmetic is not).
+static cudaError_t launch_trsm_diag(const TrsmDiagParams& p, long long columns, cudaStream_t st) {
+    DeviceInfo di;
+    const bool narrow = device_info(&di) == CYC_OK && 4 * ((columns + TRSM_CW - 1) / TRSM_CW) <= di.sms;
+    if (narrow)
+        return launch_pdl(trsm_diag_kernel<TRSM_CW_NARROW>, static_cast<unsigned>((columns + TRSM_CW_NARROW - 1) / TRSM_CW_NARROW), TRSM_THREADS,
+                          TRSM_SMEM_BYTES, st, p);
+    return launch_pdl(trsm_diag_kernel<TRSM_CW>, static_cast<unsigned>((columns + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, st, p);
+}
+static int trsm_diag_smem() {
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel<TRSM_CW>), TRSM_SMEM_BYTES)) return rc_;
+    return ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel<TRSM_CW_NARROW>), TRSM_SMEM_BYTES);
+}
+
 static int trsm_diag(const TrsmPlan& t, long long b, unsigned mask) {
     TrsmDiagParams p;
     p.L = t.L;
@@ -35,8 +50,7 @@ static int trsm_diag(const TrsmPlan& t, long long b, unsigned mask) {
     p.r0 = static_cast<int>(b * t.T);
     p.rows = static_cast<int>(t.n - b * t.T < t.T ? t.n - b * t.T : t.T);
     p.mask = mask;
-    const long long blocks = (t.m + TRSM_CW - 1) / TRSM_CW;
-    CYC_CUDA(launch_pdl(trsm_diag_kernel, static_cast<unsigned>(blocks), TRSM_THREADS, TRSM_SMEM_BYTES, t.st, p));
+    CYC_CUDA(launch_trsm_diag(p, t.m, t.st));
     g_launches.fetch_add(1);
     return CYC_OK;
 }
@@ -77,7 +91,7 @@ extern "C" int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, con
     const long long nb = (n + t.T - 1) / t.T;
     int levels = 0;
     while ((1ll << levels) < nb) ++levels;
-    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel), TRSM_SMEM_BYTES)) return rc_;
+    if (int rc_ = trsm_diag_smem()) return rc_;
     if (levels) {
         cudaMemPool_t pool;
         int rc = workspace_pool(&pool);
@@ -188,7 +202,7 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
     const bool in_place = a0 == l0;
     const long long panels = (n + T - 1) / T;
     if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(chol_diag_kernel), CHOL_SMEM_BYTES)) return rc_;
-    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(trsm_diag_kernel), TRSM_SMEM_BYTES)) return rc_;
+    if (int rc_ = trsm_diag_smem()) return rc_;
     CholAux* aux = nullptr;
     if (int rc_ = chol_aux(&aux, static_cast<size_t>(3 * panels + 2))) return rc_;
     std::lock_guard<std::mutex> aux_lock(aux->mu);
@@ -224,7 +238,7 @@ extern "C" int cyc_cholesky(int64_t n, int64_t tile, int dtype, const void* A, v
         p.n = static_cast<int>(n); p.m = static_cast<int>(r1 - r0);
         p.r0 = static_cast<int>(c0); p.rows = static_cast<int>(w);
         p.mask = have_w ? 1u : 0u;
-        if (ok(launch_pdl(trsm_diag_kernel, static_cast<unsigned>((r1 - r0 + TRSM_CW - 1) / TRSM_CW), TRSM_THREADS, TRSM_SMEM_BYTES, s, p), "trsm_diag_kernel"))
+        if (ok(launch_trsm_diag(p, r1 - r0, s), "trsm_diag_kernel"))
             g_launches.fetch_add(1);
     };
 

@@ -7,7 +7,7 @@
 // accumulator reaches this kernel as up to 32 partial-sum planes W_l (one per level of the recursive split of the
 // block rows), summed here in increasing l.
 //
-// One CTA solves one diagonal tile (rows <= 256) for 32 right-hand-side columns; lane = column, so every shared-memory
+// One CTA solves one diagonal tile (rows <= 256) for 32 right-hand-side columns (8 when the columns are few); lane = column, so every shared-memory
 // access of the right-hand side is conflict-free and every global access of B, W, X is a 128-byte row segment.
 // The lower triangle of the tile is brought into shared memory once, as 32 x 32 blocks (cp.async; 144 KB for a full
 // tile).  The tile is then processed in sub-blocks of 32 rows, with one step of look-ahead so that the sequential part
@@ -40,12 +40,12 @@ struct TrsmDiagParams {
     unsigned mask;    // bit l set: plane l holds a partial sum for these rows
 };
 
-constexpr int TRSM_T_MAX = 256, TRSM_CW = 32, TRSM_SB = 32, TRSM_THREADS = 512, TRSM_WARPS = TRSM_THREADS / 32;
+constexpr int TRSM_T_MAX = 256, TRSM_CW = 32, TRSM_CW_NARROW = 8, TRSM_SB = 32, TRSM_THREADS = 512, TRSM_WARPS = TRSM_THREADS / 32;
 constexpr int TRSM_NSB = TRSM_T_MAX / TRSM_SB;            // sub-blocks per tile
 constexpr int TRSM_BLK = TRSM_SB * TRSM_SB;               // floats per 32 x 32 block of L
 constexpr int TRSM_NBLK = TRSM_NSB * (TRSM_NSB + 1) / 2;  // blocks on and below the diagonal
 constexpr int TRSM_LT_PITCH = TRSM_SB + 4;
-constexpr int TRSM_SMEM_BYTES =
+constexpr int TRSM_SMEM_BYTES =   // sized for the wider form
     (TRSM_T_MAX * TRSM_CW + TRSM_NBLK * TRSM_BLK + TRSM_SB * TRSM_LT_PITCH + TRSM_SB) * static_cast<int>(sizeof(float));
 
 __device__ __forceinline__ void trsm_cp_async4(float* dst_smem, const float* src) {
@@ -63,25 +63,28 @@ __device__ __forceinline__ void trsm_cp_async_wait() { asm volatile("cp.async.wa
 // block (bi, bj), bj <= bi, of the tile's lower triangle; element (r, k) of a block at [r * 32 + k]
 __device__ __forceinline__ int trsm_block(int bi, int bj) { return (bi * (bi + 1) / 2 + bj) * TRSM_BLK; }
 
-// One warp:  xdst[0..ROWS)[0..32)  -=  Lrows[0..ROWS)[0..32) . xsrc[0..32)[0..32)
+// One warp:  xdst[0..ROWS)[0..CW)  -=  Lrows[0..ROWS)[0..32) . xsrc[0..32)[0..CW)
 // (Lrows: ROWS consecutive rows of one 32 x 32 block; xsrc: the 32 solved rows; xdst: the ROWS rows to update).
-// Lane = column: a lane keeps its column of x in registers and walks down the rows; the entries of L are the same
-// address in every lane (one 16-byte broadcast per four values of k), so a multiply-add costs a quarter of the
-// shared-memory traffic of a register patch per lane, and every access of x is a conflict-free row.
-template <int ROWS>
-__device__ __forceinline__ void trsm_apply(const float* __restrict__ lrows, float (*xsrc)[TRSM_CW], float (*xdst)[TRSM_CW], int lane) {
+// A lane owns one column: it keeps its column of x in registers and walks down rows; with CW = 32 a lane takes every
+// row, with CW = 8 the four lanes of a column take every fourth row each.  The entries of L are the same address in all
+// lanes of a row group (one 16-byte broadcast per four values of k), so a multiply-add costs a quarter of the
+// shared-memory traffic of a register patch per lane, and every access of x is conflict-free.
+template <int ROWS, int CW>
+__device__ __forceinline__ void trsm_apply(const float* __restrict__ lrows, float (*xsrc)[CW], float (*xdst)[CW], int lane) {
+    constexpr int G = 32 / CW;   // row groups per warp
+    static_assert(ROWS % (4 * G) == 0, "a lane takes its rows four at a time");
+    const int col = lane % CW, g = lane / CW;
     float xr[TRSM_SB];
 #pragma unroll
-    for (int k = 0; k < TRSM_SB; ++k) xr[k] = xsrc[k][lane];
-    static_assert(ROWS % 4 == 0, "rows are taken four at a time");
+    for (int k = 0; k < TRSM_SB; ++k) xr[k] = xsrc[k][col];
 #pragma unroll 1
-    for (int i = 0; i < ROWS; i += 4) {   // four rows at a time: four independent chains of multiply-adds
+    for (int i = 0; i < ROWS; i += 4 * G) {   // four rows per lane at a time: four independent chains of multiply-adds
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int k = 0; k < TRSM_SB; k += 4) {
             float4 l[4];
 #pragma unroll
-            for (int r = 0; r < 4; ++r) l[r] = *reinterpret_cast<const float4*>(lrows + (i + r) * TRSM_SB + k);
+            for (int r = 0; r < 4; ++r) l[r] = *reinterpret_cast<const float4*>(lrows + (i + g + G * r) * TRSM_SB + k);
 #pragma unroll
             for (int r = 0; r < 4; ++r) acc[r] = fmaf(l[r].x, xr[k], acc[r]);
 #pragma unroll
@@ -92,7 +95,7 @@ __device__ __forceinline__ void trsm_apply(const float* __restrict__ lrows, floa
             for (int r = 0; r < 4; ++r) acc[r] = fmaf(l[r].w, xr[k + 3], acc[r]);
         }
 #pragma unroll
-        for (int r = 0; r < 4; ++r) xdst[i + r][lane] -= acc[r];
+        for (int r = 0; r < 4; ++r) xdst[i + g + G * r][col] -= acc[r];
     }
 }
 
@@ -110,10 +113,15 @@ __device__ __forceinline__ void trsm_wait_pending(int pending) {
     }
 }
 
+// CW = right-hand-side columns per CTA: 32, or 8 when there are so few columns that 32 per CTA would leave most SMs idle
+// (a CTA's arithmetic shrinks with CW, its chain of dependent steps does not, so narrow CTAs pay only then).
+template <int CW>
 __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDiagParams p) {
+    static_assert(CW == 32 || CW == 8, "32 or 8 columns per CTA");
+    constexpr int G = 32 / CW;   // lanes per column in the updates and in the load of the right-hand side
     extern __shared__ __align__(16) float trsm_smem[];
-    float(*Xs)[TRSM_CW] = reinterpret_cast<float(*)[TRSM_CW]>(trsm_smem);  // right-hand side, then X
-    float* Lb = trsm_smem + TRSM_T_MAX * TRSM_CW;                          // the blocks of L
+    float(*Xs)[CW] = reinterpret_cast<float(*)[CW]>(trsm_smem);  // right-hand side, then X
+    float* Lb = trsm_smem + TRSM_T_MAX * CW;                     // the blocks of L
     float(*Lt)[TRSM_LT_PITCH] = reinterpret_cast<float(*)[TRSM_LT_PITCH]>(Lb + TRSM_NBLK * TRSM_BLK);
     float* dinv = reinterpret_cast<float*>(Lt) + TRSM_SB * TRSM_LT_PITCH;
 
@@ -121,7 +129,7 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
     ptx::grid_launch_dependents();
     ptx::grid_dependency_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int c = blockIdx.x * TRSM_CW + lane;
+    const int c = blockIdx.x * CW + lane % CW;   // this lane's column in the load of the right-hand side
     const bool col_ok = c < p.m;
     const int nsb = (p.rows + TRSM_SB - 1) / TRSM_SB;
 
@@ -149,16 +157,17 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
         trsm_cp_async_commit();
     }
 
-    // right-hand side of the tile: B_ii - Xa, Xa = the partial-sum planes in increasing level.  A thread holds its
-    // sixteen rows (one column) at once, so that the loads of a whole plane -- two planes at a time -- are in flight
+    // right-hand side of the tile: B_ii - Xa, Xa = the partial-sum planes in increasing level.  A thread holds all its
+    // rows (of one column) at once, so that the loads of a whole plane -- two planes at a time -- are in flight
     // together: the planes come from DRAM, and this prologue is all latency.
     {
-        constexpr int RPT = TRSM_T_MAX / TRSM_WARPS;  // rows per thread
+        constexpr int RPT = TRSM_T_MAX / (TRSM_WARPS * G);  // rows per thread: row (TRSM_WARPS * i + warp) * G + lane / CW
+        const int rsub = warp * G + lane / CW;
         float v[RPT], xa[RPT];
         unsigned okm = 0;
 #pragma unroll
         for (int i = 0; i < RPT; ++i) {
-            const int r = TRSM_WARPS * i + warp;
+            const int r = TRSM_WARPS * G * i + rsub;
             const bool ok = r < p.rows && col_ok;
             okm |= static_cast<unsigned>(ok) << i;
             v[i] = ok ? __ldg(p.B + r * p.b_r + c * p.b_c) : 0.f;
@@ -177,7 +186,7 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
 #pragma unroll
             for (int i = 0; i < RPT; ++i) {
                 const bool ok = (okm >> i) & 1u;
-                const long long at = (TRSM_WARPS * i + warp) * p.w_r;
+                const long long at = (TRSM_WARPS * G * i + rsub) * p.w_r;
                 w0[i] = ok ? __ldg(W0 + at) : 0.f;
                 w1[i] = (ok && l1 >= 0) ? __ldg(W1 + at) : 0.f;
             }
@@ -185,7 +194,7 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
             for (int i = 0; i < RPT; ++i) xa[i] = (xa[i] + w0[i]) + w1[i];
         }
 #pragma unroll
-        for (int i = 0; i < RPT; ++i) Xs[TRSM_WARPS * i + warp][lane] = v[i] - xa[i];
+        for (int i = 0; i < RPT; ++i) Xs[TRSM_WARPS * G * i + rsub][lane % CW] = v[i] - xa[i];
     }
 
     // Diagonal block s prepared for the column sweep: every row r scaled by 1 / L_rr (so that the sweep needs no
@@ -218,7 +227,7 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
 
     for (int s = 0; s < nsb; ++s) {
         const int s0 = s * TRSM_SB;
-        if (warp < 4) {
+        if (warp < CW / 8) {
             // ---- solve(s): x_r = (s_r - sum_{k<r} L_rk x_k) / L_rr evaluated as s_r/L_rr - sum_k (L_rk/L_rr) x_k.
             // ---- Four warps, one per scheduler, eight columns each; a column is shared by four lanes that hold eight
             // ---- consecutive rows each, so a step of the sweep is one shuffle (x_k from the lane that owns row k)
@@ -252,29 +261,31 @@ __global__ void __launch_bounds__(TRSM_THREADS, 1) trsm_diag_kernel(const TrsmDi
                 for (int i = 0; i < 8; ++i)
                     if (i > (k & 7) ? from : past) sv[i] = fmaf(-lv[i], xk, sv[i]);
             }
-            const int c = blockIdx.x * TRSM_CW + cl;
+            const int cx = blockIdx.x * CW + cl;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int r = s0 + 8 * q + i;
                 Xs[r][cl] = sv[i];
-                if (r < p.rows && c < p.m) p.X[r * p.x_r + c * p.x_c] = sv[i];
+                if (r < p.rows && cx < p.m) p.X[r * p.x_r + cx * p.x_c] = sv[i];
             }
-        } else if (s >= 1 && s + 1 < nsb) {
+        } else if (warp >= 4 && s >= 1 && s + 1 < nsb) {
             // ---- trailing(s): rows below sub-block s, sixteen per warp at a time, with x of sub-block s-1: the other
             // ---- twelve warps
             const int tasks = (nsb - s - 1) * (TRSM_SB / 16);
             for (int g = warp - 4; g < tasks; g += 12) {
                 const int t = s0 + TRSM_SB + 16 * g;  // first tile row of the task
-                trsm_apply<16>(Lb + trsm_block(t >> 5, s - 1) + (t & 31) * TRSM_SB, &Xs[s0 - TRSM_SB], &Xs[t], lane);
+                trsm_apply<16, CW>(Lb + trsm_block(t >> 5, s - 1) + (t & 31) * TRSM_SB, &Xs[s0 - TRSM_SB], &Xs[t], lane);
             }
         }
         if (s + 1 < nsb) trsm_wait_pending(nsb - 2 - s);  // column block s+1
         __syncthreads();  // x of sub-block s final; rows below it carry every update up to x of s-1
         if (s + 1 < nsb) {
-            // ---- next(s+1): the 32 rows of the next sub-block with x of sub-block s (warps 0-7, four rows each: this
-            // ---- step is on the critical path, so it is spread thin); its triangle is prepared by warps 8-15 meanwhile
-            if (warp < TRSM_WARPS / 2)
-                trsm_apply<4>(Lb + trsm_block(s + 1, s) + (4 * warp) * TRSM_SB, &Xs[s0], &Xs[s0 + TRSM_SB + 4 * warp], lane);
+            // ---- next(s+1): the 32 rows of the next sub-block with x of sub-block s (four rows per lane: eight warps with
+            // ---- 32 columns, two with 8 -- this step is on the critical path, so it is spread thin); its triangle is
+            // ---- prepared by warps 8-15 meanwhile
+            constexpr int NR = 4 * G;   // rows per warp: four per lane
+            if (warp < TRSM_SB / NR)
+                trsm_apply<NR, CW>(Lb + trsm_block(s + 1, s) + (NR * warp) * TRSM_SB, &Xs[s0], &Xs[s0 + TRSM_SB + NR * warp], lane);
             build_lt(s + 1);
             __syncthreads();
         }
