@@ -1034,6 +1034,7 @@ KERNEL_SOURCES = {
     "tcgen05_pair_tall": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "umma_pair_tall_kernel.cuh"],
     "tcgen05_pair_splitk": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "splitk_reduce_kernel.cuh"],
     "tcgen05_3xtf32": ["ptx.cuh", "umma_kernel.cuh", "umma_pair_kernel.cuh", "umma_pair_tf32x3_kernel.cuh"],
+    "tcgen05_3xtf32_ws": ["ptx.cuh", "umma_kernel.cuh", "umma_ws_tf32x3_kernel.cuh"],
     "scan": ["scan_kernel.cuh"],
     "fa2_d64": ["ptx.cuh", "umma_kernel.cuh", "fa2_kernel.cuh"],
     "fa2_d128": ["ptx.cuh", "umma_kernel.cuh", "fa2_kernel.cuh"],

@@ -299,7 +299,8 @@ int cyc_selftest_bounded_wait(void* stream, int64_t budget_cycles);
  * kernel), "tcgen05" (one CTA per tile), "tcgen05_pair" (CTA pair, 256x256 tiles),
  * "tcgen05_pair_tall" (CTA pair, 512x256 tiles), "tcgen05_pair_splitk" (few tiles, long k
  * loop: k-slices on different CTA pairs, partial sums added in slice order by a second kernel),
- * "tcgen05_3xtf32" (fp32 split into TF32 parts) -- or NULL if the arguments are invalid.
+ * "tcgen05_3xtf32" (fp32 split into TF32 parts), "tcgen05_3xtf32_ws" (the same with a small B
+ * kept in tensor memory while a long A streams past it) -- or NULL if the arguments are invalid.
  * Host only, makes no CUDA call. */
 const char* cyc_kernel_for(int64_t batch, int64_t M, int64_t N, int64_t K, int dtype, const void* A, const void* B,
                            const void* C, unsigned flags);

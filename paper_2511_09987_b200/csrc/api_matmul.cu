@@ -9,6 +9,7 @@
 #include "umma_pair_tall_kernel.cuh"
 #include "splitk_reduce_kernel.cuh"
 #include "umma_pair_tf32x3_kernel.cuh"
+#include "umma_ws_tf32x3_kernel.cuh"
 
 namespace cyc {
 
@@ -36,7 +37,7 @@ int validate(const Problem& q) {
     return CYC_OK;
 }
 
-enum Family { FAM_SIMT = 0, FAM_UMMA = 1, FAM_UMMA_3XTF32 = 2, FAM_UMMA_PAIR = 3, FAM_UMMA_TALL = 4, FAM_UMMA_SPLITK = 5 };
+enum Family { FAM_SIMT = 0, FAM_UMMA = 1, FAM_UMMA_3XTF32 = 2, FAM_UMMA_PAIR = 3, FAM_UMMA_TALL = 4, FAM_UMMA_SPLITK = 5, FAM_UMMA_3XTF32_WS = 6 };
 
 // the tensor-core kernels move tiles with TMA: 16-byte aligned bases and pitches
 static bool tma_ok(const Problem& q) {
@@ -76,6 +77,11 @@ static Family choose(const Problem& q) {
     if (q.dtype == CYC_F32) {
         // strict per-element k order, small or unaligned problems: the general kernel
         if ((q.flags & CYC_FLAG_FIXED_K_ORDER) || !tma_ok(q) || q.M <= 128 || q.N <= 128) return FAM_SIMT;
+        // a small B under a long A: B stays in tensor memory and A streams past it (weight-stationary form); worth its
+        // prologue from two 128-row tiles per CTA pair on
+        if (q.batch == 1 && !(q.flags & CYC_FLAG_B_COL_MAJOR) && q.N <= WS_NMAX && q.K <= WS_KMAX && q.M >= 2 * WS_ROWS * kCtaPairs &&
+            reinterpret_cast<uintptr_t>(q.C) % 16 == 0)
+            return FAM_UMMA_3XTF32_WS;
         return FAM_UMMA_3XTF32;
     }
     if (!tma_ok(q)) return FAM_SIMT;
@@ -357,6 +363,28 @@ static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
     return CYC_OK;
 }
 
+// weight-stationary form: B^T resident in tensor memory (hi) and shared memory (lo), A streamed in 128-row tiles
+static int launch_tf32x3_ws(const Problem& q, cudaStream_t st, int sms) {
+    CUtensorMap tmA, tmW, tmC;
+    int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, 1, lda_of(q), q.M * q.K, WS_BK, WS_HALF, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    rc = make_map(&tmW, q.dtype, q.B, q.N, q.K, 1, ldb_of(q), q.K * q.N, 32, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (rc) return rc;
+    rc = make_map(&tmC, q.dtype, q.C, q.N, q.M, 1, q.N, q.M * q.N, 32, 16, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (rc) return rc;
+    WsParams p;
+    p.C = static_cast<float*>(q.C);
+    p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
+    p.tiles = (q.M + WS_ROWS - 1) / WS_ROWS;
+    if (int rc_ = status_word(&p.status)) return rc_;
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(umma_ws_tf32x3_kernel), WS_SMEM_BYTES)) return rc_;
+    const long long max_pairs = sms / 2;
+    const long long pairs = p.tiles < max_pairs ? p.tiles : max_pairs;
+    CYC_CUDA(launch_pdl(umma_ws_tf32x3_kernel, static_cast<unsigned>(2 * pairs), WS_THREADS, WS_SMEM_BYTES, st, tmA, tmW, tmC, p));
+    g_launches.fetch_add(1);
+    return CYC_OK;
+}
+
 static int launch_tf32x3(const Problem& q, cudaStream_t st) {
     DeviceInfo di;
     int rc = device_info(&di);
@@ -365,6 +393,7 @@ static int launch_tf32x3(const Problem& q, cudaStream_t st) {
         snprintf(g_err, sizeof g_err, "tensor-core kernels need an sm_100 device");
         return CYC_ERR_UNSUPPORTED;
     }
+    if (choose(q) == FAM_UMMA_3XTF32_WS) return launch_tf32x3_ws(q, st, di.sms);
     return (q.flags & CYC_FLAG_B_COL_MAJOR) ? launch_tf32x3_cfg<false>(q, st, di.sms) : launch_tf32x3_cfg<true>(q, st, di.sms);
 }
 
@@ -397,6 +426,7 @@ static const char* family_name(Family f) {
         case FAM_UMMA_TALL: return "tcgen05_pair_tall";
         case FAM_UMMA_SPLITK: return "tcgen05_pair_splitk";
         case FAM_UMMA_3XTF32: return "tcgen05_3xtf32";
+        case FAM_UMMA_3XTF32_WS: return "tcgen05_3xtf32_ws";
         default: return "simt";
     }
 }
@@ -412,6 +442,7 @@ int route(const Problem& q, cudaStream_t st) {
         case FAM_UMMA_SPLITK:
             return q.dtype == CYC_BF16_F32 ? launch_umma<KIND_BF16>(q, st) : launch_umma<KIND_I8>(q, st);
         case FAM_UMMA_3XTF32:
+        case FAM_UMMA_3XTF32_WS:
             return launch_tf32x3(q, st);
         default:
             if (q.dtype == CYC_F32) return launch_simt<float, float>(q, st);

@@ -151,7 +151,11 @@ def test_kernel_selection(binding):
     assert k(1, 256, 256, 8192, "bf16") == "tcgen05_pair_splitk" # one tile, 128 k-blocks
     assert k(1, 256, 256, 8192, "bf16", fixed_k_order=True) == "tcgen05_pair"
     assert k(1, 256, 256, 512, "bf16") == "tcgen05_pair"         # k loop too short to cut
-    assert k(1, 65536, 256, 256, "f32") == "tcgen05_3xtf32"
+    assert k(1, 65536, 256, 256, "f32") == "tcgen05_3xtf32_ws"   # small B under a long A: B stays in tensor memory
+    assert k(1, 65536, 256, 256, "f32", b_col_major=True) == "tcgen05_3xtf32"
+    assert k(1, 65536, 256, 512, "f32") == "tcgen05_3xtf32"      # B too large to stay
+    assert k(1, 4096, 256, 256, "f32") == "tcgen05_3xtf32"       # too few rows to pay for the prologue
+    assert k(4, 65536, 256, 256, "f32") == "tcgen05_3xtf32"
     assert k(1, 65536, 256, 256, "f32", fixed_k_order=True) == "simt"
     assert k(1, 128, 256, 256, "f32") == "simt"
     assert k(1, 65, 127, 33, "bf16") == "simt"               # pitches not multiples of 16 bytes

@@ -89,6 +89,35 @@ def test_fp32_split_tf32_on_tensor_cores(shape, col):
     assert worst < 2e-6                # the split leaves about 2^-21 per product
 
 
+@pytest.mark.parametrize("shape", [(18944, 256, 256), (20001, 256, 256), (19000, 200, 256), (19500, 132, 100), (18944, 256, 32),
+                                   (30000, 252, 36)])
+def test_fp32_weight_stationary_on_tensor_cores(shape):
+    """Small B under a long A: B^T split once and kept in tensor memory / shared memory, A streamed in 128-row tiles
+    (ragged last tile, ragged n and k included)."""
+    w = wl("f32", *shape, seed=43, col=False, fixed=False)
+    assert family(w) == "tcgen05_3xtf32_ws"
+    worst = check_workload(w, rows_per_problem=600)
+    assert worst < 2e-6
+
+
+def test_fp32_weight_stationary_closed_forms():
+    import torch
+    from paper_2511_09987_b200 import binding
+    M, n = 19200, 256
+    assert binding.kernel_for(1, M, n, n, "f32") == "tcgen05_3xtf32_ws"
+    X = (torch.randn(M, n, device="cuda") * 3).float()
+    I = torch.eye(n, device="cuda")
+    out = binding.recurrence_matmul(X, I)                      # B = I returns A to within 2^-21 relative
+    assert (out - X).abs().max().item() <= 2.0 ** -21 * X.abs().max().item()
+    Xi = torch.randint(-1000, 1000, (M, n), device="cuda").float()      # 11-bit integers: hi part exact, lo zero
+    assert torch.equal(binding.recurrence_matmul(Xi, I), Xi)
+    P = torch.eye(n, device="cuda")[torch.randperm(n, device="cuda")]   # a permutation of the columns, exactly
+    assert torch.equal(binding.recurrence_matmul(Xi, P), Xi @ P)
+    ones = torch.ones((M, n), device="cuda")
+    assert (binding.recurrence_matmul(ones, torch.ones((n, n), device="cuda")) == n).all().item()
+    assert binding.last_device_status() == binding.CYC_OK
+
+
 def test_fp32_split_closed_forms():
     import torch
     from paper_2511_09987_b200 import binding
