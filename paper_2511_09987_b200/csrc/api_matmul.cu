@@ -368,7 +368,7 @@ static int launch_tf32x3_ws(const Problem& q, cudaStream_t st, int sms) {
     CUtensorMap tmA, tmW, tmC;
     int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, 1, lda_of(q), q.M * q.K, WS_BK, WS_HALF, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    rc = make_map(&tmW, q.dtype, q.B, q.N, q.K, 1, ldb_of(q), q.K * q.N, 32, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+    rc = make_map(&tmW, q.dtype, q.B, q.N, q.K, 1, ldb_of(q), q.K * q.N, 32, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc) return rc;
     rc = make_map(&tmC, q.dtype, q.C, q.N, q.M, 1, q.N, q.M * q.N, 32, 16, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc) return rc;

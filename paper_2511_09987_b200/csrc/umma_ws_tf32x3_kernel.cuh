@@ -18,8 +18,8 @@
 // two such buffers in turn.  (Plain stores from registers, 128 bytes per instruction, were measured at 67 clocks per
 // instruction and made the export the longest path of the kernel.)
 //
-// Roles per CTA (320 threads): warp 0 TMA producer, warp 1 MMA issuer (leader CTA), warps 2-5 first split B^T (thread =
-// row n = TMEM lane), then export; warps 6-9 split the A stages.  Every wait is bounded.
+// Roles per CTA (320 threads): warp 0 TMA producer, warp 1 MMA issuer (leader CTA), warps 2-9 first split B^T (thread =
+// row n = TMEM lane); then warps 2-5 export and warps 6-9 split the A stages.  Every wait is bounded.
 #pragma once
 #include "umma_kernel.cuh"
 
@@ -34,8 +34,8 @@ constexpr int WS_STAGE_RAW = WS_HALF * WS_BK * 4;  // 8 KB: this CTA's 64 rows x
 constexpr int WS_STAGE_BYTES = 2 * WS_STAGE_RAW;   // followed by their lo parts
 constexpr int WS_STAGES = 5;
 constexpr int WS_WLO_BYTES = (WS_KMAX / WS_BK) * 128 * 128;  // 8 slabs of 128 rows (n) x 128 B: 128 KB
-constexpr int WS_TEMP_BYTES = 4 * 128 * 128;                 // half of B^T's k range as landed: 4 boxes of 128 k x 32 n
-static_assert(WS_TEMP_BYTES <= WS_STAGES * WS_STAGE_BYTES, "the prologue borrows the ring");
+constexpr int WS_TEMP_BYTES = 4 * 64 * 128;                  // a quarter of B^T's k range as landed: 4 boxes of 64 k x 32 n
+static_assert(2 * WS_TEMP_BYTES <= WS_STAGES * WS_STAGE_BYTES, "the prologue borrows the ring for two such buffers");
 constexpr int WS_STAGING_BYTES = 4 * 2 * 16 * 128;           // per export warp two buffers of 16 rows x 128 B
 constexpr int WS_SMEM_BYTES = WS_WLO_BYTES + WS_STAGES * WS_STAGE_BYTES + WS_STAGING_BYTES + 1024 + 1024;
 
@@ -52,9 +52,9 @@ struct WsCtl {
     uint64_t empty[8];     // stage: MMAs done (both, by the leader's multicast commit)
     uint64_t acc_full[2];  // accumulator complete (both)
     uint64_t acc_empty[2]; // accumulator read out, both CTAs (leader)
-    uint64_t w_full;       // half of B^T landed in the borrowed ring (per CTA)
-    uint64_t w_free;       // ... and consumed (per CTA, 4 warps)
-    uint64_t w_ready;      // B^T split and in place, both CTAs (leader, 8 warps)
+    uint64_t w_full[2];    // a quarter of B^T landed in one of two buffers borrowed from the ring (per CTA)
+    uint64_t w_free[2];    // ... and consumed (per CTA, 8 warps)
+    uint64_t w_ready;      // B^T split and in place, both CTAs (leader, 16 warps)
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -107,7 +107,7 @@ __device__ __forceinline__ void ws_tmem_st_32x32(uint32_t taddr, const uint32_t 
 }
 __device__ __forceinline__ void ws_tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// tmA: A as [M][K] fp32, box 32 k x 64 rows, 128-byte swizzle.  tmW: B as [K][N] fp32, box 32 n x 128 k, no swizzle.
+// tmA: A as [M][K] fp32, box 32 k x 64 rows, 128-byte swizzle.  tmW: B as [K][N] fp32, box 32 n x 64 k, no swizzle.
 // tmC: C as [M][N] fp32, box 32 n x 16 rows, no swizzle.
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WS_THREADS, 1)
 umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
@@ -142,9 +142,11 @@ umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             ptx::mbar_init(&ctl->acc_full[a], 1);
             ptx::mbar_init(&ctl->acc_empty[a], 8);
         }
-        ptx::mbar_init(&ctl->w_full, 1);
-        ptx::mbar_init(&ctl->w_free, 4);
-        ptx::mbar_init(&ctl->w_ready, 8);
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(&ctl->w_full[b], 1);
+            ptx::mbar_init(&ctl->w_free[b], 8);
+        }
+        ptx::mbar_init(&ctl->w_ready, 16);
         ctl->abort = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmA);
@@ -162,20 +164,65 @@ umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
+    // B^T into place (warps 2-9, thread = row n of this CTA's half = TMEM lane): of every landed quarter (64 values of k) the
+    // warps 2-5 take the first 32, the warps 6-9 the second; hi parts to tensor memory, lo parts to shared memory in the
+    // K-major swizzled layout the MMA reads.
+    auto place_weights = [&](int part) -> bool {
+        const int q = warp & 3;                  // TMEM lane quarter this warp may access
+        const int n_loc = q * 32 + lane;
+        const uint32_t lane_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        for (int qi = 0; qi < 4; ++qi) {
+            const int b = qi & 1;
+            if (!ws_wait(&ctl->w_full[b], (qi >> 1) & 1, ctl, p.status, 8)) return false;
+            // landed: box c = n_loc / 32 holds 64 rows k (128 B each) of 32 columns n
+            const uint8_t* src = ring + b * WS_TEMP_BYTES + (n_loc >> 5) * (64 * 128) + (n_loc & 31) * 4 + part * 32 * 128;
+            const int k0 = qi * 64 + part * 32;
+            uint8_t* slab = w_lo + (k0 / WS_BK) * (128 * 128) + n_loc * 128;
+            uint32_t hi[32];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {    // 16-byte chunk c of the row: four values of k
+                uint32_t lo4[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t x = *reinterpret_cast<const uint32_t*>(src + (4 * c + e) * 128);
+                    hi[4 * c + e] = x & 0xFFFFE000u;
+                    lo4[e] = ws_lo(x);
+                }
+                *reinterpret_cast<uint4*>(slab + ((c ^ (n_loc & 7)) << 4)) = make_uint4(lo4[0], lo4[1], lo4[2], lo4[3]);
+            }
+            ws_tmem_st_32x32(lane_taddr + static_cast<uint32_t>(k0), hi);
+            ws_tmem_st_wait();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&ctl->w_free[b]);   // the borrowed buffer may be overwritten
+        }
+        ptx::fence_proxy_async_smem();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+            if (rank == 0) ptx::mbar_arrive(&ctl->w_ready);
+            else ptx::mbar_arrive_remote(&ctl->w_ready, 0);
+        }
+        return true;
+    };
+
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs, own barriers)
         if (lane == 0) {
             bool ok = true;
             ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; nothing it wrote is read before it ends
-            // B^T, this CTA's 128 columns n, in two halves of k through the (still idle) ring
-            for (int h = 0; h < 2 && ok; ++h) {
-                if (h == 1 && !ws_wait(&ctl->w_free, 0, ctl, p.status, 1)) { ok = false; break; }
-                ptx::mbar_arrive_expect_tx(&ctl->w_full, WS_TEMP_BYTES);
+            // B^T, this CTA's 128 columns n, in four quarters of k through two buffers in the (still idle) ring
+            int wq = 0;   // quarters requested
+            for (int qi = 0; qi < 4 && ok; ++qi) {
+                const int b = qi & 1;
+                if (qi >= 2 && !ws_wait(&ctl->w_free[b], 0, ctl, p.status, 1)) { ok = false; break; }
+                ++wq;
+                ptx::mbar_arrive_expect_tx(&ctl->w_full[b], WS_TEMP_BYTES);
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                    ptx::tma_load_3d(ring + c * (128 * 128), &tmW, &ctl->w_full, static_cast<int>(rank) * 128 + c * 32, h * 128, 0);
+                    ptx::tma_load_3d(ring + b * WS_TEMP_BYTES + c * (64 * 128), &tmW, &ctl->w_full[b], static_cast<int>(rank) * 128 + c * 32, qi * 64, 0);
             }
-            if (ok && !ws_wait(&ctl->w_free, 1, ctl, p.status, 2)) ok = false;   // the ring is the ring again
+            for (int b = 0; b < 2 && ok; ++b)   // the ring is the ring again
+                if (!ws_wait(&ctl->w_free[b], 1, ctl, p.status, 2)) ok = false;
             int stage = 0;
             uint32_t phase = 0;
             long long issued = 0;
@@ -191,7 +238,10 @@ umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             }
             if (!ok) {  // leave no copy in flight: wait (bounded) for what was issued
                 const long long t0 = clock64();
-                while (!ptx::mbar_try_wait(&ctl->w_full, 0) && clock64() - t0 < UMMA_WAIT_CYCLES) {}
+                for (int b = 0; b < 2; ++b) {
+                    const int uses = (wq + 1 - b) / 2;   // copies into buffer b
+                    while (uses > 0 && !ptx::mbar_try_wait(&ctl->w_full[b], (uses - 1) & 1) && clock64() - t0 < UMMA_WAIT_CYCLES) {}
+                }
                 const int back = issued < WS_STAGES ? static_cast<int>(issued) : WS_STAGES;
                 int s = stage;
                 uint32_t ph = phase;
@@ -247,11 +297,12 @@ umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
         __syncwarp();
     } else if (warp >= 6) {
-        // ------------------------------------------------------------ split warps: lo parts of the landed A stages
+        // ------------------------------------------------------------ split warps: their share of B^T, then the lo parts of
+        // ------------------------------------------------------------ the landed A stages
         const int tid = threadIdx.x - 6 * 32;   // 0 .. 127
         int stage = 0;
         uint32_t phase = 0;
-        bool ok = true;
+        bool ok = place_weights(1);
         for (long long tile = pair; ok && tile < p.tiles; tile += num_pairs) {
             for (int kb = 0; kb < num_kb; ++kb) {
                 if (!ws_wait(&ctl->full[stage], phase, ctl, p.status, 7)) { ok = false; break; }
@@ -272,45 +323,11 @@ umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             }
         }
     } else {
-        // ------------------------------------------------------------ warps 2-5: B^T into place, then the export
+        // ------------------------------------------------------------ warps 2-5: their share of B^T, then the export
         const int q = warp & 3;                  // TMEM lane quarter this warp may access
         const int n_loc = q * 32 + lane;         // row of B^T in this CTA = TMEM lane
         const uint32_t lane_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-        bool ok = true;
-        for (int h = 0; h < 2 && ok; ++h) {
-            if (!ws_wait(&ctl->w_full, h, ctl, p.status, 8)) { ok = false; break; }
-            // landed: box c = n_loc / 32 holds rows k (128 B each) of 32 columns n
-            const uint8_t* src = ring + (n_loc >> 5) * (128 * 128) + (n_loc & 31) * 4;
-#pragma unroll 1
-            for (int kk = 0; kk < 128; kk += 32) {
-                uint32_t hi[32];
-                uint8_t* slab = w_lo + ((h * 128 + kk) / WS_BK) * (128 * 128) + n_loc * 128;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {    // 16-byte chunk c of the row: four values of k
-                    uint32_t lo4[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const uint32_t x = *reinterpret_cast<const uint32_t*>(src + (kk + 4 * c + e) * 128);
-                        hi[4 * c + e] = x & 0xFFFFE000u;
-                        lo4[e] = ws_lo(x);
-                    }
-                    *reinterpret_cast<uint4*>(slab + ((c ^ (n_loc & 7)) << 4)) = make_uint4(lo4[0], lo4[1], lo4[2], lo4[3]);
-                }
-                ws_tmem_st_32x32(lane_taddr + static_cast<uint32_t>(h * 128 + kk), hi);
-            }
-            ws_tmem_st_wait();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&ctl->w_free);   // the borrowed ring may be overwritten
-        }
-        if (ok) {
-            ptx::fence_proxy_async_smem();
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (rank == 0) ptx::mbar_arrive(&ctl->w_ready);
-                else ptx::mbar_arrive_remote(&ctl->w_ready, 0);
-            }
-        }
+        bool ok = place_weights(0);
         // ---- export: C[row][n] <- accumulator (lane = n, column = row of the tile)
         const int n0 = static_cast<int>(rank) * 128 + q * 32;   // this warp's 32 columns of C
         uint8_t* my_stage = staging + (warp - 2) * (2 * 16 * 128);
