@@ -1,4 +1,4 @@
-// Weight-stationary form of the fp32 recurrence on tensor cores, for a small B (K <= 256, 128 < N <= 256) under a long A:
+// Weight-stationary form of the fp32 recurrence on tensor cores, for a small B (K <= 256, N <= 256) under a long A:
 // the shape the paper's weight-stationary program is written for -- the weights stay in the array, the other operand
 // streams past them (Section "Space-time Mappings of Dataflow Recurrences").
 //

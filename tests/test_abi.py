@@ -156,6 +156,10 @@ def test_kernel_selection(binding):
     assert k(1, 65536, 256, 512, "f32") == "tcgen05_3xtf32"      # B too large to stay
     assert k(1, 4096, 256, 256, "f32") == "tcgen05_3xtf32"       # too few rows to pay for the prologue
     assert k(4, 65536, 256, 256, "f32") == "tcgen05_3xtf32"
+    assert k(1, 65536, 64, 256, "f32") == "tcgen05_3xtf32_ws"    # fewer columns than a CTA pair's tile: still the tensor cores
+    assert k(1, 65536, 8, 256, "f32") == "tcgen05_3xtf32_ws"
+    assert k(1, 65536, 62, 256, "f32") == "simt"                 # row pitch of B and C not a multiple of 16 bytes
+    assert k(1, 65536, 128, 512, "f32") == "simt"
     assert k(1, 65536, 256, 256, "f32", fixed_k_order=True) == "simt"
     assert k(1, 128, 256, 256, "f32") == "simt"
     assert k(1, 65, 127, 33, "bf16") == "simt"               # pitches not multiples of 16 bytes
