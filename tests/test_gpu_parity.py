@@ -118,6 +118,31 @@ def test_fp32_weight_stationary_closed_forms():
     assert binding.last_device_status() == binding.CYC_OK
 
 
+def test_fp32_weight_stationary_non_finite_values_stay_in_their_rows_and_columns():
+    import torch
+    from paper_2511_09987_b200 import binding
+    M, n, k = 19072, 256, 256
+    g = torch.Generator(device="cuda").manual_seed(5)
+    A = torch.rand((M, k), device="cuda", generator=g) + 0.5          # positive: no 0 * inf
+    B = torch.rand((k, n), device="cuda", generator=g) + 0.5
+    A[5, 7] = float("inf"); A[9000, 3] = float("nan"); A[M - 1, k - 1] = float("-inf")
+    B[17, 200] = float("inf")
+    assert binding.kernel_for(1, M, n, k, "f32") == "tcgen05_3xtf32_ws"
+    C = binding.recurrence_matmul(A, B)
+    ref = A.double() @ B.double()
+    # Where the exact result is not finite the split arithmetic may give inf or NaN (an infinite hi part meets a lo part
+    # that happens to be exactly zero): what must hold is that every such entry is non-finite, every other entry is
+    # finite and as accurate as ever, and a row of infinities has the right sign where the exact result has one.
+    fin = torch.isfinite(ref)
+    assert torch.equal(torch.isfinite(C), fin)
+    assert (fin.sum(dim=1) == 0).sum().item() == 3 and (fin.sum(dim=0) == 0).sum().item() == 1   # three rows, one column
+    assert ((C.double() - ref).abs()[fin] <= 1e-5 * (A.double().abs() @ B.double().abs())[fin]).all().item()
+    both_inf = torch.isinf(C) & torch.isinf(ref)
+    assert torch.equal(torch.sign(C[both_inf]).double(), torch.sign(ref[both_inf]))
+    assert torch.isnan(C[9000]).all().item()
+    assert binding.last_device_status() == binding.CYC_OK
+
+
 def test_fp32_split_closed_forms():
     import torch
     from paper_2511_09987_b200 import binding
