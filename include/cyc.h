@@ -45,7 +45,10 @@
  *                 even): bit-reproducible.  Without the flag the library may
  *                 evaluate the sum on tensor cores with each operand split
  *                 into two TF32 parts and fp32 accumulation (error well inside
- *                 1e-5 * sum_k |A_ik||B_kj|).
+ *                 1e-5 * sum_k |A_ik||B_kj|).  Infinite or NaN inputs make exactly
+ *                 the C_ij they reach non-finite, but an infinite C_ij may come out
+ *                 as NaN (an infinite part of one operand meeting a part of the
+ *                 other that is exactly zero); the flag gives IEEE results.
  *   CYC_BF16_F32  A, B bfloat16; products exact; fp32 accumulation; C float.
  *                 k-blocks are accumulated in increasing order; results are
  *                 run-to-run identical with or without the flag (no atomics).
