@@ -81,7 +81,7 @@ static Family choose(const Problem& q) {
         // prologue from two 128-row tiles per CTA pair on.  It always does the work of 256 columns, and is still the
         // faster one for any narrower B (65536 x 64 x 256: 34 us against 119 us on the general kernel, whose tiles are 128
         // columns wide whatever N is).
-        if (q.batch == 1 && !(q.flags & CYC_FLAG_B_COL_MAJOR) && q.N <= WS_NMAX && q.K <= WS_KMAX && q.M >= 2 * WS_ROWS * kCtaPairs &&
+        if (q.batch == 1 && q.N <= WS_NMAX && q.K <= WS_KMAX && q.M >= 2 * WS_ROWS * kCtaPairs &&
             reinterpret_cast<uintptr_t>(q.C) % 16 == 0)
             return FAM_UMMA_3XTF32_WS;
         if (q.M <= 128 || q.N <= 128) return FAM_SIMT;   // too few rows or columns for a CTA pair
@@ -367,11 +367,13 @@ static int launch_tf32x3_cfg(const Problem& q, cudaStream_t st, int sms) {
 }
 
 // weight-stationary form: B^T resident in tensor memory (hi) and shared memory (lo), A streamed in 128-row tiles
+template <bool B_NK>
 static int launch_tf32x3_ws(const Problem& q, cudaStream_t st, int sms) {
     CUtensorMap tmA, tmW, tmC;
     int rc = make_map(&tmA, q.dtype, q.A, q.K, q.M, 1, lda_of(q), q.M * q.K, WS_BK, WS_HALF, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    rc = make_map(&tmW, q.dtype, q.B, q.N, q.K, 1, ldb_of(q), q.K * q.N, 32, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (B_NK) rc = make_map(&tmW, q.dtype, q.B, q.K, q.N, 1, ldb_of(q), q.K * q.N, WS_BK, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+    else rc = make_map(&tmW, q.dtype, q.B, q.N, q.K, 1, ldb_of(q), q.K * q.N, 32, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc) return rc;
     rc = make_map(&tmC, q.dtype, q.C, q.N, q.M, 1, q.N, q.M * q.N, 32, 16, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc) return rc;
@@ -380,10 +382,11 @@ static int launch_tf32x3_ws(const Problem& q, cudaStream_t st, int sms) {
     p.M = static_cast<int>(q.M); p.N = static_cast<int>(q.N); p.K = static_cast<int>(q.K);
     p.tiles = (q.M + WS_ROWS - 1) / WS_ROWS;
     if (int rc_ = status_word(&p.status)) return rc_;
-    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(umma_ws_tf32x3_kernel), WS_SMEM_BYTES)) return rc_;
+    auto kern = umma_ws_tf32x3_kernel<B_NK>;
+    if (int rc_ = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), WS_SMEM_BYTES)) return rc_;
     const long long max_pairs = sms / 2;
     const long long pairs = p.tiles < max_pairs ? p.tiles : max_pairs;
-    CYC_CUDA(launch_pdl(umma_ws_tf32x3_kernel, static_cast<unsigned>(2 * pairs), WS_THREADS, WS_SMEM_BYTES, st, tmA, tmW, tmC, p));
+    CYC_CUDA(launch_pdl(kern, static_cast<unsigned>(2 * pairs), WS_THREADS, WS_SMEM_BYTES, st, tmA, tmW, tmC, p));
     g_launches.fetch_add(1);
     return CYC_OK;
 }
@@ -396,7 +399,8 @@ static int launch_tf32x3(const Problem& q, cudaStream_t st) {
         snprintf(g_err, sizeof g_err, "tensor-core kernels need an sm_100 device");
         return CYC_ERR_UNSUPPORTED;
     }
-    if (choose(q) == FAM_UMMA_3XTF32_WS) return launch_tf32x3_ws(q, st, di.sms);
+    if (choose(q) == FAM_UMMA_3XTF32_WS)
+        return (q.flags & CYC_FLAG_B_COL_MAJOR) ? launch_tf32x3_ws<true>(q, st, di.sms) : launch_tf32x3_ws<false>(q, st, di.sms);
     return (q.flags & CYC_FLAG_B_COL_MAJOR) ? launch_tf32x3_cfg<false>(q, st, di.sms) : launch_tf32x3_cfg<true>(q, st, di.sms);
 }
 

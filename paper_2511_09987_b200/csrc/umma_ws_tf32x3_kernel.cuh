@@ -18,6 +18,9 @@
 // two such buffers in turn.  (Plain stores from registers, 128 bytes per instruction, were measured at 67 clocks per
 // instruction and made the export the longest path of the kernel.)
 //
+// B stored [N][K] is B^T as it stands: its tiles land by TMA directly where the lo parts belong, in the layout the MMA
+// reads; B stored [K][N] passes through two buffers borrowed from the still idle ring and is transposed by the threads.
+//
 // Roles per CTA (320 threads): warp 0 TMA producer, warp 1 MMA issuer (leader CTA), warps 2-9 first split B^T (thread =
 // row n = TMEM lane); then warps 2-5 export and warps 6-9 split the A stages.  Every wait is bounded.
 #pragma once
@@ -107,8 +110,11 @@ __device__ __forceinline__ void ws_tmem_st_32x32(uint32_t taddr, const uint32_t 
 }
 __device__ __forceinline__ void ws_tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// tmA: A as [M][K] fp32, box 32 k x 64 rows, 128-byte swizzle.  tmW: B as [K][N] fp32, box 32 n x 64 k, no swizzle.
-// tmC: C as [M][N] fp32, box 32 n x 16 rows, no swizzle.
+// tmA: A as [M][K] fp32, box 32 k x 64 rows, 128-byte swizzle.  tmC: C as [M][N] fp32, box 32 n x 16 rows, no swizzle.
+// tmW: B stored [K][N] (B_NK = false): box 32 n x 64 k, no swizzle; B stored [N][K] (B_NK = true: B^T as it is in memory):
+// box 32 k x 128 n, 128-byte swizzle -- the tiles then land in the layout the MMA reads, and the lo parts replace them
+// in place.
+template <bool B_NK>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WS_THREADS, 1)
 umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                       const __grid_constant__ CUtensorMap tmC, const WsParams p) {
@@ -171,7 +177,25 @@ umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         const int q = warp & 3;                  // TMEM lane quarter this warp may access
         const int n_loc = q * 32 + lane;
         const uint32_t lane_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-        for (int qi = 0; qi < 4; ++qi) {
+        if constexpr (B_NK) {
+            // all eight slabs landed in place (row n at n * 128, 16-byte chunks permuted by n % 8): hi parts out, lo parts over them
+            if (!ws_wait(&ctl->w_full[0], 0, ctl, p.status, 8)) return false;
+            for (int j = part; j < WS_KMAX / WS_BK; j += 2) {
+                uint8_t* row = w_lo + j * (128 * 128) + n_loc * 128;
+                uint32_t hi[32];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint4* ptr = reinterpret_cast<uint4*>(row + ((c ^ (n_loc & 7)) << 4));
+                    const uint4 x = *ptr;
+                    hi[4 * c] = x.x & 0xFFFFE000u; hi[4 * c + 1] = x.y & 0xFFFFE000u;
+                    hi[4 * c + 2] = x.z & 0xFFFFE000u; hi[4 * c + 3] = x.w & 0xFFFFE000u;
+                    *ptr = make_uint4(ws_lo(x.x), ws_lo(x.y), ws_lo(x.z), ws_lo(x.w));
+                }
+                ws_tmem_st_32x32(lane_taddr + static_cast<uint32_t>(j * WS_BK), hi);
+            }
+            ws_tmem_st_wait();
+        }
+        for (int qi = 0; qi < (B_NK ? 0 : 4); ++qi) {
             const int b = qi & 1;
             if (!ws_wait(&ctl->w_full[b], (qi >> 1) & 1, ctl, p.status, 8)) return false;
             // landed: box c = n_loc / 32 holds 64 rows k (128 B each) of 32 columns n
@@ -212,7 +236,14 @@ umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             ptx::grid_dependency_wait();  // the set-up above may overlap the previous kernel; nothing it wrote is read before it ends
             // B^T, this CTA's 128 columns n, in four quarters of k through two buffers in the (still idle) ring
             int wq = 0;   // quarters requested
-            for (int qi = 0; qi < 4 && ok; ++qi) {
+            if constexpr (B_NK) {   // B^T as stored: straight into its place, the ring stays free
+                wq = 1;
+                ptx::mbar_arrive_expect_tx(&ctl->w_full[0], WS_WLO_BYTES);
+#pragma unroll
+                for (int j = 0; j < WS_KMAX / WS_BK; ++j)
+                    ptx::tma_load_3d(w_lo + j * (128 * 128), &tmW, &ctl->w_full[0], j * WS_BK, static_cast<int>(rank) * 128, 0);
+            }
+            for (int qi = 0; qi < (B_NK ? 0 : 4) && ok; ++qi) {
                 const int b = qi & 1;
                 if (qi >= 2 && !ws_wait(&ctl->w_free[b], 0, ctl, p.status, 1)) { ok = false; break; }
                 ++wq;
@@ -221,7 +252,7 @@ umma_ws_tf32x3_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 for (int c = 0; c < 4; ++c)
                     ptx::tma_load_3d(ring + b * WS_TEMP_BYTES + c * (64 * 128), &tmW, &ctl->w_full[b], static_cast<int>(rank) * 128 + c * 32, qi * 64, 0);
             }
-            for (int b = 0; b < 2 && ok; ++b)   // the ring is the ring again
+            for (int b = 0; b < (B_NK ? 0 : 2) && ok; ++b)   // the ring is the ring again
                 if (!ws_wait(&ctl->w_free[b], 1, ctl, p.status, 2)) ok = false;
             int stage = 0;
             uint32_t phase = 0;

@@ -152,7 +152,7 @@ def test_kernel_selection(binding):
     assert k(1, 256, 256, 8192, "bf16", fixed_k_order=True) == "tcgen05_pair"
     assert k(1, 256, 256, 512, "bf16") == "tcgen05_pair"         # k loop too short to cut
     assert k(1, 65536, 256, 256, "f32") == "tcgen05_3xtf32_ws"   # small B under a long A: B stays in tensor memory
-    assert k(1, 65536, 256, 256, "f32", b_col_major=True) == "tcgen05_3xtf32"
+    assert k(1, 65536, 256, 256, "f32", b_col_major=True) == "tcgen05_3xtf32_ws"
     assert k(1, 65536, 256, 512, "f32") == "tcgen05_3xtf32"      # B too large to stay
     assert k(1, 4096, 256, 256, "f32") == "tcgen05_3xtf32"       # too few rows to pay for the prologue
     assert k(4, 65536, 256, 256, "f32") == "tcgen05_3xtf32"

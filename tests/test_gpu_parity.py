@@ -91,10 +91,13 @@ def test_fp32_split_tf32_on_tensor_cores(shape, col):
 
 @pytest.mark.parametrize("shape", [(18944, 256, 256), (20001, 256, 256), (19000, 200, 256), (19500, 132, 100), (18944, 256, 32),
                                    (30000, 252, 36), (19000, 128, 256), (21000, 64, 96), (19001, 100, 4), (19000, 4, 256), (19000, 20, 8)])
-def test_fp32_weight_stationary_on_tensor_cores(shape):
+@pytest.mark.parametrize("col", [False, True])
+def test_fp32_weight_stationary_on_tensor_cores(shape, col):
     """Small B under a long A: B^T split once and kept in tensor memory / shared memory, A streamed in 128-row tiles
-    (ragged last tile, ragged n and k included)."""
-    w = wl("f32", *shape, seed=43, col=False, fixed=False)
+    (ragged last tile, ragged n and k included; B stored [K][N] or [N][K])."""
+    if col and shape[2] % 4:
+        pytest.skip("row pitch of B stored [N][K] not a multiple of 16 bytes")
+    w = wl("f32", *shape, seed=43, col=col, fixed=False)
     assert family(w) == "tcgen05_3xtf32_ws"
     worst = check_workload(w, rows_per_problem=600)
     assert worst < 2e-6
