@@ -31,7 +31,9 @@
  * tail, one scratch per (device, stream) -- 19.4 MB for the matrix multiply, 21.3 MB for
  * attention, at most eight of each per device -- allocated the first time such a schedule
  * runs on a stream and kept until the process exits (a stream beyond the eighth, or one that
- * is being captured before it has a scratch, runs the schedule without a sliced tail).
+ * is being captured before it has a scratch, runs the schedule without a sliced tail).  A call
+ * captured into a CUDA graph keeps using the scratch of the stream it was captured on: replays
+ * of such graphs must not overlap one another.
  *
  * Layouts.  A is [M][K] row-major (K contiguous).  B is [K][N] row-major, or,
  * with CYC_FLAG_B_COL_MAJOR, stored as [N][K] (element B_kj at B[j*K + k]).
