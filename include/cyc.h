@@ -225,6 +225,11 @@ int cyc_block_trsm(int64_t n, int64_t m, int64_t tile, int dtype, const void* L,
  *   flags  0 (the paper's recurrence has no mask and no other scale)
  * N, M >= 1 need not be multiples of the tile sizes (128 queries, 128 keys).  Asynchronous on
  * `stream`; the caller owns all buffers; errors as for cyc_recurrence_matmul.
+ * Results are run-to-run identical for the same arguments on the same stream.  Where the last
+ * round of the grid is cut by key range (see "Device memory" above) the parts round their
+ * exponentials against their own reference maxima, so a call that runs without that cut (a
+ * stream without scratch, a capture on such a stream) agrees with one that runs with it to the
+ * bf16 rounding of the exponentials, not bit for bit.
  */
 int cyc_flash_attention(int64_t batch, int64_t N, int64_t M, int64_t d, int dtype, const void* Q, const void* K, const void* V,
                         void* O, void* stream, unsigned flags);
