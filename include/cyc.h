@@ -53,7 +53,11 @@
  *                 other that is exactly zero); the flag gives IEEE results.
  *   CYC_BF16_F32  A, B bfloat16; products exact; fp32 accumulation; C float.
  *                 k-blocks are accumulated in increasing order; results are
- *                 run-to-run identical with or without the flag (no atomics).
+ *                 run-to-run identical with or without the flag (no atomics) for
+ *                 the same arguments on the same stream.  Without the flag the
+ *                 grouping of the fp32 additions follows the schedule (k-slices,
+ *                 sliced tail), so a call on a stream that runs another schedule
+ *                 (see "Device memory" above) may differ in the last bits.
  *                 Without the flag, problems with few output tiles and a long k
  *                 loop are cut into k-slices whose partial sums are added in
  *                 slice order (split-K; needs a workspace from a stream-ordered
